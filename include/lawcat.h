@@ -1,0 +1,167 @@
+/*
+ * lawcat.h -- C ABI of the LAWCAT linearized-attention layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer (paper Section 4, Fig. 1):
+ *   1. causal depthwise Conv1D across tokens, width conv_k = r+1, on the query and on the key stream,
+ *      separate weights per stream (Section 4.1; appendix "share the linear and Conv layers");
+ *   2. one shared per-head linear layer followed by a nonlinearity -- the feature map phi -- applied to both
+ *      conv outputs, giving qdot and kdot (Section 4.1, Section 4.2 first paragraph);
+ *   3. normalized gated linear attention: S_t = G_t (.) S_{t-1} + kdot_t^T v_t (Eq. 4), output
+ *      o_t = qdot_t S_t / (qdot_t . z_t) with z_t the same recurrence on kdot_t alone (Eq. 8).
+ *
+ * Conventions shared by every entry point
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, contiguous in the stated shape with the
+ *     last index fastest, and 16-byte aligned. The library never allocates, frees or synchronizes; work is
+ *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - `p->dtype` is the storage type of q, k, v, gate, the conv and mix weights, the conv caches, qdot, kdot,
+ *     o and the input gradients: float (LAWCAT_F32) or bfloat16 (LAWCAT_BF16). All arithmetic accumulates
+ *     in fp32. States S, z, the denominator `den` and all weight gradients are always fp32.
+ *   - Heads: H query heads, H_kv key/value heads, H % H_kv == 0, G = H / H_kv. Query head h reads key and
+ *     value head h / G. kdot, the gate and the state are per QUERY head because the mix weights are.
+ *   - Gate: gate[b,t,h,:] has gate_dim = d_k entries (one decay per key channel) or 1 (one per head).
+ *     LAWCAT_GATE_LOGITS: log-decay g = logsigmoid(gate) / gate_tau ("sigmoid" gate of Section 4.2);
+ *     LAWCAT_GATE_LOGDECAY: g = gate itself, which must be <= 0. The decay is alpha = exp(g) in (0, 1].
+ *     Token t's decay multiplies S_{t-1}; it never touches token t's own kdot_t^T v_t (J_{t,t} = 1, Eq. 6).
+ *   - Conv taps: w[(head*d_k + c)*conv_k + delta] multiplies x[t - delta], delta = 0 is the current token.
+ *     Rows with t - delta < 0 come from the conv cache when one is given, otherwise they are zero.
+ *     A conv cache holds the conv_k-1 raw (pre-conv) tokens that precede t = 0, oldest first.
+ *   - Mix: y[e] = sum_c u[c] * W[h][c][e]; the same W[h] serves the query stream and the key stream.
+ *   - A NULL optional input means "absent" (zero state, zero cache); a NULL optional output is not written.
+ *   - `ws` is caller-provided scratch of at least lawcat_workspace_bytes(p, op) bytes (may be NULL when 0).
+ *   - Return value: a lawcat_status. Argument problems are detected on the host before anything is enqueued.
+ *     `dev_status` (optional device int, caller-zeroed) receives a nonzero lawcat_status if a kernel had to
+ *     give up asynchronously (a bounded wait that ran out); kernels never trap.
+ *   - Supported shapes: 16 <= d_k, d_v <= 128 and multiples of 16; 1 <= conv_k <= 8; gate_dim in {1, d_k}.
+ *     Anything else returns LAWCAT_ERR_UNSUPPORTED; nothing falls back to the host.
+ */
+#ifndef LAWCAT_H_
+#define LAWCAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LAWCAT_OK = 0,
+  LAWCAT_ERR_INVALID_ARG = 1,
+  LAWCAT_ERR_UNSUPPORTED = 2,
+  LAWCAT_ERR_CUDA = 3,
+  LAWCAT_ERR_WORKSPACE_TOO_SMALL = 4,
+  LAWCAT_ERR_TIMEOUT = 5,
+  LAWCAT_ERR_NUMERIC = 6
+} lawcat_status;
+
+enum { LAWCAT_F32 = 0, LAWCAT_BF16 = 1 };
+enum { LAWCAT_PHI_SOFTMAX = 0, LAWCAT_PHI_ELU1 = 1, LAWCAT_PHI_IDENTITY = 2 };
+enum { LAWCAT_GATE_LOGITS = 0, LAWCAT_GATE_LOGDECAY = 1 };
+enum {
+  LAWCAT_OP_CONV_FWD = 0,
+  LAWCAT_OP_CONV_BWD = 1,
+  LAWCAT_OP_GLA_FWD = 2,
+  LAWCAT_OP_GLA_BWD = 3,
+  LAWCAT_OP_LAYER_FWD = 4,
+  LAWCAT_OP_DECODE_STEP = 5
+};
+
+typedef struct {
+  int32_t B, T, H, H_kv, d_k, d_v;
+  int32_t conv_k;    /* conv width r+1 (the paper uses 4, Section 4.1) */
+  int32_t gate_dim;  /* d_k or 1 */
+  int32_t chunk;     /* tokens per chunk of the chunkwise-parallel form; 0 = library chooses */
+  int32_t dtype;     /* LAWCAT_F32 | LAWCAT_BF16 */
+  int32_t phi;       /* LAWCAT_PHI_* : softmax over the d_k mix outputs, 1+ELU (Section 2), identity */
+  int32_t gate_mode; /* LAWCAT_GATE_* */
+  float gate_tau;    /* divisor of logsigmoid in LOGITS mode; 1 = the plain sigmoid gate */
+  float eps;         /* added to the denominator of Eq. 8 */
+  int32_t normalize; /* 1 = Eq. 8; 0 = numerator only (the "NN" ablation, Table 2) */
+} lawcat_params;
+
+/* Scratch bytes entry point `op` (LAWCAT_OP_*) needs for these parameters; 0 on invalid parameters. */
+size_t lawcat_workspace_bytes(const lawcat_params* p, int op);
+
+/* Static, human-readable name of a status code. */
+const char* lawcat_status_string(int status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int lawcat_version(void);
+
+/*
+ * Causal depthwise conv on q and k (Section 4.1: qtilde_t = sum_delta w_delta q_{t-delta}), then, when W is not
+ * NULL, the shared per-head linear layer and phi (Section 4.1; Section 4.2 defines qdot, kdot).
+ *   q [B,T,H,d_k]  k [B,T,H_kv,d_k]  w_q [H*d_k,conv_k]  w_k [H_kv*d_k,conv_k]  W [H,d_k,d_k] or NULL
+ *   cache_q [B,conv_k-1,H*d_k], cache_k [B,conv_k-1,H_kv*d_k]  (nullable)
+ *   out, W != NULL: qdot [B,T,H,d_k], kdot [B,T,H,d_k]   (kdot per query head: phi uses W[h])
+ *   out, W == NULL: qdot = conv(q) [B,T,H,d_k], kdot = conv(k) [B,T,H_kv,d_k]
+ */
+int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const void* w_q, const void* w_k,
+                    const void* W, const void* cache_q, const void* cache_k, void* qdot, void* kdot, void* ws,
+                    size_t ws_bytes, void* stream, int* dev_status);
+
+/*
+ * Backward of lawcat_conv_fwd (needed by the layer-wise distillation of Section 5.1; the paper prints no formulas,
+ * this is the chain rule on conv -> mix -> phi). d_qdot, d_kdot have the shapes of the forward outputs.
+ *   out: dq [B,T,H,d_k], dk [B,T,H_kv,d_k] in p->dtype; dw_q, dw_k, dW in fp32, shaped like w_q, w_k, W.
+ * Weight gradients are overwritten, not accumulated. dW must be NULL exactly when W is NULL. Any output may be NULL.
+ */
+int lawcat_conv_bwd(const lawcat_params* p, const void* q, const void* k, const void* w_q, const void* w_k,
+                    const void* W, const void* cache_q, const void* cache_k, const void* d_qdot,
+                    const void* d_kdot, void* dq, void* dk, float* dw_q, float* dw_k, float* dW, void* ws,
+                    size_t ws_bytes, void* stream, int* dev_status);
+
+/*
+ * Normalized gated linear attention on given feature-mapped streams (Eq. 4 - Eq. 8).
+ *   qdot, kdot [B,T,H,d_k]  v [B,T,H_kv,d_v]  gate [B,T,H,gate_dim]
+ *   S0 [B,H,d_k,d_v] fp32, z0 [B,H,d_k] fp32: state before token 0 (nullable = zero, Eq. 5)
+ *   out: o [B,T,H,d_v]; den [B,T,H] fp32 = qdot_t . z_t + eps (nullable; gla_bwd needs it);
+ *        S_T, z_T = state after the last token (nullable)
+ */
+int lawcat_gla_fwd(const lawcat_params* p, const void* qdot, const void* kdot, const void* v, const void* gate,
+                   const float* S0, const float* z0, void* o, float* den, float* S_T, float* z_T, void* ws,
+                   size_t ws_bytes, void* stream, int* dev_status);
+
+/*
+ * Backward of lawcat_gla_fwd for an upstream gradient dO [B,T,H,d_v] (distillation step, Section 5.1; chain rule
+ * on Eq. 4 and Eq. 8). o and den are the forward outputs.
+ *   out: d_qdot, d_kdot [B,T,H,d_k]; dv [B,T,H_kv,d_v] (summed over the G query heads of a group);
+ *        dgate [B,T,H,gate_dim] -- the gradient with respect to the `gate` input (logits or log-decays).
+ * No gradient flows into S0, z0 and none is taken from S_T, z_T.
+ */
+int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, const void* v, const void* gate,
+                   const float* S0, const float* z0, const void* o, const float* den, const void* dO,
+                   void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws, size_t ws_bytes, void* stream,
+                   int* dev_status);
+
+/*
+ * The whole layer forward, fused: conv -> mix -> phi -> normalized GLA (Fig. 1); the prefill path of Section 5.5.
+ * Inputs as in lawcat_conv_fwd (W required) and lawcat_gla_fwd. The conv caches and the state allow a long
+ * sequence to be processed in pieces (Section 4.1 on caching; streaming use in Section 6):
+ *   cache_q_out [B,conv_k-1,H*d_k], cache_k_out [B,conv_k-1,H_kv*d_k] = the last conv_k-1 raw tokens seen
+ *   (taken from the input caches when T < conv_k-1); S_T, z_T = the state after the last token. All nullable.
+ * The *_out buffers must not alias the *_in buffers.
+ */
+int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const void* v, const void* gate,
+                     const void* w_q, const void* w_k, const void* W, const void* cache_q_in,
+                     const void* cache_k_in, const float* S0, const float* z0, void* o, void* cache_q_out,
+                     void* cache_k_out, float* S_T, float* z_T, void* ws, size_t ws_bytes, void* stream,
+                     int* dev_status);
+
+/*
+ * One recurrent decode step for B sequences (p->T is ignored): the layer at a single token, using the conv cache
+ * of Section 4.1 and the constant-size state of Eq. 4.
+ *   q_t [B,H,d_k]  k_t [B,H_kv,d_k]  v_t [B,H_kv,d_v]  gate_t [B,H,gate_dim]
+ *   S [B,H,d_k,d_v], z [B,H,d_k] fp32 and cache_q, cache_k (layout as above) are REQUIRED and updated IN PLACE:
+ *   the state advances by one token, the caches drop their oldest row and append q_t, k_t.
+ *   out: o_t [B,H,d_v]
+ */
+int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t, const void* v_t,
+                       const void* gate_t, const void* w_q, const void* w_k, const void* W, float* S, float* z,
+                       void* cache_q, void* cache_k, void* o_t, void* ws, size_t ws_bytes, void* stream,
+                       int* dev_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAWCAT_H_ */

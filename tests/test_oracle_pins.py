@@ -1,0 +1,352 @@
+"""Pins of the fp64 CPU oracle against what the paper and the mathematics fix (no GPU involved).
+
+Each test compares the oracle with something that is not the oracle: a brute-force statement of a closed form the
+paper gives (Eq. 2, Eq. 6-8), a special case with a known answer, an invariant, a library routine, or finite
+differences of the oracle's own forward for the hand-derived backward.
+"""
+import numpy as np
+import pytest
+from scipy.special import softmax as sp_softmax
+
+from oracle import lawcat_oracle as O
+
+RNG = np.random.default_rng(20250918)
+
+
+def rnd(*shape):
+    return RNG.standard_normal(shape)
+
+
+def logsigmoid(a):
+    return -np.logaddexp(0.0, -a)
+
+
+# --------------------------------------------------------------------------- conv (Section 4.1)
+def brute_conv(x, w, cache, K):
+    B, T, NH, d = x.shape
+    C = NH * d
+    xf = x.reshape(B, T, C)
+    pre = np.zeros((B, K - 1, C)) if cache is None else cache
+    full = np.concatenate([pre, xf], axis=1)  # token t sits at row t + K - 1
+    out = np.zeros((B, T, C))
+    for t in range(T):
+        for delta in range(K):
+            out[:, t] += w[:, delta][None, :] * full[:, t + K - 1 - delta]
+    return out.reshape(B, T, NH, d)
+
+
+@pytest.mark.parametrize("T,K", [(1, 4), (3, 4), (9, 4), (17, 2), (6, 1), (12, 8)])
+def test_conv_direct_sum(T, K):
+    x, w = rnd(2, T, 3, 8), rnd(24, K)
+    np.testing.assert_allclose(O.conv(x, w, None, K), brute_conv(x, w, None, K), rtol=0, atol=1e-13)
+    cache = rnd(2, K - 1, 24)
+    np.testing.assert_allclose(O.conv(x, w, cache, K), brute_conv(x, w, cache, K), rtol=0, atol=1e-13)
+
+
+def test_conv_unit_taps_are_shifts():
+    x = rnd(1, 10, 2, 4)
+    for delta in range(4):
+        w = np.zeros((8, 4))
+        w[:, delta] = 1.0
+        y = O.conv(x, w, None, 4)
+        want = np.zeros_like(x)
+        want[:, delta:] = x[:, : 10 - delta]
+        assert np.array_equal(y, want)
+
+
+def test_conv_cache_equals_prepended_tokens():
+    K = 4
+    x, w = rnd(2, 11, 2, 4), rnd(8, K)
+    head, tail = x[:, : K - 1], x[:, K - 1:]
+    full = O.conv(x, w, None, K)
+    part = O.conv(tail, w, head.reshape(2, K - 1, 8), K)
+    np.testing.assert_allclose(part, full[:, K - 1:], rtol=0, atol=1e-14)
+
+
+def test_conv_linear_and_causal():
+    K = 4
+    x1, x2, w = rnd(1, 12, 2, 4), rnd(1, 12, 2, 4), rnd(8, K)
+    np.testing.assert_allclose(O.conv(2 * x1 - 3 * x2, w, None, K),
+                               2 * O.conv(x1, w, None, K) - 3 * O.conv(x2, w, None, K), atol=1e-13)
+    x3 = x1.copy()
+    x3[:, 7:] += rnd(1, 5, 2, 4)
+    assert np.array_equal(O.conv(x3, w, None, K)[:, :7], O.conv(x1, w, None, K)[:, :7])
+
+
+# --------------------------------------------------------------------------- mix + phi (Section 4.1)
+def test_mix_identity_passthrough():
+    u = rnd(2, 5, 3, 8)
+    W = np.broadcast_to(np.eye(8), (3, 8, 8)).copy()
+    assert np.array_equal(O.mix_phi(u, W, 3, O.PHI_IDENTITY), u)
+
+
+def test_mix_against_library_routines():
+    u, W = rnd(2, 7, 2, 8), rnd(4, 8, 8)
+    y = np.einsum("btnc,nce->btne", np.repeat(u, 2, axis=2), W)  # head h reads input head h // 2
+    np.testing.assert_allclose(O.mix_phi(u, W, 4, O.PHI_IDENTITY), y, atol=1e-13)
+    np.testing.assert_allclose(O.mix_phi(u, W, 4, O.PHI_SOFTMAX), sp_softmax(y, axis=-1), atol=1e-14)
+    np.testing.assert_allclose(O.mix_phi(u, W, 4, O.PHI_ELU1), np.where(y > 0, y + 1, np.exp(y)), atol=1e-14)
+
+
+def test_softmax_phi_positive_and_normalised():
+    p = O.mix_phi(5 * rnd(1, 9, 2, 16), rnd(2, 16, 16), 2, O.PHI_SOFTMAX)
+    assert (p > 0).all()
+    np.testing.assert_allclose(p.sum(-1), 1.0, atol=1e-14)
+
+
+def test_same_map_for_query_and_key():
+    # identical conv outputs pushed through the shared layer give identical features (Section 4.1)
+    u, W = rnd(1, 6, 2, 8), rnd(2, 8, 8)
+    assert np.array_equal(O.mix_phi(u, W, 2), O.mix_phi(u.copy(), W, 2))
+
+
+# --------------------------------------------------------------------------- GLA forward (Eq. 4 - Eq. 8)
+def quadratic_form(qd, kd, v, alpha, normalize=True):
+    """Eq. 8 for one head with J_{i,t} built as an explicit running product of the gates (Eq. 6)."""
+    T, dk = qd.shape
+    o = np.zeros((T, v.shape[1]))
+    den = np.zeros(T)
+    for t in range(T):
+        num = np.zeros(v.shape[1])
+        dn = 0.0
+        for i in range(t + 1):
+            J = np.ones(dk)
+            for zz in range(i + 1, t + 1):
+                J = J * alpha[zz]
+            wti = np.sum(qd[t] * J * kd[i])
+            num += wti * v[i]
+            dn += wti
+        o[t] = num / dn if normalize else num
+        den[t] = dn
+    return o, den
+
+
+@pytest.mark.parametrize("gate_dim,T", [(0, 1), (0, 13), (1, 24), (0, 40)])
+def test_recurrence_equals_quadratic_form(gate_dim, T):
+    H, dk, dv = 2, 6, 5
+    p = O.OracleParams(1, T, H, H, dk, dv, gate_dim=gate_dim, gate_tau=2.0)
+    qd, kd = np.abs(rnd(1, T, H, dk)), np.abs(rnd(1, T, H, dk))
+    v, a = rnd(1, T, H, dv), 2 * rnd(1, T, H, p.gd)
+    r = O.gla_fwd(p, qd, kd, v, a)
+    alpha = np.broadcast_to(np.exp(logsigmoid(a) / 2.0), (1, T, H, dk))
+    for h in range(H):
+        o, den = quadratic_form(qd[0, :, h], kd[0, :, h], v[0, :, h], alpha[0, :, h])
+        np.testing.assert_allclose(r["o"][0, :, h], o, rtol=1e-11, atol=1e-13)
+        np.testing.assert_allclose(r["den"][0, :, h], den, rtol=1e-11)
+    # numerator-only variant
+    p0 = O.OracleParams(1, T, H, H, dk, dv, gate_dim=gate_dim, gate_tau=2.0, normalize=0)
+    r0 = O.gla_fwd(p0, qd, kd, v, a)
+    o0, _ = quadratic_form(qd[0, :, 1], kd[0, :, 1], v[0, :, 1], alpha[0, :, 1], normalize=False)
+    np.testing.assert_allclose(r0["o"][0, :, 1], o0, rtol=1e-11, atol=1e-13)
+
+
+def test_zero_decay_is_kernel_linear_attention():
+    # all gates 1 -> Eq. 2 by direct double sum
+    T, dk, dv = 19, 5, 4
+    p = O.OracleParams(1, T, 1, 1, dk, dv, gate_mode=O.GATE_LOGDECAY)
+    qd, kd, v = np.abs(rnd(1, T, 1, dk)), np.abs(rnd(1, T, 1, dk)), rnd(1, T, 1, dv)
+    r = O.gla_fwd(p, qd, kd, v, np.zeros((1, T, 1, dk)))
+    for t in range(T):
+        wts = np.array([qd[0, t, 0] @ kd[0, i, 0] for i in range(t + 1)])
+        want = (wts[:, None] * v[0, : t + 1, 0]).sum(0) / wts.sum()
+        np.testing.assert_allclose(r["o"][0, t, 0], want, rtol=1e-12, atol=1e-14)
+
+
+def test_total_decay_returns_current_value():
+    # alpha = 0: S_t = kdot_t^T v_t, so o_t = v_t exactly up to one rounding of the division
+    T, dk, dv = 9, 4, 6
+    p = O.OracleParams(1, T, 1, 1, dk, dv, gate_mode=O.GATE_LOGDECAY)
+    qd, kd, v = np.abs(rnd(1, T, 1, dk)), np.abs(rnd(1, T, 1, dk)), rnd(1, T, 1, dv)
+    r = O.gla_fwd(p, qd, kd, v, np.full((1, T, 1, dk), -1e9))
+    np.testing.assert_allclose(r["o"], v, rtol=1e-14)
+
+
+def test_normaliser_properties():
+    T, H, dk, dv = 30, 2, 8, 7
+    p = O.OracleParams(2, T, H, 1, dk, dv)
+    qd, kd = np.abs(rnd(2, T, H, dk)) + 0.1, np.abs(rnd(2, T, H, dk)) + 0.1
+    v, a = rnd(2, T, 1, dv), rnd(2, T, H, dk)
+    o = O.gla_fwd(p, qd, kd, v, a)["o"]
+    np.testing.assert_allclose(o[:, 0], np.repeat(v[:, 0], H, axis=1), rtol=1e-14)  # first output is v_1
+    vmin = np.minimum.accumulate(v, axis=1)
+    vmax = np.maximum.accumulate(v, axis=1)
+    assert (o >= vmin - 1e-12).all() and (o <= vmax + 1e-12).all()                 # convex combination of values
+    const = np.broadcast_to(rnd(1, 1, 1, dv), v.shape).copy()
+    oc = O.gla_fwd(p, qd, kd, const, a)["o"]
+    np.testing.assert_allclose(oc, np.broadcast_to(const[:, :, :1], oc.shape), rtol=1e-12)
+    o_scaled = O.gla_fwd(p, 3.7 * qd, kd, v, a)["o"]                               # scale of qdot cancels
+    np.testing.assert_allclose(o_scaled, o, rtol=1e-12, atol=1e-14)
+
+
+def test_causality_bitwise():
+    T, t0 = 21, 12
+    sh = dict(B=1, T=T, H=2, H_kv=1, d_k=8, d_v=8)
+    p = O.OracleParams(**sh)
+    q, k, v, a = rnd(1, T, 2, 8), rnd(1, T, 1, 8), rnd(1, T, 1, 8), rnd(1, T, 2, 8)
+    wq, wk, W = rnd(16, 4), rnd(8, 4), rnd(2, 8, 8)
+    base = O.layer_fwd(p, q, k, v, a, wq, wk, W)["o"]
+    q2, k2, v2, a2 = q.copy(), k.copy(), v.copy(), a.copy()
+    for x in (q2, k2, v2, a2):
+        x[:, t0 + 1:] += rnd(*x[:, t0 + 1:].shape)
+    pert = O.layer_fwd(p, q2, k2, v2, a2, wq, wk, W)["o"]
+    assert np.array_equal(base[:, : t0 + 1], pert[:, : t0 + 1])
+    assert not np.array_equal(base[:, t0 + 1:], pert[:, t0 + 1:])
+
+
+def _layer_inputs(B, T, H, Hkv, dk, dv, gd=0):
+    gd = gd or dk
+    return dict(q=rnd(B, T, H, dk), k=rnd(B, T, Hkv, dk), v=rnd(B, T, Hkv, dv), gate=rnd(B, T, H, gd),
+                w_q=rnd(H * dk, 4) / 2, w_k=rnd(Hkv * dk, 4) / 2, W=rnd(H, dk, dk) / np.sqrt(dk))
+
+
+@pytest.mark.parametrize("split", [1, 2, 3, 10])
+def test_split_calls_carry_state_and_caches(split):
+    B, T, H, Hkv, dk, dv = 2, 17, 4, 2, 8, 6
+    x = _layer_inputs(B, T, H, Hkv, dk, dv)
+    full = O.layer_fwd(O.OracleParams(B, T, H, Hkv, dk, dv), **x)
+    sl = lambda a, lo, hi: a[:, lo:hi]
+    r1 = O.layer_fwd(O.OracleParams(B, split, H, Hkv, dk, dv), sl(x["q"], 0, split), sl(x["k"], 0, split),
+                     sl(x["v"], 0, split), sl(x["gate"], 0, split), x["w_q"], x["w_k"], x["W"])
+    r2 = O.layer_fwd(O.OracleParams(B, T - split, H, Hkv, dk, dv), sl(x["q"], split, T), sl(x["k"], split, T),
+                     sl(x["v"], split, T), sl(x["gate"], split, T), x["w_q"], x["w_k"], x["W"],
+                     r1["cache_q"], r1["cache_k"], r1["S_T"], r1["z_T"])
+    np.testing.assert_allclose(np.concatenate([r1["o"], r2["o"]], 1), full["o"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(r2["S_T"], full["S_T"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(r2["z_T"], full["z_T"], rtol=1e-12)
+    assert np.array_equal(r2["cache_q"], full["cache_q"]) and np.array_equal(r2["cache_k"], full["cache_k"])
+    assert np.array_equal(full["cache_q"], x["q"][:, -3:].reshape(B, 3, -1))
+
+
+def test_decode_steps_equal_prefill():
+    B, T, H, Hkv, dk, dv = 2, 9, 4, 2, 8, 8
+    x = _layer_inputs(B, T, H, Hkv, dk, dv, gd=1)
+    p = O.OracleParams(B, T, H, Hkv, dk, dv, gate_dim=1)
+    full = O.layer_fwd(p, **x)
+    S, z = np.zeros((B, H, dk, dv)), np.zeros((B, H, dk))
+    cq, ck = np.zeros((B, 3, H * dk)), np.zeros((B, 3, Hkv * dk))
+    for t in range(T):
+        r = O.decode_step(p, x["q"][:, t], x["k"][:, t], x["v"][:, t], x["gate"][:, t], x["w_q"], x["w_k"],
+                          x["W"], S, z, cq, ck)
+        np.testing.assert_allclose(r["o"], full["o"][:, t], rtol=1e-12, atol=1e-14)
+        S, z, cq, ck = r["S"], r["z"], r["cache_q"], r["cache_k"]
+    np.testing.assert_allclose(S, full["S_T"], rtol=1e-12, atol=1e-14)
+
+
+def test_gqa_equals_mha_with_repeated_kv():
+    B, T, H, Hkv, dk, dv = 1, 11, 4, 2, 8, 8
+    x = _layer_inputs(B, T, H, Hkv, dk, dv)
+    a = O.layer_fwd(O.OracleParams(B, T, H, Hkv, dk, dv), **x)["o"]
+    y = dict(x)
+    y["k"] = np.repeat(x["k"], 2, axis=2)
+    y["v"] = np.repeat(x["v"], 2, axis=2)
+    y["w_k"] = np.repeat(x["w_k"].reshape(Hkv, dk, 4), 2, axis=0).reshape(H * dk, 4)
+    b = O.layer_fwd(O.OracleParams(B, T, H, H, dk, dv), **y)["o"]
+    np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-15)
+
+
+# --------------------------------------------------------------------------- gradients
+def _fd(fun, x, dO, h=1e-6):
+    """Central finite differences of sum(dO * fun(x)) with respect to every entry of x."""
+    g = np.zeros_like(x)
+    flat, gf = x.reshape(-1), g.reshape(-1)
+    for i in range(flat.size):
+        old = flat[i]
+        flat[i] = old + h
+        fp = np.sum(dO * fun())
+        flat[i] = old - h
+        fm = np.sum(dO * fun())
+        flat[i] = old
+        gf[i] = (fp - fm) / (2 * h)
+    return g
+
+
+@pytest.mark.parametrize("gate_dim,gate_mode,normalize,with_state",
+                         [(0, O.GATE_LOGITS, 1, False), (1, O.GATE_LOGITS, 1, True),
+                          (0, O.GATE_LOGDECAY, 1, True), (0, O.GATE_LOGITS, 0, False)])
+def test_gla_bwd_finite_differences(gate_dim, gate_mode, normalize, with_state):
+    B, T, H, Hkv, dk, dv = 1, 6, 2, 1, 4, 3
+    p = O.OracleParams(B, T, H, Hkv, dk, dv, gate_dim=gate_dim, gate_mode=gate_mode, normalize=normalize,
+                       gate_tau=2.0)
+    qd, kd = np.abs(rnd(B, T, H, dk)) + 0.2, np.abs(rnd(B, T, H, dk)) + 0.2
+    v, dO = rnd(B, T, Hkv, dv), rnd(B, T, H, dv)
+    a = rnd(B, T, H, p.gd)
+    if gate_mode == O.GATE_LOGDECAY:
+        a = -np.abs(a) * 0.3
+    S0 = np.abs(rnd(B, H, dk, dv)) if with_state else None
+    z0 = np.abs(rnd(B, H, dk)) + 0.5 if with_state else None
+    g = O.gla_bwd(p, qd, kd, v, a, dO, S0, z0)
+    f = lambda: O.gla_fwd(p, qd, kd, v, a, S0, z0)["o"]
+    for name, x in (("d_qdot", qd), ("d_kdot", kd), ("dv", v), ("dgate", a)):
+        np.testing.assert_allclose(g[name], _fd(f, x, dO), rtol=2e-6, atol=1e-8, err_msg=name)
+
+
+def test_gate_gradient_reverse_cumsum_identity():
+    # o' depends on the log-decays only through their running sum, hence
+    # dg_s = sum_{t>=s} (qdot_t * dqdot_t - kdot_t * dkdot_t)
+    B, T, H, dk, dv = 1, 12, 2, 5, 4
+    p = O.OracleParams(B, T, H, H, dk, dv, gate_mode=O.GATE_LOGDECAY)
+    qd, kd = np.abs(rnd(B, T, H, dk)) + 0.1, np.abs(rnd(B, T, H, dk)) + 0.1
+    v, dO, g_in = rnd(B, T, H, dv), rnd(B, T, H, dv), -np.abs(rnd(B, T, H, dk)) * 0.2
+    g = O.gla_bwd(p, qd, kd, v, g_in, dO)
+    per_t = qd * g["d_qdot"] - kd * g["d_kdot"]
+    want = np.flip(np.cumsum(np.flip(per_t, 1), 1), 1)
+    np.testing.assert_allclose(g["dgate"], want, rtol=1e-10, atol=1e-12)
+
+
+def test_value_shift_identity():
+    # v -> v + c shifts every o_t by c (weights sum to one), so sum_t dv = sum_{t,h} dO per value channel
+    B, T, H, Hkv, dk, dv = 2, 10, 4, 2, 4, 5
+    p = O.OracleParams(B, T, H, Hkv, dk, dv)
+    qd, kd = np.abs(rnd(B, T, H, dk)) + 0.1, np.abs(rnd(B, T, H, dk)) + 0.1
+    v, dO, a = rnd(B, T, Hkv, dv), rnd(B, T, H, dv), rnd(B, T, H, dk)
+    g = O.gla_bwd(p, qd, kd, v, a, dO)
+    want = dO.reshape(B, T, Hkv, 2, dv).sum(axis=(1, 3))  # per (b, kv head, channel)
+    np.testing.assert_allclose(g["dv"].sum(axis=1), want, rtol=1e-10, atol=1e-12)
+
+
+@pytest.mark.parametrize("phi,with_cache,with_mix",
+                         [(O.PHI_SOFTMAX, False, True), (O.PHI_ELU1, True, True), (O.PHI_IDENTITY, True, True),
+                          (O.PHI_SOFTMAX, True, False)])
+def test_conv_bwd_finite_differences(phi, with_cache, with_mix):
+    B, T, H, Hkv, d, K = 1, 5, 2, 1, 3, 3
+    p = O.OracleParams(B, T, H, Hkv, d, d, conv_k=K, phi=phi)
+    q, k = rnd(B, T, H, d), rnd(B, T, Hkv, d)
+    wq, wk = rnd(H * d, K), rnd(Hkv * d, K)
+    W = rnd(H, d, d) if with_mix else None
+    cq = rnd(B, K - 1, H * d) if with_cache else None
+    ck = rnd(B, K - 1, Hkv * d) if with_cache else None
+    dqd = rnd(B, T, H, d)
+    dkd = rnd(B, T, H if with_mix else Hkv, d)
+    g = O.conv_bwd(p, q, k, wq, wk, W, dqd, dkd, cq, ck)
+
+    def fq():
+        u = O.conv(q, wq, cq, K)
+        return O.mix_phi(u, W, H, phi) if with_mix else u
+
+    def fk():
+        u = O.conv(k, wk, ck, K)
+        return O.mix_phi(u, W, H, phi) if with_mix else u
+
+    np.testing.assert_allclose(g["dq"], _fd(fq, q, dqd), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(g["dk"], _fd(fk, k, dkd), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(g["dw_q"], _fd(fq, wq, dqd), rtol=2e-6, atol=1e-8)
+    np.testing.assert_allclose(g["dw_k"], _fd(fk, wk, dkd), rtol=2e-6, atol=1e-8)
+    if with_mix:
+        total = lambda: np.concatenate([fq().ravel(), fk().ravel()])
+        dboth = np.concatenate([dqd.ravel(), dkd.ravel()])
+        np.testing.assert_allclose(g["dW"], _fd(total, W, dboth), rtol=2e-6, atol=1e-8)
+
+
+def test_whole_layer_gradient_chain():
+    # composition gla_bwd -> conv_bwd against finite differences of the whole layer forward
+    B, T, H, Hkv, d = 1, 5, 2, 1, 3
+    p = O.OracleParams(B, T, H, Hkv, d, d, gate_tau=1.0)
+    x = _layer_inputs(B, T, H, Hkv, d, d)
+    dO = rnd(B, T, H, d)
+    fwd = O.layer_fwd(p, **x)
+    g1 = O.gla_bwd(p, fwd["qdot"], fwd["kdot"], x["v"], x["gate"], dO)
+    g2 = O.conv_bwd(p, x["q"], x["k"], x["w_q"], x["w_k"], x["W"], g1["d_qdot"], g1["d_kdot"])
+    f = lambda: O.layer_fwd(p, **x)["o"]
+    for name, got in (("q", g2["dq"]), ("k", g2["dk"]), ("v", g1["dv"]), ("gate", g1["dgate"]),
+                      ("w_q", g2["dw_q"]), ("w_k", g2["dw_k"]), ("W", g2["dW"])):
+        np.testing.assert_allclose(got, _fd(f, x[name], dO), rtol=5e-6, atol=1e-8, err_msg=name)
