@@ -31,7 +31,7 @@
  *   - Return value: a lawcat_status. Argument problems are detected on the host before anything is enqueued.
  *     `dev_status` (optional device int, caller-zeroed) receives a nonzero lawcat_status if a kernel had to
  *     give up asynchronously (a bounded wait that ran out); kernels never trap.
- *   - Supported shapes: 16 <= d_k, d_v <= 128 and multiples of 16; 1 <= conv_k <= 8; gate_dim in {1, d_k}.
+ *   - Supported shapes: d_k and d_v in {16, 32, 64, 128}; 1 <= conv_k <= 8; gate_dim in {1, d_k}.
  *     Anything else returns LAWCAT_ERR_UNSUPPORTED; nothing falls back to the host.
  */
 #ifndef LAWCAT_H_
@@ -104,7 +104,7 @@ int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const 
  * Backward of lawcat_conv_fwd (needed by the layer-wise distillation of Section 5.1; the paper prints no formulas,
  * this is the chain rule on conv -> mix -> phi). d_qdot, d_kdot have the shapes of the forward outputs.
  *   out: dq [B,T,H,d_k], dk [B,T,H_kv,d_k] in p->dtype; dw_q, dw_k, dW in fp32, shaped like w_q, w_k, W.
- * Weight gradients are overwritten, not accumulated. dW must be NULL exactly when W is NULL. Any output may be NULL.
+ * Weight gradients are overwritten, not accumulated. dW must be NULL when W is NULL. Any output may be NULL.
  */
 int lawcat_conv_bwd(const lawcat_params* p, const void* q, const void* k, const void* w_q, const void* w_k,
                     const void* W, const void* cache_q, const void* cache_k, const void* d_qdot,
@@ -124,7 +124,8 @@ int lawcat_gla_fwd(const lawcat_params* p, const void* qdot, const void* kdot, c
 
 /*
  * Backward of lawcat_gla_fwd for an upstream gradient dO [B,T,H,d_v] (distillation step, Section 5.1; chain rule
- * on Eq. 4 and Eq. 8). o and den are the forward outputs.
+ * on Eq. 4 and Eq. 8). o and den (the forward outputs) are accepted for symmetry and may be NULL: the backward
+ * recomputes the denominator and dO.o in fp32, because the stored o is rounded to the storage type.
  *   out: d_qdot, d_kdot [B,T,H,d_k]; dv [B,T,H_kv,d_v] (summed over the G query heads of a group);
  *        dgate [B,T,H,gate_dim] -- the gradient with respect to the `gate` input (logits or log-decays).
  * No gradient flows into S0, z0 and none is taken from S_T, z_T.

@@ -1,0 +1,75 @@
+// Shared device/host helpers of the LAWCAT CUDA library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lawcat.h"
+
+namespace lawcat {
+
+typedef __nv_bfloat16 bf16;
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p);
+template <> __device__ __forceinline__ float ldf<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ldf<bf16>(const bf16* p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void stf(T* p, float v);
+template <> __device__ __forceinline__ void stf<float>(float* p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<bf16>(bf16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+// Log-decay of one gate entry (Section 4.2: sigmoid gate). LOGITS: logsigmoid(a) / tau, LOGDECAY: a itself.
+__device__ __forceinline__ float log_decay(float a, int gate_mode, float inv_tau) {
+  if (gate_mode == LAWCAT_GATE_LOGDECAY) return a;
+  float ls = fminf(a, 0.f) - log1pf(expf(-fabsf(a)));
+  return ls * inv_tau;
+}
+// d(log-decay)/d(gate entry)
+__device__ __forceinline__ float log_decay_grad(float a, int gate_mode, float inv_tau) {
+  if (gate_mode == LAWCAT_GATE_LOGDECAY) return 1.f;
+  return (1.f - 1.f / (1.f + expf(-a))) * inv_tau;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- host-side launchers implemented in the .cu files (all return a lawcat_status) -------------------------------
+struct Ctx {
+  const lawcat_params* p;
+  cudaStream_t stream;
+  int* dev_status;
+};
+
+int launch_conv_plain(const Ctx& c, const void* x, const void* w, const void* cache, void* out, int NH);
+int launch_convmix_fwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
+                       const void* cache_q, const void* cache_k, void* qdot, void* kdot, bool out_f32);
+int launch_conv_bwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
+                    const void* cache_q, const void* cache_k, const void* d_qdot, const void* d_kdot, void* dq,
+                    void* dk, float* dw_q, float* dw_k, float* dW, void* ws);
+int launch_cache_out(const Ctx& c, const void* q, const void* k, const void* cache_q_in, const void* cache_k_in,
+                     void* cache_q_out, void* cache_k_out);
+int launch_gla_fwd_rec(const Ctx& c, const void* qdot, const void* kdot, bool qk_f32, const void* v,
+                       const void* gate, const float* S0, const float* z0, void* o, float* den, float* S_T,
+                       float* z_T);
+int launch_gla_bwd_rec(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate,
+                       const float* S0, const float* z0, const void* o, const float* den, const void* dO,
+                       void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws);
+int launch_decode(const Ctx& c, const void* q_t, const void* k_t, const void* v_t, const void* gate_t,
+                  const void* w_q, const void* w_k, const void* W, float* S, float* z, void* cache_q, void* cache_k,
+                  void* o_t);
+
+#define LAWCAT_CHECK_LAUNCH()                                 \
+  do {                                                        \
+    if (cudaGetLastError() != cudaSuccess) return LAWCAT_ERR_CUDA; \
+  } while (0)
+
+}  // namespace lawcat
