@@ -89,6 +89,18 @@ const char* lawcat_status_string(int status);
 int lawcat_version(void);
 
 /*
+ * Profiling aids (the paper has no counterpart; its only timing is an end-to-end latency plot, Section 5.5).
+ * lawcat_launch_count: kernels this library has launched in this process so far (monotonic, host counter).
+ * lawcat_trace_begin:  from now on bracket every kernel launch with a pair of CUDA events on its stream.
+ * lawcat_trace_end:    stop tracing, wait for the recorded events (this call synchronizes on them) and write one line
+ *                      per kernel, "<name> <launches> <total milliseconds>\n", into the HOST buffer buf (NUL-terminated,
+ *                      truncated to buf_bytes). Tracing creates CUDA events; it is meant for benchmarks, not serving.
+ */
+unsigned long long lawcat_launch_count(void);
+int lawcat_trace_begin(void);
+int lawcat_trace_end(char* buf, size_t buf_bytes);
+
+/*
  * Causal depthwise conv on q and k (Section 4.1: qtilde_t = sum_delta w_delta q_{t-delta}), then, when W is not
  * NULL, the shared per-head linear layer and phi (Section 4.1; Section 4.2 defines qdot, kdot).
  *   q [B,T,H,d_k]  k [B,T,H_kv,d_k]  w_q [H*d_k,conv_k]  w_k [H_kv*d_k,conv_k]  W [H,d_k,d_k] or NULL
@@ -161,6 +173,18 @@ int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t,
                        const void* gate_t, const void* w_q, const void* w_k, const void* W, float* S, float* z,
                        void* cache_q, void* cache_k, void* o_t, void* ws, size_t ws_bytes, void* stream,
                        int* dev_status);
+
+/*
+ * The layer forward of Fig. 1 for callers whose tensors live in HOST memory (pinned memory makes the copies
+ * asynchronous). h_* are host pointers laid out like the device tensors of lawcat_layer_fwd (no caches, zero initial
+ * state); `arena` is caller-owned DEVICE scratch of at least lawcat_layer_fwd_host_arena_bytes(p) bytes that receives
+ * the inputs, the output and the workspace. Enqueues on `stream`: host-to-device copies, the layer, the copy of o back
+ * to h_o. Returns without synchronizing; h_o is valid once the stream has drained.
+ */
+size_t lawcat_layer_fwd_host_arena_bytes(const lawcat_params* p);
+int lawcat_layer_fwd_host(const lawcat_params* p, const void* h_q, const void* h_k, const void* h_v,
+                          const void* h_gate, const void* h_w_q, const void* h_w_k, const void* h_W, void* h_o,
+                          void* arena, size_t arena_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -20,8 +20,10 @@ PHI_SOFTMAX, PHI_ELU1, PHI_IDENTITY = 0, 1, 2
 GATE_LOGITS, GATE_LOGDECAY = 0, 1
 OP_CONV_FWD, OP_CONV_BWD, OP_GLA_FWD, OP_GLA_BWD, OP_LAYER_FWD, OP_DECODE_STEP = range(6)
 
-EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "lawcat_conv_fwd", "lawcat_conv_bwd",
-           "lawcat_gla_fwd", "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_decode_step"]
+EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "lawcat_launch_count",
+           "lawcat_trace_begin", "lawcat_trace_end", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
+           "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
+           "lawcat_layer_fwd_host"]
 
 
 class LawcatError(RuntimeError):
@@ -63,6 +65,13 @@ def lib() -> ctypes.CDLL:
         L.lawcat_status_string.restype = ctypes.c_char_p
         L.lawcat_status_string.argtypes = [ctypes.c_int]
         L.lawcat_version.restype = ctypes.c_int
+        L.lawcat_launch_count.restype = ctypes.c_ulonglong
+        L.lawcat_layer_fwd_host_arena_bytes.restype = ctypes.c_size_t
+        L.lawcat_layer_fwd_host_arena_bytes.argtypes = [ctypes.POINTER(Params)]
+        L.lawcat_layer_fwd_host.restype = ctypes.c_int
+        L.lawcat_layer_fwd_host.argtypes = [ctypes.POINTER(Params)] + [ctypes.c_void_p] * 9 + \
+                                           [ctypes.c_size_t, ctypes.c_void_p]
+        L.lawcat_trace_end.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
         for name, nptr in (("lawcat_conv_fwd", 9), ("lawcat_conv_bwd", 14), ("lawcat_gla_fwd", 10),
                            ("lawcat_gla_bwd", 13), ("lawcat_layer_fwd", 16), ("lawcat_decode_step", 12)):
             f = getattr(L, name)
@@ -75,6 +84,27 @@ def lib() -> ctypes.CDLL:
 
 def status_string(status: int) -> str:
     return lib().lawcat_status_string(status).decode()
+
+
+def launch_count() -> int:
+    return int(lib().lawcat_launch_count())
+
+
+def trace_begin() -> None:
+    lib().lawcat_trace_begin()
+
+
+def trace_end() -> dict:
+    """Stop tracing; returns {kernel name: (launches, total device milliseconds)}."""
+    buf = ctypes.create_string_buffer(1 << 16)
+    st = lib().lawcat_trace_end(buf, len(buf))
+    if st != 0:
+        raise LawcatError(st, "lawcat_trace_end")
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, n, ms = line.split()
+        out[name] = (int(n), float(ms))
+    return out
 
 
 def workspace_bytes(p: Params, op: int) -> int:
@@ -183,6 +213,21 @@ def lawcat_decode_step(p: Params, q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cach
     _call("lawcat_decode_step", p, [q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cache_q, cache_k, o_t], ws, nb, stream,
           dev_status)
     return o_t
+
+
+def lawcat_layer_fwd_host(p: Params, h_q, h_k, h_v, h_gate, h_w_q, h_w_k, h_W, h_o, arena, stream=None):
+    """Host tensors in (pinned for asynchronous copies), host tensor h_o out; `arena` is a CUDA uint8 tensor of at
+    least ``lawcat_layer_fwd_host_arena_bytes`` bytes. Enqueues copies + layer + copy back; does not synchronize."""
+    hp = lambda t: ctypes.c_void_p(t.data_ptr())
+    st = lib().lawcat_layer_fwd_host(ctypes.byref(p), *[hp(t) for t in (h_q, h_k, h_v, h_gate, h_w_q, h_w_k, h_W, h_o)],
+                                     _ptr(arena), arena.numel(), _stream(stream))
+    if st != 0:
+        raise LawcatError(st, "lawcat_layer_fwd_host")
+    return h_o
+
+
+def host_arena_bytes(p: Params) -> int:
+    return int(lib().lawcat_layer_fwd_host_arena_bytes(ctypes.byref(p)))
 
 
 def to_device(x, dtype, device="cuda"):

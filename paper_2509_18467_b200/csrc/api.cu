@@ -172,4 +172,58 @@ int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t,
   return launch_decode(c, q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cache_q, cache_k, o_t);
 }
 
+// ---- host-buffer variant of the layer forward ---------------------------------------------------------------------
+static size_t host_arena_layout(const lawcat_params* p, size_t off[10]) {
+  const size_t es = p->dtype == LAWCAT_F32 ? 4 : 2;
+  const size_t n[9] = {elems(p, p->H, p->d_k) * es,      // q
+                       elems(p, p->H_kv, p->d_k) * es,   // k
+                       elems(p, p->H_kv, p->d_v) * es,   // v
+                       elems(p, p->H, p->gate_dim) * es, // gate
+                       (size_t)p->H * p->d_k * p->conv_k * es, (size_t)p->H_kv * p->d_k * p->conv_k * es,
+                       (size_t)p->H * p->d_k * p->d_k * es,  // w_q, w_k, W
+                       elems(p, p->H, p->d_v) * es,      // o
+                       lawcat_workspace_bytes(p, LAWCAT_OP_LAYER_FWD)};
+  size_t o = 0;
+  for (int i = 0; i < 9; ++i) {
+    off[i] = o;
+    o += align_up(n[i], 256);
+  }
+  off[9] = o;
+  return o;
+}
+
+size_t lawcat_layer_fwd_host_arena_bytes(const lawcat_params* p) {
+  if (check_params(p, true) != LAWCAT_OK) return 0;
+  size_t off[10];
+  return host_arena_layout(p, off);
+}
+
+int lawcat_layer_fwd_host(const lawcat_params* p, const void* h_q, const void* h_k, const void* h_v,
+                          const void* h_gate, const void* h_w_q, const void* h_w_k, const void* h_W, void* h_o,
+                          void* arena, size_t arena_bytes, void* stream) {
+  int r = check_params(p, true);
+  if (r) return r;
+  if (!h_q || !h_k || !h_v || !h_gate || !h_w_q || !h_w_k || !h_W || !h_o || !arena || !aligned16(arena))
+    return LAWCAT_ERR_INVALID_ARG;
+  size_t off[10];
+  if (arena_bytes < host_arena_layout(p, off)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
+  char* a = (char*)arena;
+  cudaStream_t st = (cudaStream_t)stream;
+  const void* src[7] = {h_q, h_k, h_v, h_gate, h_w_q, h_w_k, h_W};
+  const size_t es = p->dtype == LAWCAT_F32 ? 4 : 2;
+  const size_t nb[7] = {elems(p, p->H, p->d_k) * es, elems(p, p->H_kv, p->d_k) * es, elems(p, p->H_kv, p->d_v) * es,
+                        elems(p, p->H, p->gate_dim) * es, (size_t)p->H * p->d_k * p->conv_k * es,
+                        (size_t)p->H_kv * p->d_k * p->conv_k * es, (size_t)p->H * p->d_k * p->d_k * es};
+  for (int i = 0; i < 7; ++i)
+    if (nb[i] && cudaMemcpyAsync(a + off[i], src[i], nb[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return LAWCAT_ERR_CUDA;
+  r = lawcat_layer_fwd(p, a + off[0], a + off[1], a + off[2], a + off[3], a + off[4], a + off[5], a + off[6], nullptr,
+                       nullptr, nullptr, nullptr, a + off[7], nullptr, nullptr, nullptr, nullptr, a + off[8],
+                       off[9] - off[8], stream, nullptr);
+  if (r) return r;
+  const size_t no = elems(p, p->H, p->d_v) * es;
+  if (no && cudaMemcpyAsync(h_o, a + off[7], no, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LAWCAT_ERR_CUDA;
+  return LAWCAT_OK;
+}
+
 }  // extern "C"

@@ -67,6 +67,19 @@ int launch_decode(const Ctx& c, const void* q_t, const void* k_t, const void* v_
                   const void* w_q, const void* w_k, const void* W, float* S, float* z, void* cache_q, void* cache_k,
                   void* o_t);
 
+// Counts one kernel launch; while tracing is on it also brackets the launch with CUDA events on its stream.
+struct LaunchScope {
+  LaunchScope(const char* name, cudaStream_t s);
+  ~LaunchScope();
+  cudaStream_t stream;
+  int idx;
+};
+#define LAWCAT_LAUNCH(name, strm, ...)       \
+  do {                                       \
+    ::lawcat::LaunchScope _ls(name, strm);   \
+    __VA_ARGS__;                             \
+  } while (0)
+
 #define LAWCAT_CHECK_LAUNCH()                                 \
   do {                                                        \
     if (cudaGetLastError() != cudaSuccess) return LAWCAT_ERR_CUDA; \

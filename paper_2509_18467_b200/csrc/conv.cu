@@ -54,6 +54,7 @@ int launch_conv_plain(const Ctx& c, const void* x, const void* w, const void* ca
   if (total == 0) return LAWCAT_OK;
   const int threads = 256;
   const unsigned blocks = (unsigned)((total + threads - 1) / threads);
+  LaunchScope _ls("conv_plain", c.stream);
   if (p.dtype == LAWCAT_F32)
     conv_plain_kernel<float, TR><<<blocks, threads, 0, c.stream>>>((const float*)x, (const float*)w,
                                                                      (const float*)cache, (float*)out, p.B, p.T, C,
@@ -173,6 +174,7 @@ int launch_convmix_fwd(const Ctx& c, const void* q, const void* k, const void* w
       return LAWCAT_ERR_CUDA;                                                                                  \
     convmix_fwd_kernel<TI, TO><<<grid, CM_THREADS, smem, c.stream>>>(a);                                       \
   } while (0)
+  LaunchScope _ls("convmix_fwd", c.stream);
   if (p.dtype == LAWCAT_F32) LAUNCH_CM(float, float);
   else if (out_f32) LAUNCH_CM(bf16, float);
   else LAUNCH_CM(bf16, bf16);
@@ -386,6 +388,7 @@ static int conv_bwd_stream(const Ctx& c, const TD* du, const TI* x, const TI* w,
   const int C = NH * p.d_k;
   const size_t total = (size_t)p.B * p.T * C;
   if (dx) {
+    LaunchScope _ls("conv_bwd_dx", c.stream);
     conv_bwd_dx_kernel<TD, TI, TI><<<(unsigned)((total + 255) / 256), 256, 0, c.stream>>>(du, w, dx, p.B, p.T, C,
                                                                                            p.conv_k);
     LAWCAT_CHECK_LAUNCH();
@@ -393,6 +396,7 @@ static int conv_bwd_stream(const Ctx& c, const TD* du, const TI* x, const TI* w,
   if (dw) {
     if (cudaMemsetAsync(dw, 0, sizeof(float) * (size_t)C * p.conv_k, c.stream) != cudaSuccess) return LAWCAT_ERR_CUDA;
     dim3 grid(p.B * ((p.T + DW_SPAN - 1) / DW_SPAN), (C + 127) / 128);
+    LaunchScope _ls("conv_bwd_dw", c.stream);
     conv_bwd_dw_kernel<TD, TI><<<grid, 128, 0, c.stream>>>(du, x, cache, dw, p.B, p.T, C, p.conv_k);
     LAWCAT_CHECK_LAUNCH();
   }
@@ -432,6 +436,7 @@ static int conv_bwd_typed(const Ctx& c, const void* q, const void* k, const void
       return LAWCAT_ERR_CUDA;                                                                                    \
     convmix_bwd_kernel<TI, D><<<grid, CM_THREADS, smem, c.stream>>>(a);                                          \
   } while (0)
+  LaunchScope _ls("convmix_bwd", c.stream);
   switch (p.d_k) {
     case 16: LAUNCH_CB(16); break;
     case 32: LAUNCH_CB(32); break;
@@ -478,6 +483,7 @@ static int cache_out_typed(const Ctx& c, const void* x, const void* cin, void* c
   const lawcat_params& p = *c.p;
   const size_t total = (size_t)p.B * (p.conv_k - 1) * NH * p.d_k;
   if (!cout || total == 0) return LAWCAT_OK;
+  LaunchScope _ls("cache_out", c.stream);
   cache_out_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, c.stream>>>((const T*)x, (const T*)cin, (T*)cout,
                                                                               p.B, p.T, NH * p.d_k, p.conv_k);
   LAWCAT_CHECK_LAUNCH();

@@ -125,15 +125,17 @@ static int decode_typed(const Ctx& c, DecodeArgs& a, void* cache_q, void* cache_
   const lawcat_params& p = *c.p;
   if (p.B * p.H == 0) return LAWCAT_OK;
   const size_t smem = sizeof(float) * ((size_t)5 * p.d_k + p.d_v + (size_t)(DEC_THREADS / 16) * p.d_v + 8);
-  decode_kernel<T><<<p.B * p.H, DEC_THREADS, smem, c.stream>>>(a);
+  LAWCAT_LAUNCH("decode", c.stream, decode_kernel<T><<<p.B * p.H, DEC_THREADS, smem, c.stream>>>(a));
   LAWCAT_CHECK_LAUNCH();
   if (p.conv_k > 1) {
     const size_t nq = (size_t)p.B * p.H * p.d_k, nk = (size_t)p.B * p.H_kv * p.d_k;
-    cache_shift_kernel<T><<<(unsigned)((nq + 255) / 256), 256, 0, c.stream>>>((T*)cache_q, (const T*)a.q_t, p.B,
-                                                                               p.H * p.d_k, p.conv_k);
+    LAWCAT_LAUNCH("cache_shift", c.stream,
+                  cache_shift_kernel<T><<<(unsigned)((nq + 255) / 256), 256, 0, c.stream>>>(
+                      (T*)cache_q, (const T*)a.q_t, p.B, p.H * p.d_k, p.conv_k));
     LAWCAT_CHECK_LAUNCH();
-    cache_shift_kernel<T><<<(unsigned)((nk + 255) / 256), 256, 0, c.stream>>>((T*)cache_k, (const T*)a.k_t, p.B,
-                                                                               p.H_kv * p.d_k, p.conv_k);
+    LAWCAT_LAUNCH("cache_shift", c.stream,
+                  cache_shift_kernel<T><<<(unsigned)((nk + 255) / 256), 256, 0, c.stream>>>(
+                      (T*)cache_k, (const T*)a.k_t, p.B, p.H_kv * p.d_k, p.conv_k));
     LAWCAT_CHECK_LAUNCH();
   }
   return LAWCAT_OK;

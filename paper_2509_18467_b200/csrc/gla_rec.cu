@@ -124,6 +124,7 @@ static int gla_fwd_launch(const Ctx& c, GlaArgs& a) {
   const size_t smem = sizeof(float) * ((size_t)3 * TB * p.d_k + (size_t)TB * CW + (size_t)TB * RG * CW);
   const int threads = RG * CW;
   const unsigned grid = p.B * p.H;
+  LaunchScope _ls("gla_fwd_rec", c.stream);
   switch (R) {
     case 16: gla_fwd_rec_kernel<TQ, TS, 16><<<grid, threads, smem, c.stream>>>(a); break;
     case 32: gla_fwd_rec_kernel<TQ, TS, 32><<<grid, threads, smem, c.stream>>>(a); break;
@@ -418,22 +419,24 @@ static int gla_bwd_typed(const Ctx& c, GlaArgs& a, void* dv_out) {
   const size_t smem_col = sizeof(float) * ((size_t)3 * TB * dk + (size_t)TB * (dv + 1) + (size_t)TB * RG * dv);
   const int row_thr = (dk * NSEG + 31) / 32 * 32, col_thr = (RG * dv + 31) / 32 * 32;
   // sweep 1: dqdot (forward in time) ; sweep 2: per-head dv (backward in time) ; sweep 3: dkdot + dgate
-  if (CS == 32) gla_bwd_row_kernel<TS, 32, 0><<<grid, row_thr, smem_row, c.stream>>>(a);
-  else gla_bwd_row_kernel<TS, 16, 0><<<grid, row_thr, smem_row, c.stream>>>(a);
+  LAWCAT_LAUNCH("gla_bwd_row_fwd", c.stream,
+                if (CS == 32) gla_bwd_row_kernel<TS, 32, 0><<<grid, row_thr, smem_row, c.stream>>>(a);
+                else gla_bwd_row_kernel<TS, 16, 0><<<grid, row_thr, smem_row, c.stream>>>(a));
   LAWCAT_CHECK_LAUNCH();
-  switch (R) {
-    case 16: gla_bwd_col_kernel<TS, 16><<<grid, col_thr, smem_col, c.stream>>>(a); break;
-    case 32: gla_bwd_col_kernel<TS, 32><<<grid, col_thr, smem_col, c.stream>>>(a); break;
-    case 64: gla_bwd_col_kernel<TS, 64><<<grid, col_thr, smem_col, c.stream>>>(a); break;
-    default: return LAWCAT_ERR_UNSUPPORTED;
-  }
+  if (R != 16 && R != 32 && R != 64) return LAWCAT_ERR_UNSUPPORTED;
+  LAWCAT_LAUNCH("gla_bwd_col", c.stream,
+                if (R == 16) gla_bwd_col_kernel<TS, 16><<<grid, col_thr, smem_col, c.stream>>>(a);
+                else if (R == 32) gla_bwd_col_kernel<TS, 32><<<grid, col_thr, smem_col, c.stream>>>(a);
+                else gla_bwd_col_kernel<TS, 64><<<grid, col_thr, smem_col, c.stream>>>(a));
   LAWCAT_CHECK_LAUNCH();
-  if (CS == 32) gla_bwd_row_kernel<TS, 32, 1><<<grid, row_thr, smem_row, c.stream>>>(a);
-  else gla_bwd_row_kernel<TS, 16, 1><<<grid, row_thr, smem_row, c.stream>>>(a);
+  LAWCAT_LAUNCH("gla_bwd_row_rev", c.stream,
+                if (CS == 32) gla_bwd_row_kernel<TS, 32, 1><<<grid, row_thr, smem_row, c.stream>>>(a);
+                else gla_bwd_row_kernel<TS, 16, 1><<<grid, row_thr, smem_row, c.stream>>>(a));
   LAWCAT_CHECK_LAUNCH();
   const size_t total = (size_t)p.B * p.T * p.H_kv * dv;
-  dv_group_reduce_kernel<TS><<<(unsigned)((total + 255) / 256), 256, 0, c.stream>>>(a.dvh, (TS*)dv_out, total, p.H_kv,
-                                                                                   p.H / p.H_kv, dv);
+  LAWCAT_LAUNCH("dv_group_reduce", c.stream,
+                dv_group_reduce_kernel<TS><<<(unsigned)((total + 255) / 256), 256, 0, c.stream>>>(
+                    a.dvh, (TS*)dv_out, total, p.H_kv, p.H / p.H_kv, dv));
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }

@@ -4,30 +4,7 @@ import numpy as np
 from oracle import lawcat_oracle as O
 from paper_2509_18467_b200 import inputs as I
 
-# Tolerances (stated by the benchmark definition): fp32 mode max relative error 1e-4, bf16 mode 1e-2 of the output RMS.
-TOL_F32 = 1e-4
-TOL_BF16 = 1e-2
-BF16_HALF_ULP = 2.0 ** -8   # worst relative error of rounding a value to bfloat16 storage
-
-
-def err_f32(x, y):
-    """max_i |x_i - y_i| / max(|y_i|, rms(y))"""
-    x, y = np.asarray(x, np.float64), np.asarray(y, np.float64)
-    if y.size == 0:
-        return 0.0
-    rms = np.sqrt(np.mean(y * y)) + 1e-300
-    return float(np.max(np.abs(x - y) / np.maximum(np.abs(y), rms)))
-
-
-def err_bf16(x, y):
-    """Returns (strict, computed): strict = max_i |x_i - y_i| / rms(y); computed discounts, per element, the half ulp
-    that storing the result in bfloat16 costs whatever was computed: max_i (|x_i - y_i| - 2^-8 |y_i|)+ / rms(y)."""
-    x, y = np.asarray(x, np.float64), np.asarray(y, np.float64)
-    if y.size == 0:
-        return 0.0, 0.0
-    rms = np.sqrt(np.mean(y * y)) + 1e-300
-    d = np.abs(x - y)
-    return float(np.max(d) / rms), float(np.max(np.maximum(d - BF16_HALF_ULP * np.abs(y), 0.0)) / rms)
+from paper_2509_18467_b200.metrics import TOL_BF16, TOL_F32, err_bf16, err_f32  # noqa: F401
 
 
 def check(x, y, dtype, what, f32_store=False):
