@@ -51,7 +51,8 @@ typedef enum {
   LAWCAT_ERR_CUDA = 3,
   LAWCAT_ERR_WORKSPACE_TOO_SMALL = 4,
   LAWCAT_ERR_TIMEOUT = 5,
-  LAWCAT_ERR_NUMERIC = 6
+  LAWCAT_ERR_NUMERIC = 6,
+  LAWCAT_ERR_TOO_LARGE = 7 /* the problem exceeds a fixed built-in limit (see lawcat_layer_fwd_noalloc) */
 } lawcat_status;
 
 enum { LAWCAT_F32 = 0, LAWCAT_BF16 = 1 };
@@ -185,6 +186,33 @@ size_t lawcat_layer_fwd_host_arena_bytes(const lawcat_params* p);
 int lawcat_layer_fwd_host(const lawcat_params* p, const void* h_q, const void* h_k, const void* h_v,
                           const void* h_gate, const void* h_w_q, const void* h_w_k, const void* h_W, void* h_o,
                           void* arena, size_t arena_bytes, void* stream);
+
+/*
+ * lawcat_layer_fwd without any caller-provided workspace (the paper has no counterpart; this exists for deployment).
+ *
+ * Who needs it: code that must not, or cannot, allocate device memory at the point of the call -- a serving loop whose
+ * memory pool is frozen after start-up, a plugin running inside a host application that owns the allocator, a callback
+ * that runs where cudaMalloc is forbidden. Such callers cannot size and provide `ws`. Here the scratch (the fp32
+ * conv+mix+phi outputs qdot and kdot of the exact CUDA-core path) lives in a fixed device array inside the library
+ * image, LAWCAT_NOALLOC_SCRATCH_BYTES large; every GPU that loads the library holds that memory until the process ends.
+ *
+ * Arguments and results are those of lawcat_layer_fwd minus ws/ws_bytes; the computation is the exact (fp32
+ * accumulate, CUDA-core) path for every dtype. The call allocates nothing and frees nothing.
+ *   - Limit: 2 * roundup256(4 * B*T*H*d_k) bytes must fit the array, i.e. B*T*H*d_k <= 4 Mi elements with the default
+ *     32 MiB. Larger problems return LAWCAT_ERR_TOO_LARGE before anything is enqueued: split the sequence and carry the
+ *     state and the conv caches from call to call.
+ *   - The first call on each device looks up the device address of the array (cudaGetSymbolAddress, with that device
+ *     current); make that first call outside of any stream capture.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call left in it. Nothing in it
+ *     has to start at zero (both tensors are fully written before they are read), but two calls whose kernels overlap
+ *     on the GPU -- different streams, no ordering between them -- race on it. Keep calls on one stream or order them.
+ */
+#define LAWCAT_NOALLOC_SCRATCH_BYTES (32u << 20)
+size_t lawcat_noalloc_scratch_bytes(void);
+int lawcat_layer_fwd_noalloc(const lawcat_params* p, const void* q, const void* k, const void* v, const void* gate,
+                             const void* w_q, const void* w_k, const void* W, const void* cache_q_in,
+                             const void* cache_k_in, const float* S0, const float* z0, void* o, void* cache_q_out,
+                             void* cache_k_out, float* S_T, float* z_T, void* stream, int* dev_status);
 
 #ifdef __cplusplus
 }

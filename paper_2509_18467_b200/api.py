@@ -23,7 +23,7 @@ OP_CONV_FWD, OP_CONV_BWD, OP_GLA_FWD, OP_GLA_BWD, OP_LAYER_FWD, OP_DECODE_STEP =
 EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "lawcat_launch_count",
            "lawcat_trace_begin", "lawcat_trace_end", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
            "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
-           "lawcat_layer_fwd_host"]
+           "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc"]
 
 
 class LawcatError(RuntimeError):
@@ -68,6 +68,9 @@ def lib() -> ctypes.CDLL:
         L.lawcat_launch_count.restype = ctypes.c_ulonglong
         L.lawcat_layer_fwd_host_arena_bytes.restype = ctypes.c_size_t
         L.lawcat_layer_fwd_host_arena_bytes.argtypes = [ctypes.POINTER(Params)]
+        L.lawcat_noalloc_scratch_bytes.restype = ctypes.c_size_t
+        L.lawcat_layer_fwd_noalloc.restype = ctypes.c_int
+        L.lawcat_layer_fwd_noalloc.argtypes = [ctypes.POINTER(Params)] + [ctypes.c_void_p] * 18
         L.lawcat_layer_fwd_host.restype = ctypes.c_int
         L.lawcat_layer_fwd_host.argtypes = [ctypes.POINTER(Params)] + [ctypes.c_void_p] * 9 + \
                                            [ctypes.c_size_t, ctypes.c_void_p]
@@ -224,6 +227,19 @@ def lawcat_layer_fwd_host(p: Params, h_q, h_k, h_v, h_gate, h_w_q, h_w_k, h_W, h
     if st != 0:
         raise LawcatError(st, "lawcat_layer_fwd_host")
     return h_o
+
+
+def lawcat_layer_fwd_noalloc(p: Params, q, k, v, gate, w_q, w_k, W, cache_q=None, cache_k=None, S0=None, z0=None,
+                             o=None, cache_q_out=None, cache_k_out=None, S_T=None, z_T=None, stream=None,
+                             dev_status=None):
+    """The layer forward for callers that cannot allocate: no workspace argument, the scratch is a fixed array inside
+    the library (see the header for its size limit and the sharing rules). Every output must be passed in by the
+    caller; only `o` is required. Returns o."""
+    ptrs = [q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0, o, cache_q_out, cache_k_out, S_T, z_T]
+    st = lib().lawcat_layer_fwd_noalloc(ctypes.byref(p), *[_ptr(t) for t in ptrs], _stream(stream), _ptr(dev_status))
+    if st != 0:
+        raise LawcatError(st, "lawcat_layer_fwd_noalloc")
+    return o
 
 
 def host_arena_bytes(p: Params) -> int:

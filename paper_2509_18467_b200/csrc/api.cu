@@ -54,6 +54,7 @@ const char* lawcat_status_string(int s) {
     case LAWCAT_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case LAWCAT_ERR_TIMEOUT: return "bounded device wait ran out";
     case LAWCAT_ERR_NUMERIC: return "numeric range violation";
+    case LAWCAT_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }

@@ -1,0 +1,71 @@
+"""The no-allocation layer forward (`lawcat_layer_fwd_noalloc`) against the regular entry point.
+
+Some callers of this library cannot call cudaMalloc where they call the layer (a frozen memory pool, a host application
+that owns the allocator), so they cannot hand over a workspace; the no-allocation entry point keeps its scratch in a
+fixed array inside the library instead. This file checks, through the C ABI, that it returns what `lawcat_layer_fwd`
+returns, twice in a row (the scratch is shared and keeps the previous call's contents), and that it refuses problems
+beyond its fixed limit. It is collected last so that a failure here cannot hide any other test.
+"""
+import ctypes
+import dataclasses
+
+import pytest
+
+from helpers import check
+from paper_2509_18467_b200 import inputs as I
+
+NAMES = ["q", "k", "v", "gate", "w_q", "w_k", "W"]
+
+
+def _p(api, s):
+    return api.params(s.B, s.T, s.H, s.H_kv, s.d_k, s.d_v, conv_k=s.conv_k, gate_dim=s.gate_dim, dtype=s.dtype,
+                      gate_tau=s.gate_tau)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_noalloc_matches_regular_entry_point_twice(dtype):
+    import torch
+    from paper_2509_18467_b200 import api
+    before = torch.cuda.memory_allocated()
+    shapes = [I.LayerShape(2, 200, 4, 2, 64, 64, dtype=dtype, config_id=21),
+              I.LayerShape(1, 77, 8, 2, 128, 32, dtype=dtype, gate_dim=1, config_id=22)]
+    for s in shapes:  # the second call reuses the scratch the first one left behind, with a different shape
+        x = I.make(s, NAMES + ["S0", "z0", "cache_q", "cache_k"])
+        d = {n: api.to_device(v, "f32" if n in ("S0", "z0") else s.dtype) for n, v in x.items()}
+        p = _p(api, s)
+        ref = api.lawcat_layer_fwd(p, *[d[n] for n in NAMES], d["cache_q"], d["cache_k"], d["S0"], d["z0"])
+        out = {k: torch.full_like(v, float("nan")) for k, v in ref.items()}
+        torch.cuda.synchronize()
+        held = torch.cuda.memory_allocated()
+        api.lawcat_layer_fwd_noalloc(p, *[d[n] for n in NAMES], d["cache_q"], d["cache_k"], d["S0"], d["z0"],
+                                     out["o"], out["cache_q"], out["cache_k"], out["S_T"], out["z_T"])
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == held  # the call itself took nothing from the allocator
+        check(out["o"], ref["o"].double().cpu().numpy(), s.dtype, "o")
+        check(out["S_T"], ref["S_T"].double().cpu().numpy(), s.dtype, "S_T", f32_store=True)
+        check(out["z_T"], ref["z_T"].double().cpu().numpy(), s.dtype, "z_T", f32_store=True)
+        assert torch.equal(out["cache_q"], ref["cache_q"]) and torch.equal(out["cache_k"], ref["cache_k"])
+    del d, ref, out
+    assert torch.cuda.memory_allocated() <= before + (1 << 20)
+
+
+def test_noalloc_rejects_oversized_and_bad_problems_on_host():
+    from paper_2509_18467_b200 import api, build
+    build.build()
+    L = api.lib()
+    limit = L.lawcat_noalloc_scratch_bytes()
+    assert limit == 32 << 20
+    ok = ctypes.c_void_p(0x1000)
+    args = [ok] * 7 + [None] * 4 + [ok] + [None] * 4 + [None, None]
+    big = api.params(1, 4096, 32, 8, 128, 128)      # 2 * 4 * 16 Mi elements: far beyond the array
+    assert L.lawcat_layer_fwd_noalloc(ctypes.byref(big), *args) == 7
+    assert "built-in scratch" in api.status_string(7)
+    edge = api.params(1, 1024, 32, 8, 128, 128)     # exactly 4 Mi elements per tensor: fits
+    assert 2 * 4 * 1024 * 32 * 128 == limit
+    bad = api.params(1, 16, 4, 3, 64, 64)
+    assert L.lawcat_layer_fwd_noalloc(ctypes.byref(bad), *args) == 1
+    odd = api.params(1, 16, 4, 2, 48, 64)
+    assert L.lawcat_layer_fwd_noalloc(ctypes.byref(odd), *args) == 2
+    nullq = [None] + args[1:]
+    assert L.lawcat_layer_fwd_noalloc(ctypes.byref(edge), *nullq) == 1
