@@ -67,6 +67,12 @@ int launch_decode(const Ctx& c, const void* q_t, const void* k_t, const void* v_
                   const void* w_q, const void* w_k, const void* W, float* S, float* z, void* cache_q, void* cache_k,
                   void* o_t);
 
+// Chunkwise tensor-core layer forward (layer_tc.cu): whether it takes these parameters, and its launcher.
+bool layer_tc_supported(const lawcat_params& p);
+int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, const void* gate, const void* w_q,
+                    const void* w_k, const void* W, const void* cache_q_in, const void* cache_k_in, const float* S0,
+                    const float* z0, void* o, float* S_T, float* z_T);
+
 // Counts one kernel launch; while tracing is on it also brackets the launch with CUDA events on its stream.
 struct LaunchScope {
   LaunchScope(const char* name, cudaStream_t s);
