@@ -4,13 +4,14 @@
 //
 // One CTA walks one (batch, query head, segment of the sequence) in chunks of C = 64 tokens. Per chunk:
 //   TMA      raw q, k (with the 3 halo rows the conv needs), gate logits and v tiles -> 128-byte-swizzled shared memory
-//   conv     u = sum_delta w_delta * x_{t-delta} in fp32 -> bf16 rows of one stacked A operand (rows 0-63 the query
+//   conv     u = sum_delta w_delta * x_{t-delta} in fp32 -> fp16 rows of one stacked A operand (rows 0-63 the query
 //            tokens, rows 64-127 the key tokens: both streams share W_h, so ONE M=128 MMA mixes both)
 //   gate     g = logsigmoid(a)/tau, b = running sum of g inside the chunk, E_t = exp(b_t - b_mid) per channel (a scan
 //            outwards from the middle token keeps every factor within exp(+-32 max|g|))
-//   MMA 1    Y = [u_q; u_k] W_h                                   (bf16, fp32 accumulate in TMEM)
+//   MMA 1    Y = [u_q; u_k] W_h      (fp16 operands: 3 more mantissa bits than bf16 for u; fp32 accumulate in TMEM)
 //   phi      row softmax in registers (one thread per token row). Query rows keep exp(y - max) unnormalized: a positive
-//            per-token factor cancels in Eq. 8. qs = phi_q * E_t, ks = phi_k / E_i (bf16), kh = phi_k * exp(b_C - b_i)
+//            per-token factor cancels in Eq. 8. qs = phi_q * E_t, ks = phi_k / E_i: fp16 while the chunk's E stay
+//            within 2^+-8 (3 more mantissa bits; the usual case), bf16 otherwise (range); kh = phi_k * exp(b_C - b_i)
 //            (fp16, <= phi_k)
 //   MMA 2    P = qs ks^T ; O' = qs (exp(b_mid) S_prev) ; [S|z] = exp(b_C) [S|z] + kh^T [v|1]
 //   mask     P_ti = 0 for i > t, rounded to fp16 (bf16 weights would cost up to 2^-9 relative error per weight, which
@@ -38,17 +39,24 @@ constexpr uint32_t OFF_W = 0;                       // W_h^T, K-major, 2 slabs x
 constexpr uint32_t OFF_SBF = OFF_W + 32768;         // exp(b_mid) * S, bf16, MN-major, 2 slabs x [128 x 128 B]
 constexpr uint32_t OFF_A = OFF_SBF + 32768;         // stacked A operand: conv outputs, then qs / ks in place
 constexpr uint32_t OFF_KH = OFF_A + 32768;          // kh, fp16, MN-major A of the state update, 2 slabs x [64 x 128 B]
-constexpr uint32_t OFF_G = OFF_KH + 16384;          // gate logits, then E in place (bf16), 2 slabs x [64 x 128 B]
+constexpr uint32_t OFF_G = OFF_KH + 16384;          // gate logits (bf16), 2 slabs x [64 x 128 B]
 constexpr uint32_t OFF_V = OFF_G + 16384;           // v bf16, then fp16 in place, MN-major B, 2 slabs x [64 x 128 B]
 constexpr uint32_t RAW_SLAB = 9216;                 // 67 rows x 128 B rounded up to 1024
 constexpr uint32_t OFF_QRAW = OFF_V + 16384;        // raw q tile (2 slabs); later the masked scores P (fp16, 16 KB)
+constexpr uint32_t OFF_E = OFF_QRAW;                // after the conv: E fp32 [64 x 128] over the raw q and k tiles (32 KB)
 constexpr uint32_t OFF_KRAW = OFF_QRAW + 2 * RAW_SLAB;  // raw k tile (2 slabs); later the output staging (16 KB)
 constexpr uint32_t OFF_SZ = OFF_KRAW + 2 * RAW_SLAB;    // exp(b_mid) * z as a [128 x 16] bf16 operand (column 0 is z)
 constexpr uint32_t OFF_ONES = OFF_SZ + 4096;        // [64 x 16] fp16 operand whose column 0 is 1 (the "1" of [v|1])
-constexpr uint32_t OFF_VEC = OFF_ONES + 2048;       // dm[128], dC[128], e63[128] fp32
-constexpr uint32_t OFF_BAR = OFF_VEC + 3 * 512;     // mbarriers and scalars
+constexpr uint32_t OFF_QB = OFF_ONES + 2048;        // qs in bf16 for the read-out MMA, K-major, 2 slabs x [64 x 128 B]
+constexpr uint32_t OFF_VEC = OFF_QB + 16384;        // dm[128], dC[128], e63[128], qsum[64] fp32
+constexpr uint32_t OFF_BAR = OFF_VEC + 3 * 512 + 256;  // mbarriers and scalars
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 64;
-constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;  // slack for the manual 1024-byte alignment
+// The M = 128 read-out MMA reads 128 rows per slab of the 64-row qs tile: its (unused) rows 64-127 reach 8 KB past the
+// tile, so the allocation extends that far; plus slack for the manual 1024-byte alignment.
+constexpr uint32_t SMEM_ALLOC = OFF_QB + 16384 + 8192 + 1024;
+static_assert(SMEM_ALLOC >= SMEM_BYTES + 1024 && SMEM_ALLOC <= 232448, "shared memory budget");
+constexpr float SMAX_F16 = 3.0e4f;  // largest |state entry| for which the read-out operands are kept in fp16
+constexpr float RMAX_F16 = 8.f;  // largest log2 range of E for which the score operands are kept in fp16
 
 // tensor memory map (32-bit columns)
 constexpr uint32_t COL_Y = 0;      // [128 x 128] mix output
@@ -76,6 +84,14 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
   f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
 }
 
+// channels [8 jj, 8 jj + 8) of row t of the fp32 E tile (see the gate pass for its layout)
+__device__ __forceinline__ void load_E8(uint32_t base, int t, int jj, float* E) {
+  const uint4 lo = lds128(base + t * 512 + (((2 * jj) ^ (t & 7)) << 4));
+  const uint4 hi = lds128(base + t * 512 + (((2 * jj + 1) ^ (t & 7)) << 4));
+  E[0] = __uint_as_float(lo.x); E[1] = __uint_as_float(lo.y); E[2] = __uint_as_float(lo.z); E[3] = __uint_as_float(lo.w);
+  E[4] = __uint_as_float(hi.x); E[5] = __uint_as_float(hi.y); E[6] = __uint_as_float(hi.z); E[7] = __uint_as_float(hi.w);
+}
+
 // log2 of the decay of one gate entry: LOGITS: log2(sigmoid(a)) / tau, LOGDECAY: a * log2(e).
 __device__ __forceinline__ float log2_decay(float a, int gate_mode, float inv_tau) {
   const float L2E = 1.4426950408889634f;
@@ -98,7 +114,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   float* const s_dm = reinterpret_cast<float*>(sg + OFF_VEC);
   float* const s_dC = s_dm + 128;
   float* const s_e63 = s_dm + 256;
-  volatile int* const s_flags = reinterpret_cast<volatile int*>(sg + OFF_BAR + 32);  // [0] tmem base, [1] abort
+  float* const s_qsum = s_dm + 384;  // per query token: sum of exp(y - max), the dropped softmax normalizer
+  volatile int* const s_flags = reinterpret_cast<volatile int*>(sg + OFF_BAR + 32);  // [0] tmem base, [1] abort, [2] rmax
+  int* const s_rmax = const_cast<int*>(s_flags) + 2;  // bits of the largest |log2 E| of the chunk (a non-negative float)
+  // Range tracking for the fp16 read-out operand (all as bits of non-negative floats): largest |state entry| seen by the
+  // last state pass, largest |v| of the chunk, and the resulting bound on the state the NEXT state pass will convert
+  // (|S_new| <= |S_old| + 64 max|v| because kh <= 1).
+  int* const s_smax = s_rmax + 1;
+  int* const s_vmax = s_rmax + 2;
+  int* const s_sbound = s_rmax + 3;
   const uint32_t bar_load = sb + OFF_BAR, bar_mma = sb + OFF_BAR + 8;
 
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -117,6 +141,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     mbar_init(bar_mma, 1);
     mbar_fence_init();
     s_flags[1] = 0;
+    *s_smax = 0; *s_vmax = 0; *s_sbound = 0;
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_g);
     tma_prefetch_desc(&tm_o);
   }
@@ -133,9 +158,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       uint32_t w[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint16_t lo = reinterpret_cast<const uint16_t*>(Wh)[(size_t)(oc * 8 + 2 * i) * D + e];
-        const uint16_t hi = reinterpret_cast<const uint16_t*>(Wh)[(size_t)(oc * 8 + 2 * i + 1) * D + e];
-        w[i] = (uint32_t)lo | ((uint32_t)hi << 16);
+        w[i] = pack_f16(__bfloat162float(Wh[(size_t)(oc * 8 + 2 * i) * D + e]),
+                        __bfloat162float(Wh[(size_t)(oc * 8 + 2 * i + 1) * D + e]));
       }
       sts128(sb + OFF_W + (oc >> 3) * 16384 + sw128(e, oc & 7), make_uint4(w[0], w[1], w[2], w[3]));
     }
@@ -166,17 +190,23 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // initial state into tensor memory: thread c owns row c of [S | z]
   if (tid < D) {
     const bool have = a.S0 != nullptr && (a.per_seg_state || seg == 0);
-    float s[32];
+    float s[32], mx = 0.f;
 #pragma unroll
     for (int blk = 0; blk < 4; ++blk) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i)
+      for (int i = 0; i < 32; ++i) {
         s[i] = have ? a.S0[(state_idx * D + tid) * D + blk * 32 + i] : 0.f;
+        mx = fmaxf(mx, fabsf(s[i]));
+      }
       tmem_st32(lane_base + COL_S + blk * 32, s);
     }
     const bool havez = a.z0 != nullptr && (a.per_seg_state || seg == 0);
-    tmem_st1(lane_base + COL_S + D, havez ? a.z0[state_idx * D + tid] : 0.f);
+    const float z0v = havez ? a.z0[state_idx * D + tid] : 0.f;
+    tmem_st1(lane_base + COL_S + D, z0v);
     tmem_wait_st();
+    mx = fmaxf(mx, fabsf(z0v));
+    if (!(mx < 3.0e38f)) mx = 3.0e38f;  // NaN or inf in the given state: no fp16 operand
+    atomicMax(s_sbound, __float_as_int(mx));
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -209,6 +239,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     store_pending = false;
     LAWCAT_WAIT_ALL(bar_load, ph_load);
+    if (tid == 0) *s_rmax = 0;
 
     // rows before the first token of the sequence come from the conv cache (TMA zero-filled them)
     if (t0 == 0 && a.K > 1 && (a.cache_q || a.cache_k)) {
@@ -242,12 +273,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int ch = 0; ch < 8; ++ch)
           u[ch] = fmaf(cw[ch][0], x0[ch], fmaf(cw[ch][1], x1[ch], fmaf(cw[ch][2], x2[ch], cw[ch][3] * x3[ch])));
         sts128(dst + sw128(cv_stream * 64 + r0 + i, jc),
-               make_uint4(pack_bf16(u[0], u[1]), pack_bf16(u[2], u[3]), pack_bf16(u[4], u[5]), pack_bf16(u[6], u[7])));
+               make_uint4(pack_f16(u[0], u[1]), pack_f16(u[2], u[3]), pack_f16(u[4], u[5]), pack_f16(u[6], u[7])));
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) { x3[ch] = x2[ch]; x2[ch] = x1[ch]; x1[ch] = x0[ch]; }
       }
     }
 
+    __syncthreads();  // the raw q, k tiles are dead from here on: E takes their place
     if (tid < D) {
       // ---- gate: thread = channel; scans outwards from the middle token ------------------------------------------------
       const int c = tid;
@@ -260,9 +292,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         asm volatile("ld.shared.u16 %0, [%1];" : "=h"(raw) : "r"(gaddr(t)));
         return log2_decay(__uint_as_float((uint32_t)raw << 16), a.gate_mode, a.inv_tau);
       };
+      // E[t][c] fp32, 512-byte rows whose 16-byte chunks are XOR-swizzled with t & 7 (conflict-free for this
+      // column-wise writer and for the row-wise readers of the phi pass)
       auto putE = [&](int t, float e) {
-        const uint16_t v = __bfloat16_as_ushort(__float2bfloat16_rn(e));
-        asm volatile("st.shared.u16 [%0], %1;" ::"r"(gaddr(t)), "h"(v) : "memory");
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(sb + OFF_E + t * 512 + (((c >> 2) ^ (t & 7)) << 4) + (c & 3) * 4), "f"(e)
+                     : "memory");
       };
       bool clamped = false;
       float f = 0.f;
@@ -271,7 +305,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         f += g2(t);
         putE(t, ex2f(f));
       }
-      float r = 0.f, cur = g2(MID);  // E overwrites the logits in place: read entry t before writing it
+      float r = 0.f, cur = g2(MID);
 #pragma unroll 8
       for (int t = MID - 1; t >= 0; --t) {
         r += cur;
@@ -285,18 +319,24 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const float bm = r + g0;
       s_dm[c] = ex2f(bm);
       s_dC[c] = ex2f(bm + f);
-      s_e63[c] = __bfloat162float(__float2bfloat16_rn(ex2f(f)));
+      s_e63[c] = ex2f(f);
+      atomicMax(s_rmax, __float_as_int(fmaxf(-r, -f)));  // r, f <= 0: the largest exponent magnitude of this channel
       if (clamped && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_NUMERIC);
     } else {
       // ---- v: bf16 -> fp16 in place (exact for |v| in the fp16 normal range) ------------------------------------------
       const int vt = tid - D;
+      float vm = 0.f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const uint32_t ad = sb + OFF_V + (uint32_t)(vt + 128 * i) * 16;
         float x[8];
         unpack8(lds128(ad), x);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) vm = fmaxf(vm, fabsf(x[e]));
         sts128(ad, make_uint4(pack_f16(x[0], x[1]), pack_f16(x[2], x[3]), pack_f16(x[4], x[5]), pack_f16(x[6], x[7])));
       }
+      vm = warp_max(vm);
+      if ((tid & 31) == 0) atomicMax(s_vmax, __float_as_int(vm < 3.0e38f ? vm : 3.0e38f));
     }
     fence_proxy_async();
     __syncthreads();
@@ -304,7 +344,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ---- MMA 1: Y = [u_q; u_k] W_h ------------------------------------------------------------------------------------
     if (tid == 0) {
       tc_fence_after_sync();
-      constexpr uint32_t ID = instr_desc(128, 128, FMT_BF16, MAJOR_K, MAJOR_K);
+      constexpr uint32_t ID = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_K);
 #pragma unroll
       for (int k = 0; k < 8; ++k)
         mma_f16(tmem + COL_Y, smem_desc(sb + OFF_A + (k >> 2) * 16384 + (k & 3) * 32, 16, 1024, LAYOUT_SW128),
@@ -316,17 +356,24 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (tid < D) {
       const int c = tid;
       const float dm = s_dm[c], dC = s_dC[c];
-      float s[32];
+      const bool sf16 = __int_as_float(*s_rmax) <= RMAX_F16 && __int_as_float(*s_sbound) < SMAX_F16;
+      float s[32], mx = 0.f;
 #pragma unroll
       for (int blk = 0; blk < 4; ++blk) {
         tmem_ld32(lane_base + COL_S + blk * 32, s);
         tmem_wait_ld();
         if (MODE == 0) {
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4)
+          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(s[i]));
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            float w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = dm * s[8 * q4 + i];
             sts128(sb + OFF_SBF + (blk >> 1) * 16384 + sw128(c, (blk & 1) * 4 + q4),
-                   make_uint4(pack_bf16(dm * s[8 * q4 + 0], dm * s[8 * q4 + 1]), pack_bf16(dm * s[8 * q4 + 2], dm * s[8 * q4 + 3]),
-                              pack_bf16(dm * s[8 * q4 + 4], dm * s[8 * q4 + 5]), pack_bf16(dm * s[8 * q4 + 6], dm * s[8 * q4 + 7])));
+                   sf16 ? make_uint4(pack_f16(w[0], w[1]), pack_f16(w[2], w[3]), pack_f16(w[4], w[5]), pack_f16(w[6], w[7]))
+                        : make_uint4(pack_bf16(w[0], w[1]), pack_bf16(w[2], w[3]), pack_bf16(w[4], w[5]), pack_bf16(w[6], w[7])));
+          }
         }
 #pragma unroll
         for (int i = 0; i < 32; ++i) s[i] *= dC;
@@ -334,8 +381,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       const float z = tmem_ld1(lane_base + COL_S + D);
       tmem_wait_ld();
-      if (MODE == 0)
-        *reinterpret_cast<bf16*>(sg + OFF_SZ + (c >> 3) * 128 + (c & 7) * 16) = __float2bfloat16_rn(dm * z);
+      if (MODE == 0) {
+        const uint16_t zb = sf16 ? __half_as_ushort(__float2half_rn(dm * z)) : __bfloat16_as_ushort(__float2bfloat16_rn(dm * z));
+        *reinterpret_cast<uint16_t*>(sg + OFF_SZ + (c >> 3) * 128 + (c & 7) * 16) = zb;
+        mx = warp_max(fmaxf(mx, fabsf(z)));
+        if ((tid & 31) == 0) atomicMax(s_smax, __float_as_int(mx < 3.0e38f ? mx : 3.0e38f));
+      }
       tmem_st1(lane_base + COL_S + D, dC * z);
       tmem_wait_st();
     }
@@ -353,18 +404,28 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
       for (int i = 1; i < D; ++i) m = fmaxf(m, y[i]);
       const float mb = m * L2E;
+      const bool f16 = __int_as_float(*s_rmax) <= RMAX_F16;
+      const bool sf16 = f16 && __int_as_float(*s_sbound) < SMAX_F16;
       if (tid < C) {
         const int t = tid;
+        float qsum = 0.f;
 #pragma unroll
         for (int jj = 0; jj < 16; ++jj) {
           float E[8];
-          unpack8(lds128(sb + OFF_G + (jj >> 3) * 8192 + sw128(t, jj & 7)), E);
+          load_E8(sb + OFF_E, t, jj, E);
           float v[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] = ex2f(fmaf(y[jj * 8 + i], L2E, -mb)) * E[i];
-          sts128(sb + OFF_A + (jj >> 3) * 16384 + sw128(t, jj & 7),
-                 make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7])));
+          for (int i = 0; i < 8; ++i) {
+            const float ex = ex2f(fmaf(y[jj * 8 + i], L2E, -mb));
+            qsum += ex;
+            v[i] = ex * E[i];
+          }
+          const uint4 vb = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+          const uint4 vh = make_uint4(pack_f16(v[0], v[1]), pack_f16(v[2], v[3]), pack_f16(v[4], v[5]), pack_f16(v[6], v[7]));
+          sts128(sb + OFF_QB + (jj >> 3) * 8192 + sw128(t, jj & 7), sf16 ? vh : vb);
+          sts128(sb + OFF_A + (jj >> 3) * 16384 + sw128(t, jj & 7), f16 ? vh : vb);
         }
+        s_qsum[t] = qsum;
       } else {
         const int i_tok = tid - C;
         float sum = 0.f;
@@ -377,7 +438,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
         for (int jj = 0; jj < 16; ++jj) {
           float E[8];
-          unpack8(lds128(sb + OFF_G + (jj >> 3) * 8192 + sw128(i_tok, jj & 7)), E);
+          load_E8(sb + OFF_E, i_tok, jj, E);
           const float4 ea = *reinterpret_cast<const float4*>(s_e63 + jj * 8);
           const float4 eb = *reinterpret_cast<const float4*>(s_e63 + jj * 8 + 4);
           const float e63[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
@@ -389,7 +450,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           if (MODE == 0)
             sts128(sb + OFF_A + (jj >> 3) * 16384 + sw128(C + i_tok, jj & 7),
-                   make_uint4(pack_bf16(ks[0], ks[1]), pack_bf16(ks[2], ks[3]), pack_bf16(ks[4], ks[5]), pack_bf16(ks[6], ks[7])));
+                   f16 ? make_uint4(pack_f16(ks[0], ks[1]), pack_f16(ks[2], ks[3]), pack_f16(ks[4], ks[5]), pack_f16(ks[6], ks[7]))
+                       : make_uint4(pack_bf16(ks[0], ks[1]), pack_bf16(ks[2], ks[3]), pack_bf16(ks[4], ks[5]), pack_bf16(ks[6], ks[7])));
           sts128(sb + OFF_KH + (jj >> 3) * 8192 + sw128(i_tok, jj & 7),
                  make_uint4(pack_f16(kh[0], kh[1]), pack_f16(kh[2], kh[3]), pack_f16(kh[4], kh[5]), pack_f16(kh[6], kh[7])));
         }
@@ -403,16 +465,23 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (tid == 0) {
       tc_fence_after_sync();
       if (MODE == 0) {
-        constexpr uint32_t ID_P = instr_desc(128, 64, FMT_BF16, MAJOR_K, MAJOR_K);
-        constexpr uint32_t ID_O = instr_desc(128, 128, FMT_BF16, MAJOR_K, MAJOR_MN);
-        constexpr uint32_t ID_OZ = instr_desc(128, 16, FMT_BF16, MAJOR_K, MAJOR_MN);
+        const uint32_t ID_P = __int_as_float(*s_rmax) <= RMAX_F16 ? instr_desc(128, 64, FMT_F16, MAJOR_K, MAJOR_K)
+                                                                  : instr_desc(128, 64, FMT_BF16, MAJOR_K, MAJOR_K);
+        const bool sf16 = __int_as_float(*s_rmax) <= RMAX_F16 && __int_as_float(*s_sbound) < SMAX_F16;
+        const uint32_t ID_O = instr_desc(128, 128, sf16 ? FMT_F16 : FMT_BF16, MAJOR_K, MAJOR_MN);
+        const uint32_t ID_OZ = instr_desc(128, 16, sf16 ? FMT_F16 : FMT_BF16, MAJOR_K, MAJOR_MN);
+        // bound on the state after this chunk's update, for the next chunk's choice of operand type
+        *s_sbound = __float_as_int(__int_as_float(*s_smax) + 64.f * fmaxf(__int_as_float(*s_vmax), 1.f));
+        *s_smax = 0;
+        *s_vmax = 0;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t ad = smem_desc(sb + OFF_A + (k >> 2) * 16384 + (k & 3) * 32, 16, 1024, LAYOUT_SW128);
           mma_f16(tmem + COL_P, ad, smem_desc(sb + OFF_A + (k >> 2) * 16384 + 8192 + (k & 3) * 32, 16, 1024, LAYOUT_SW128),
                   ID_P, k > 0);
-          mma_f16(tmem + COL_O, ad, smem_desc(sb + OFF_SBF + k * 2048, 16384, 1024, LAYOUT_SW128), ID_O, k > 0);
-          mma_f16(tmem + COL_O + D, ad, smem_desc(sb + OFF_SZ + k * 256, 128, 2048, LAYOUT_NONE), ID_OZ, k > 0);
+          const uint64_t qb = smem_desc(sb + OFF_QB + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024, LAYOUT_SW128);
+          mma_f16(tmem + COL_O, qb, smem_desc(sb + OFF_SBF + k * 2048, 16384, 1024, LAYOUT_SW128), ID_O, k > 0);
+          mma_f16(tmem + COL_O + D, qb, smem_desc(sb + OFF_SZ + k * 256, 128, 2048, LAYOUT_NONE), ID_OZ, k > 0);
         }
       }
       constexpr uint32_t ID_S = instr_desc(128, 128, FMT_F16, MAJOR_MN, MAJOR_MN);
@@ -474,7 +543,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int blk = 0; blk < 4; ++blk) {
           tmem_ld32(lane_base + COL_O + blk * 32, o);
           tmem_wait_ld();
-          const float inv = 1.f / (den + a.eps);
+          // the query features went in scaled by qsum (unnormalized softmax), so eps scales the same way
+          const float inv = 1.f / (den + a.eps * s_qsum[t]);
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
             sts128(sb + OFF_KRAW + (blk >> 1) * 8192 + sw128(t, (blk & 1) * 4 + q4),
