@@ -41,6 +41,10 @@ size_t elems(const lawcat_params* p, int heads, int d) { return (size_t)p->B * (
 
 }  // namespace
 
+namespace lawcat {
+int validate_params(const lawcat_params* p, bool need_T) { return check_params(p, need_T); }
+}  // namespace lawcat
+
 extern "C" {
 
 int lawcat_version(void) { return 100; }
@@ -68,6 +72,7 @@ size_t lawcat_workspace_bytes(const lawcat_params* p, int op) {
       return align_up(sizeof(float) * elems(p, p->H, p->d_v), 256) + 2 * align_up(sizeof(float) * elems(p, p->H, 1), 256) +
              align_up(sizeof(float) * elems(p, p->H, p->d_k), 256);
     case LAWCAT_OP_LAYER_FWD:
+      if (layer_tc_supported(*p)) return align_up(layer_tc_workspace_bytes(*p), 256);
       return 2 * align_up(sizeof(float) * elems(p, p->H, p->d_k), 256);
     default:
       return 0;
@@ -151,7 +156,7 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
   if (need && (!ws || ws_bytes < need)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
   Ctx c{p, (cudaStream_t)stream, dev_status};
   if (layer_tc_supported(*p)) {  // chunkwise tensor-core kernel
-    if ((r = launch_layer_tc(c, q, k, v, gate, w_q, w_k, W, cache_q_in, cache_k_in, S0, z0, o, S_T, z_T))) return r;
+    if ((r = launch_layer_tc(c, q, k, v, gate, w_q, w_k, W, cache_q_in, cache_k_in, S0, z0, o, S_T, z_T, ws))) return r;
     return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
   }
   // exact path: conv + mix + phi into fp32 scratch, then the recurrent GLA

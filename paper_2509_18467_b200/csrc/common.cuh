@@ -67,11 +67,16 @@ int launch_decode(const Ctx& c, const void* q_t, const void* k_t, const void* v_
                   const void* w_q, const void* w_k, const void* W, float* S, float* z, void* cache_q, void* cache_k,
                   void* o_t);
 
+// Host-side check of a parameter block (api.cu): LAWCAT_OK, LAWCAT_ERR_INVALID_ARG or LAWCAT_ERR_UNSUPPORTED.
+int validate_params(const lawcat_params* p, bool need_T);
+
 // Chunkwise tensor-core layer forward (layer_tc.cu): whether it takes these parameters, and its launcher.
 bool layer_tc_supported(const lawcat_params& p);
+int layer_tc_segments(const lawcat_params& p);
+size_t layer_tc_workspace_bytes(const lawcat_params& p);
 int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, const void* gate, const void* w_q,
                     const void* w_k, const void* W, const void* cache_q_in, const void* cache_k_in, const float* S0,
-                    const float* z0, void* o, float* S_T, float* z_T);
+                    const float* z0, void* o, float* S_T, float* z_T, void* ws);
 
 // Counts one kernel launch; while tracing is on it also brackets the launch with CUDA events on its stream.
 struct LaunchScope {

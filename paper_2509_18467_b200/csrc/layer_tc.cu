@@ -69,12 +69,15 @@ constexpr uint32_t LOAD_BYTES = 4 * RAW_ROWS * 128 + 4 * C * 128;
 
 struct TcArgs {
   const bf16 *w_q, *w_k, *W, *cache_q, *cache_k;
-  const float *S0, *z0;  // state before the first token of each CTA's segment: [B,H,nseg?,...] see seg_state_stride
-  float *S_T, *z_T;      // state after the last token (full mode: last segment only)
+  const float *S0, *z0;  // state before the first token of the CTA's segment
+  float *S_T, *z_T;      // state after the last token of the CTA's segment
+  float* dtot;           // [B,H,nseg,128]: log2 of the total decay of the segment per key channel (nullable)
   int* dev_status;
   int T, H, Hkv, K;
   int nseg, seg_len;     // segments per sequence and tokens per segment (a multiple of C)
-  int per_seg_state;     // 1: S0/z0/S_T/z_T are indexed [b,h,seg]; 0: [b,h] (S0 applies to segment 0, S_T to the last)
+  int grid_nseg;         // segments of each sequence covered by this launch (the first grid_nseg of nseg)
+  int seg_in;            // 1: S0/z0 are indexed [b,h,seg]; 0: [b,h] and they apply to segment 0 only
+  int seg_out;           // 1: S_T/z_T are indexed [b,h,seg]; 0: [b,h] and only the last segment writes them
   int gate_mode;
   float inv_tau, eps;
 };
@@ -126,14 +129,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t bar_load = sb + OFF_BAR, bar_mma = sb + OFF_BAR + 8;
 
   const int tid = threadIdx.x, warp = tid >> 5;
-  const int seg = blockIdx.x % a.nseg;
-  const int bh = blockIdx.x / a.nseg;
+  const int seg = blockIdx.x % a.grid_nseg;
+  const int bh = blockIdx.x / a.grid_nseg;
   const int h = bh % a.H, b = bh / a.H;
   const int G = a.H / a.Hkv, j = h / G;
   const int t_begin = seg * a.seg_len;
   const int t_end = min(a.T, t_begin + a.seg_len);
   const int nchunks = (t_end - t_begin + C - 1) / C;
-  const size_t state_idx = a.per_seg_state ? (size_t)bh * a.nseg + seg : (size_t)bh;
+  const size_t seg_idx = (size_t)bh * a.nseg + seg;
+  const size_t in_idx = a.seg_in ? seg_idx : (size_t)bh, out_idx = a.seg_out ? seg_idx : (size_t)bh;
+  float dsum = 0.f;  // gate threads: log2 of this channel's total decay over the segment
 
   // ---- one-time setup --------------------------------------------------------------------------------------------
   if (tid == 0) {
@@ -189,19 +194,19 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   // initial state into tensor memory: thread c owns row c of [S | z]
   if (tid < D) {
-    const bool have = a.S0 != nullptr && (a.per_seg_state || seg == 0);
+    const bool have = a.S0 != nullptr && (a.seg_in || seg == 0);
     float s[32], mx = 0.f;
 #pragma unroll
     for (int blk = 0; blk < 4; ++blk) {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        s[i] = have ? a.S0[(state_idx * D + tid) * D + blk * 32 + i] : 0.f;
+        s[i] = have ? a.S0[(in_idx * D + tid) * D + blk * 32 + i] : 0.f;
         mx = fmaxf(mx, fabsf(s[i]));
       }
       tmem_st32(lane_base + COL_S + blk * 32, s);
     }
-    const bool havez = a.z0 != nullptr && (a.per_seg_state || seg == 0);
-    const float z0v = havez ? a.z0[state_idx * D + tid] : 0.f;
+    const bool havez = a.z0 != nullptr && (a.seg_in || seg == 0);
+    const float z0v = havez ? a.z0[in_idx * D + tid] : 0.f;
     tmem_st1(lane_base + COL_S + D, z0v);
     tmem_wait_st();
     mx = fmaxf(mx, fabsf(z0v));
@@ -319,6 +324,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const float bm = r + g0;
       s_dm[c] = ex2f(bm);
       s_dC[c] = ex2f(bm + f);
+      dsum += bm + f;
       s_e63[c] = ex2f(f);
       atomicMax(s_rmax, __float_as_int(fmaxf(-r, -f)));  // r, f <= 0: the largest exponent magnitude of this channel
       if (clamped && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_NUMERIC);
@@ -566,7 +572,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   // ---- final state ---------------------------------------------------------------------------------------------------
   tc_fence_after_sync();
-  if (tid < D && a.S_T != nullptr && (a.per_seg_state || seg == a.nseg - 1)) {
+  if (tid < D && a.dtot != nullptr) a.dtot[seg_idx * D + tid] = dsum;
+  if (tid < D && a.S_T != nullptr && (a.seg_out || seg == a.nseg - 1)) {
     float s[32];
 #pragma unroll
     for (int blk = 0; blk < 4; ++blk) {
@@ -574,11 +581,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_wait_ld();
 #pragma unroll
       for (int i = 0; i < 32; i += 4)
-        *reinterpret_cast<float4*>(a.S_T + (state_idx * D + tid) * D + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
+        *reinterpret_cast<float4*>(a.S_T + (out_idx * D + tid) * D + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
     }
     const float z = tmem_ld1(lane_base + COL_S + D);
     tmem_wait_ld();
-    if (a.z_T) a.z_T[state_idx * D + tid] = z;
+    if (a.z_T) a.z_T[out_idx * D + tid] = z;
   }
 
 done:
@@ -622,7 +629,46 @@ static bool make_map(CUtensorMap* m, const void* ptr, int heads, int T, int B, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// State at the start of every segment from the per-segment end states (computed from zero) and total decays:
+// start[0] = given state; start[s] = decay[s-1] * start[s-1] + local[s-1]  (Eq. 4 unrolled over whole segments).
+// One thread per state entry (the d_k x d_v entries of S, then the d_k entries of z) of one (batch, head).
+__global__ void segment_scan_kernel(const float* __restrict__ S0, const float* __restrict__ z0,
+                                    const float* __restrict__ loc_S, const float* __restrict__ loc_z,
+                                    const float* __restrict__ dtot, float* __restrict__ start_S,
+                                    float* __restrict__ start_z, int BH, int nseg) {
+  const int per = D * D + D;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= BH * per) return;
+  const int bh = idx / per, r = idx % per;
+  const bool isz = r >= D * D;
+  const int c = isz ? r - D * D : r / D;  // key channel: the decay is per row of the state
+  const int e = isz ? 0 : r % D;
+  float cur = isz ? (z0 ? z0[(size_t)bh * D + c] : 0.f) : (S0 ? S0[((size_t)bh * D + c) * D + e] : 0.f);
+  for (int sgm = 0; sgm < nseg; ++sgm) {
+    const size_t si = (size_t)bh * nseg + sgm;
+    if (isz) start_z[si * D + c] = cur; else start_S[(si * D + c) * D + e] = cur;
+    if (sgm + 1 < nseg) {
+      const float loc = isz ? loc_z[si * D + c] : loc_S[(si * D + c) * D + e];
+      cur = fmaf(exp2f(dtot[si * D + c]), cur, loc);
+    }
+  }
+}
+
 }  // namespace tc
+
+// Segments per sequence: enough thread blocks to fill the SMs (one block per SM), but at least 16 chunks per segment.
+int layer_tc_segments(const lawcat_params& p) {
+  const int chunks = (p.T + tc::C - 1) / tc::C;
+  int n = 148 / (p.B * p.H);
+  if (n > chunks / 16) n = chunks / 16;
+  return n < 1 ? 1 : n;
+}
+
+size_t layer_tc_workspace_bytes(const lawcat_params& p) {
+  const int nseg = layer_tc_segments(p);
+  if (nseg == 1) return 0;
+  return sizeof(float) * (size_t)p.B * p.H * nseg * (2 * (tc::D * tc::D + tc::D) + tc::D);
+}
 
 bool layer_tc_supported(const lawcat_params& p) {
   return p.dtype == LAWCAT_BF16 && p.d_k == tc::D && p.d_v == tc::D && p.gate_dim == p.d_k &&
@@ -632,7 +678,7 @@ bool layer_tc_supported(const lawcat_params& p) {
 
 int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, const void* gate, const void* w_q,
                     const void* w_k, const void* W, const void* cache_q_in, const void* cache_k_in, const float* S0,
-                    const float* z0, void* o, float* S_T, float* z_T) {
+                    const float* z0, void* o, float* S_T, float* z_T, void* ws) {
   using namespace tc;
   const lawcat_params& p = *c.p;
   CUtensorMap tq, tk, tv, tg, to;
@@ -643,15 +689,51 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   TcArgs a{};
   a.w_q = (const bf16*)w_q; a.w_k = (const bf16*)w_k; a.W = (const bf16*)W;
   a.cache_q = (const bf16*)cache_q_in; a.cache_k = (const bf16*)cache_k_in;
-  a.S0 = S0; a.z0 = z0; a.S_T = S_T; a.z_T = z_T; a.dev_status = c.dev_status;
+  a.dev_status = c.dev_status;
   a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k;
-  a.nseg = 1; a.seg_len = (p.T + C - 1) / C * C; a.per_seg_state = 0;
   a.gate_mode = p.gate_mode; a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps;
+  const int nseg = layer_tc_segments(p);
+  a.nseg = nseg;
+  a.seg_len = ((p.T + nseg - 1) / nseg + C - 1) / C * C;
   if (cudaFuncSetAttribute(layer_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
       cudaFuncSetAttribute(layer_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess)
     return LAWCAT_ERR_CUDA;
+  const int BH = p.B * p.H;
+  if (nseg == 1) {
+    a.S0 = S0; a.z0 = z0; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
+    a.grid_nseg = 1; a.seg_in = 0; a.seg_out = 0;
+    LaunchScope _ls("layer_tc", c.stream);
+    layer_tc_kernel<0><<<BH, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, to, a);
+    LAWCAT_CHECK_LAUNCH();
+    return LAWCAT_OK;
+  }
+  // Several segments per sequence: (1) every segment but the last computes its end state from a zero state, and the
+  // total decay of the segment; (2) a scan over the segments turns these into the state at each segment's start;
+  // (3) the layer runs on all segments at once, each from its start state.
+  const size_t nS = (size_t)BH * nseg * D * D, nz = (size_t)BH * nseg * D;
+  float* loc_S = (float*)ws;
+  float* loc_z = loc_S + nS;
+  float* dtot = loc_z + nz;
+  float* start_S = dtot + nz;
+  float* start_z = start_S + nS;
+  {
+    TcArgs b1 = a;
+    b1.S0 = nullptr; b1.z0 = nullptr; b1.S_T = loc_S; b1.z_T = loc_z; b1.dtot = dtot;
+    b1.grid_nseg = nseg - 1; b1.seg_in = 1; b1.seg_out = 1;
+    LaunchScope _ls("layer_tc_state", c.stream);
+    layer_tc_kernel<1><<<BH * (nseg - 1), THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, to, b1);
+    LAWCAT_CHECK_LAUNCH();
+  }
+  {
+    const int total = BH * (D * D + D);
+    LaunchScope _ls("segment_scan", c.stream);
+    segment_scan_kernel<<<(total + 255) / 256, 256, 0, c.stream>>>(S0, z0, loc_S, loc_z, dtot, start_S, start_z, BH, nseg);
+    LAWCAT_CHECK_LAUNCH();
+  }
+  a.S0 = start_S; a.z0 = start_z; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
+  a.grid_nseg = nseg; a.seg_in = 1; a.seg_out = 0;
   LaunchScope _ls("layer_tc", c.stream);
-  layer_tc_kernel<0><<<p.B * p.H * a.nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, to, a);
+  layer_tc_kernel<0><<<BH * nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, to, a);
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }

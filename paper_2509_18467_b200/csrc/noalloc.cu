@@ -43,18 +43,10 @@ int lawcat_layer_fwd_noalloc(const lawcat_params* p, const void* q, const void* 
                              const void* cache_k_in, const float* S0, const float* z0, void* o, void* cache_q_out,
                              void* cache_k_out, float* S_T, float* z_T, void* stream, int* dev_status) {
   if (!p) return LAWCAT_ERR_INVALID_ARG;
-  // the exact path's scratch: two fp32 tensors [B,T,H,d_k]; this also validates the parameter block (0 = invalid)
-  const size_t half = align_up(sizeof(float) * (size_t)p->B * (size_t)(p->T > 0 ? p->T : 0) * p->H * p->d_k, 256);
-  lawcat_params probe = *p;
-  probe.B = 1;
-  probe.T = 1;
-  if (lawcat_workspace_bytes(&probe, LAWCAT_OP_LAYER_FWD) == 0 || p->B < 0 || p->T < 0) {
-    // let the regular entry point classify the problem (invalid argument vs unsupported shape); nothing is enqueued
-    return lawcat_layer_fwd(p, q, k, v, gate, w_q, w_k, W, cache_q_in, cache_k_in, S0, z0, o, cache_q_out,
-                            cache_k_out, S_T, z_T, nullptr, 0, stream, dev_status) == LAWCAT_ERR_UNSUPPORTED
-               ? LAWCAT_ERR_UNSUPPORTED
-               : LAWCAT_ERR_INVALID_ARG;
-  }
+  const int bad = validate_params(p, true);  // invalid argument vs unsupported shape; nothing is enqueued
+  if (bad) return bad;
+  // the exact path's scratch: two fp32 tensors [B,T,H,d_k]
+  const size_t half = align_up(sizeof(float) * (size_t)p->B * (size_t)p->T * p->H * p->d_k, 256);
   if (2 * half > kScratchBytes) return LAWCAT_ERR_TOO_LARGE;
   const void* const req[] = {w_q, w_k, W};
   for (const void* x : req)
