@@ -86,12 +86,12 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
                     const float* z0, void* o, float* S_T, float* z_T, void* ws) {
   using namespace tc;
   const lawcat_params& p = *c.p;
-  CUtensorMap tq, tk, tv, tg, to;
-  if (!make_map(&tq, q, p.H, p.T, p.B, RAW_ROWS) || !make_map(&tk, k, p.H_kv, p.T, p.B, RAW_ROWS) ||
-      !make_map(&tv, v, p.H_kv, p.T, p.B, C) || !make_map(&tg, gate, p.H, p.T, p.B, C) ||
-      !make_map(&to, o, p.H, p.T, p.B, C))
+  CUtensorMap tq, tk, tv, tg;
+  if (!make_map(&tq, q, p.H, p.T, p.B, C) || !make_map(&tk, k, p.H_kv, p.T, p.B, C) ||
+      !make_map(&tv, v, p.H_kv, p.T, p.B, C) || !make_map(&tg, gate, p.H, p.T, p.B, C))
     return LAWCAT_ERR_CUDA;
   TcArgs a{};
+  a.q = (const bf16*)q; a.k = (const bf16*)k; a.o = (bf16*)o;
   a.w_q = (const bf16*)w_q; a.w_k = (const bf16*)w_k; a.W = (const bf16*)W;
   a.cache_q = (const bf16*)cache_q_in; a.cache_k = (const bf16*)cache_k_in;
   a.dev_status = c.dev_status;
@@ -108,7 +108,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
     a.S0 = S0; a.z0 = z0; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
     a.grid_nseg = 1; a.seg_in = 0; a.seg_out = 0;
     LaunchScope _ls("layer_tc", c.stream);
-    layer_tc_kernel<0><<<BH, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, to, a);
+    layer_tc_kernel<0><<<BH, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
     LAWCAT_CHECK_LAUNCH();
     return LAWCAT_OK;
   }
@@ -126,7 +126,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
     b1.S0 = nullptr; b1.z0 = nullptr; b1.S_T = loc_S; b1.z_T = loc_z; b1.dtot = dtot;
     b1.grid_nseg = nseg - 1; b1.seg_in = 1; b1.seg_out = 1;
     LaunchScope _ls("layer_tc_state", c.stream);
-    layer_tc_kernel<1><<<BH * (nseg - 1), THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, to, b1);
+    layer_tc_kernel<1><<<BH * (nseg - 1), THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, b1);
     LAWCAT_CHECK_LAUNCH();
   }
   {
@@ -138,7 +138,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   a.S0 = start_S; a.z0 = start_z; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
   a.grid_nseg = nseg; a.seg_in = 1; a.seg_out = 0;
   LaunchScope _ls("layer_tc", c.stream);
-  layer_tc_kernel<0><<<BH * nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, to, a);
+  layer_tc_kernel<0><<<BH * nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }

@@ -2,26 +2,31 @@
 // conv (Section 4.1) -> shared linear layer + softmax feature map (Section 4.1) -> normalized gated linear attention
 // (Eq. 4 - Eq. 8) in its chunkwise-parallel form, with the d_k x (d_v+1) state [S | z] kept in tensor memory in fp32.
 //
-// One CTA walks one (batch, query head, segment of the sequence) in chunks of C = 64 tokens. Per chunk:
-//   TMA      raw q, k (with the 3 halo rows the conv needs), gate logits and v tiles -> 128-byte-swizzled shared memory
-//   conv     u = sum_delta w_delta * x_{t-delta} in fp32 -> fp16 rows of one stacked A operand (rows 0-63 the query
-//            tokens, rows 64-127 the key tokens: both streams share W_h, so ONE M=128 MMA mixes both)
-//   gate     g = log2 sigmoid(a) / tau per entry, then a scan outwards from the middle token gives the exponents
-//            x_t = b_t - b_mid (b the running sum of g) in fp32. The middle reference keeps every factor 2^x within
-//            2^(+-32 max|g|).
-//   MMA 1    Y = [u_q; u_k] W_h      (fp16 operands: 3 more mantissa bits than bf16 for u; fp32 accumulate in TMEM)
-//   phi      row softmax, one thread per token row, 32 columns at a time straight from tensor memory. Query rows keep
-//            exp(y - max) unnormalized: a positive per-token factor cancels in Eq. 8. The decay factors ride in the
-//            exponent of the softmax: qs = 2^(y' + x_t), ks = phi_k 2^(-x_i), kh = phi_k 2^(b_C - b_i) (fp16, <= phi_k)
-//   MMA 2    P = qs ks^T ; O' = qs (2^b_mid [S|z]) ; [S|z] = 2^b_C [S|z] + kh^T [v|1]
-//   mask     P_ti = 0 for i > t, rounded to fp16
-//   MMA 3    O' += P [v|1]   (fp16 operands; v converts from bf16 to fp16 exactly)
-//   out      o_t = O'_t[:d_v] / (O'_t[d_v] + eps) -> bf16 -> TMA store
+// One CTA walks one (batch, query head, segment of the sequence) in chunks of C = 64 tokens. The work of a chunk is
+// split over specialized warps that hand tiles to one another through mbarriers, so that consecutive chunks overlap:
+//   TMA warp    raw q, k tiles (one stacked [128 x 128] tile: rows 0-63 query tokens, rows 64-127 key tokens), gate
+//               logits and v tiles -> 128-byte-swizzled shared memory
+//   prep warps  conv: u = sum_delta w_delta * x_{t-delta} in fp32 -> fp16, IN PLACE over the raw tile, which thereby
+//               becomes the stacked A operand of the mix (both streams share W_h, so ONE M=128 MMA mixes both);
+//               gate: g = log2 sigmoid(a) / tau per entry, then a scan outwards from the middle token gives the
+//               exponents x_t = b_t - b_mid (b the running sum of g) in fp32 (the middle reference keeps every factor
+//               2^x within 2^(+-32 max|g|)); v: bf16 -> fp16 in place (exact)
+//   MMA warp    MMA 1: Y = [u_q; u_k] W_h  (fp16 operands, fp32 accumulate in TMEM)
+//   row warps   phi: row softmax, one thread per token row, 32 columns at a time straight from tensor memory. Query rows
+//               keep exp(y - max) unnormalized: a positive per-token factor cancels in Eq. 8. The decay factors ride in
+//               the exponent of the softmax: qs = 2^(y' + x_t), ks = phi_k 2^(-x_i), kh = phi_k 2^(b_C - b_i) (<= phi_k)
+//   state warps 2^b_mid [S|z] as a 16-bit operand, accumulator [S|z] *= 2^b_C
+//   MMA warp    MMA 2: P = qs ks^T ; O' = qs (2^b_mid [S|z]) ; [S|z] += kh^T [v|1]
+//   row warps   mask: P_ti = 0 for i > t, rounded to fp16
+//   MMA warp    MMA 3: O' += P [v|1]
+//   row warps   o_t = O'_t[:d_v] / (O'_t[d_v] + eps) -> bf16 -> global memory
 // Operand precision: qs, ks and the state operand are fp16 (11-bit mantissa) while the chunk's x stay within
 // +-8 and the state within +-3e4 -- the usual case -- and bf16 otherwise (range first). bf16 score weights would
 // cost up to 2^-9 relative error per weight, which the first tokens of a sequence do not average out.
 // Every MMA uses M = 128; where only 64 rows are meaningful (P, O') the upper 64 TMEM lanes hold unused results.
-// Loops over column blocks are deliberately NOT unrolled: the chunk loop must stay well inside the instruction cache.
+// Loops over column blocks are deliberately NOT unrolled: each role's loop must stay inside the instruction cache.
+// Every wait is bounded: a wait that runs out raises the abort flag, every role leaves its loop, the CTA frees its
+// tensor memory and reports LAWCAT_ERR_TIMEOUT through dev_status.
 #pragma once
 #include <cuda.h>
 
@@ -34,30 +39,35 @@ namespace tc {
 constexpr int D = 128;       // d_k = d_v
 constexpr int C = 64;        // tokens per chunk
 constexpr int MID = 31;      // reference token of the in-chunk decay factorization
-constexpr int HALO = 3;      // halo rows loaded in front of a chunk (conv width up to 4)
-constexpr int RAW_ROWS = C + HALO;
-constexpr int THREADS = 256;
+constexpr int HALO = 3;      // raw rows in front of a chunk that the conv needs (conv width up to 4)
+
+// warps: 0-7 prep, 8-11 row warps (TMEM quadrant = warp & 3), 12-15 state warps (same), 16 TMA, 17 MMA
+constexpr int PREP_THREADS = 256;
+constexpr int ROW_WARP0 = 8, STATE_WARP0 = 12, TMA_WARP = 16, MMA_WARP = 17;
+constexpr int THREADS = 18 * 32;
 
 // shared memory map (byte offsets from a 1024-byte aligned base)
-constexpr uint32_t OFF_W = 0;                       // W_h^T fp16, K-major, 2 slabs x [128 x 128 B]
-constexpr uint32_t OFF_SBF = OFF_W + 32768;         // 2^b_mid * S, 16 bit, MN-major, 2 slabs x [128 x 128 B]
-constexpr uint32_t OFF_A = OFF_SBF + 32768;         // stacked A operand: conv outputs, then qs / ks in place
-constexpr uint32_t OFF_KH = OFF_A + 32768;          // kh^T, fp16, K-major A of the state update, [128 channels x 64 tokens]
-constexpr uint32_t OFF_G = OFF_KH + 16384;          // gate logits (bf16), 2 slabs x [64 x 128 B]
-constexpr uint32_t OFF_V = OFF_G + 16384;           // v bf16, then fp16 in place, MN-major B, 2 slabs x [64 x 128 B]
-constexpr uint32_t RAW_SLAB = 9216;                 // 67 rows x 128 B rounded up to 1024
-constexpr uint32_t OFF_QRAW = OFF_V + 16384;        // raw q tile (2 slabs); later the masked scores P (fp16, 16 KB)
-constexpr uint32_t OFF_X = OFF_QRAW;                // after the conv: exponents x fp32 [64 x 128] over the raw tiles (32 KB)
-constexpr uint32_t OFF_KRAW = OFF_QRAW + 2 * RAW_SLAB;  // raw k tile (2 slabs); later the output staging (16 KB)
-constexpr uint32_t OFF_SZ = OFF_KRAW + 2 * RAW_SLAB;    // 2^b_mid * z as a [128 x 16] operand (column 0 is z)
-constexpr uint32_t OFF_ONES = OFF_SZ + 4096;        // [64 x 16] fp16 operand whose column 0 is 1 (the "1" of [v|1])
-constexpr uint32_t OFF_VEC = OFF_ONES + 2048;       // bm[128], ft[128], e63[128], qsum[64] fp32
-constexpr uint32_t OFF_BAR = OFF_VEC + 3 * 512 + 256;  // mbarriers and scalars
-constexpr uint32_t SMEM_BYTES = OFF_BAR + 64;
-constexpr uint32_t SMEM_ALLOC = SMEM_BYTES + 1024;  // slack for the manual 1024-byte alignment
+constexpr uint32_t OFF_W = 0;                     // W_h^T fp16, K-major, 2 slabs x [128 x 128 B]
+constexpr uint32_t OFF_SBF = OFF_W + 32768;       // 2^b_mid * S, 16 bit, MN-major, 2 slabs x [128 x 128 B]
+constexpr uint32_t OFF_AU = OFF_SBF + 32768;      // raw q|k tile, then conv output in place: A of MMA 1, 2 slabs
+constexpr uint32_t OFF_QK = OFF_AU + 32768;       // qs (rows 0-63) | ks (rows 64-127), 16 bit, K-major, 2 slabs
+constexpr uint32_t OFF_X = OFF_QK + 32768;        // exponents x fp32 [64 x 128], XOR-swizzled 16-byte chunks
+constexpr uint32_t OFF_KH = OFF_X + 32768;        // kh^T fp16, K-major A of the state update, [128 channels x 64 tokens]
+constexpr uint32_t OFF_G = OFF_KH + 16384;        // gate logits bf16, 2 slabs x [64 x 128 B]
+constexpr uint32_t OFF_V = OFF_G + 16384;         // v bf16, then fp16 in place, MN-major B, 2 slabs x [64 x 128 B]
+constexpr uint32_t OFF_PH = OFF_V + 16384;        // masked scores fp16, K-major, [64 x 128 B]; an M=128 MMA also reads
+                                                  // (and ignores) the 8 KB that follow
+constexpr uint32_t OFF_SZ = OFF_PH + 8192;        // 2^b_mid * z as a [128 x 16] operand (column 0 is z)
+constexpr uint32_t OFF_ONES = OFF_SZ + 4096;      // [64 x 16] fp16 operand whose column 0 is 1 (the "1" of [v|1])
+constexpr uint32_t OFF_HALO = OFF_ONES + 2048;    // [2 streams][3 rows][16 x 16 B]: raw rows in front of the next chunk
+constexpr uint32_t OFF_VEC = OFF_HALO + 1536;     // per parity: bm[128], ft[128], e63[128] fp32 (2 x 1536 B)
+constexpr uint32_t OFF_BAR = OFF_VEC + 3072;      // mbarriers (8 B each) and scalars
+constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+constexpr uint32_t SMEM_ALLOC = SMEM_BYTES;  // all dynamic, declared 1024-byte aligned (the kernel checks it)
+static_assert(OFF_PH + 16384 <= SMEM_BYTES, "the unused rows of the score operand must stay inside the allocation");
 static_assert(SMEM_ALLOC <= 232448, "shared memory budget");
 constexpr float SMAX_F16 = 3.0e4f;  // largest |state entry| for which the operands are kept in fp16
-constexpr float RMAX_F16 = 8.f;     // largest |log2 E| for which the operands are kept in fp16
+constexpr float RMAX_F16 = 8.f;     // largest |x| for which the operands are kept in fp16
 
 // tensor memory map (32-bit columns)
 constexpr uint32_t COL_Y = 0;      // [128 x 128] mix output
@@ -68,13 +78,35 @@ constexpr uint32_t COL_SZ = 448;   // [128 x 16] column 0: normalizer state z
 constexpr uint32_t COL_OZ = 464;   // [128 x 16] column 0: denominator
 constexpr uint32_t TMEM_COLS = 512;
 
-constexpr uint32_t LOAD_BYTES = 4 * RAW_ROWS * 128 + 4 * C * 128;
+// mbarrier indices. "full": producer -> consumer, "free": consumer -> producer. Each completes once per chunk, so the
+// wait parity of chunk n is n & 1.
+enum {
+  B_RAW_FULL = 0,  // TMA: raw q|k tile landed                      -> prep (conv)
+  B_G_FULL,        // TMA: gate tile landed                          -> prep (gate)
+  B_V_FULL,        // TMA: v tile landed                             -> prep (v convert)
+  B_G_FREE,        // prep: gate tile consumed                       -> TMA
+  B_U_FULL,        // prep: conv output written                      -> MMA 1
+  B_X_FULL,        // prep: exponents, per-channel sums, range flags -> row warps, state warps
+  B_VH_FULL,       // prep: v converted                              -> MMA 2, state warps
+  B_MMA1,          // MMA 1 complete: Y ready -> row warps; raw tile free -> TMA
+  B_Y_FREE,        // row warps: Y consumed                          -> MMA 1 of the next chunk
+  B_X_FREE,        // row warps: exponents consumed                  -> prep (gate of the next chunk)
+  B_QK_FULL,       // row warps: qs, ks, kh written                  -> MMA 2
+  B_SBF_FULL,      // state warps: state operand written, S decayed  -> MMA 2
+  B_MMA2,          // MMA 2 complete: P ready, state updated, qs/ks/kh/state operand free
+  B_PH_FULL,       // row warps: masked scores written               -> MMA 3
+  B_MMA3,          // MMA 3 complete: O' ready -> row warps; v tile free -> TMA
+  B_O_FREE,        // row warps: O' consumed                         -> MMA 2 of the next chunk
+  NUM_BARS
+};
 
 struct TcArgs {
+  const bf16 *q, *k;     // raw streams (for the halo rows in front of a segment)
   const bf16 *w_q, *w_k, *W, *cache_q, *cache_k;
   const float *S0, *z0;  // state before the first token of the CTA's segment
   float *S_T, *z_T;      // state after the last token of the CTA's segment
   float* dtot;           // [B,H,nseg,128]: log2 of the total decay of the segment per key channel (nullable)
+  bf16* o;               // [B,T,H,128]
   int* dev_status;
   int T, H, Hkv, K;
   int nseg, seg_len;     // segments per sequence and tokens per segment (a multiple of C)
@@ -89,15 +121,6 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
   f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
   f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
 }
-__device__ __forceinline__ void unpack8h(const uint4& v, float* f) {
-  const __half2* h = reinterpret_cast<const __half2*>(&v);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 t = __half22float2(h[i]);
-    f[2 * i] = t.x;
-    f[2 * i + 1] = t.y;
-  }
-}
 // 8 values -> 8 packed 16-bit values, fp16 or bf16
 __device__ __forceinline__ uint4 pack8(const float* v, bool f16) {
   return f16 ? make_uint4(pack_f16(v[0], v[1]), pack_f16(v[2], v[3]), pack_f16(v[4], v[5]), pack_f16(v[6], v[7]))
@@ -105,9 +128,6 @@ __device__ __forceinline__ uint4 pack8(const float* v, bool f16) {
 }
 __device__ __forceinline__ uint16_t to16(float x, bool f16) {
   return f16 ? __half_as_ushort(__float2half_rn(x)) : __bfloat16_as_ushort(__float2bfloat16_rn(x));
-}
-__device__ __forceinline__ float from16(uint16_t x, bool f16) {
-  return f16 ? __half2float(__ushort_as_half(x)) : __uint_as_float((uint32_t)x << 16);
 }
 
 // channels [8 jj, 8 jj + 8) of row t of the fp32 exponent tile (see the gate pass for its layout)
@@ -127,55 +147,104 @@ __device__ __forceinline__ float log2_decay(float a, int gate_mode, float inv_ta
   return -fmaxf(x, lg2f(1.f + ex2f(fminf(x, 126.f)))) * inv_tau;
 }
 
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// Named barrier that also returns the OR of `flag` over its threads: roles that synchronize among themselves leave
+// their loop only through such a barrier, all together.
+__device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool flag) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %3, 0;\n\t"
+      "bar.red.or.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(nthreads), "r"((uint32_t)flag)
+      : "memory");
+  return r != 0;
+}
+
+// Bounded wait that also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > 4000000000LL) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+
 // MODE 0: the layer forward. MODE 1: state only (no query stream, no output): the end state of a segment that starts
 // from the given state, used to hand the state across segments of one sequence.
 template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g,
-                const __grid_constant__ CUtensorMap tm_o, const TcArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t sb = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* const sg = smem_raw + (sb - smem_u32(smem_raw));  // generic pointer to the aligned base
-  float* const s_bm = reinterpret_cast<float*>(sg + OFF_VEC);  // per key channel: b_mid (log2)
-  float* const s_ft = s_bm + 128;                             // per key channel: b_C - b_mid (log2)
-  float* const s_e63 = s_bm + 256;                            // 2^ft
-  float* const s_qsum = s_bm + 384;  // per query token: sum of exp(y - max), the dropped softmax normalizer
-  volatile int* const s_flags = reinterpret_cast<volatile int*>(sg + OFF_BAR + 32);  // [0] tmem base, [1] abort
-  // Range tracking (all as bits of non-negative floats): largest |log2 E| of the chunk; largest |state entry| seen by
-  // the last state pass; largest |v| of the chunk; and the resulting bound on the state the NEXT state pass converts
-  // (|S_new| <= |S_old| + 64 max|v| because kh <= 1).
-  int* const s_rmax = const_cast<int*>(s_flags) + 2;
-  int* const s_smax = s_rmax + 1;
-  int* const s_vmax = s_rmax + 2;
-  int* const s_sbound = s_rmax + 3;
-  const uint32_t bar_load = sb + OFF_BAR, bar_mma = sb + OFF_BAR + 8;
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g, const TcArgs a) {
+  extern __shared__ __align__(1024) uint8_t sg[];
+  const uint32_t sb = smem_u32(sg);
+  volatile int* const s_flags = reinterpret_cast<volatile int*>(sg + OFF_BAR + 8 * NUM_BARS);  // [0] tmem base, [1] abort
+  // Range tracking, all as bits of non-negative floats. Per chunk parity: largest |x| of the chunk (rmax), largest |v|
+  // of the chunk (vmax), bound on the state entries the chunk's state pass converts (sbound); smax: largest |state
+  // entry| seen by the running state pass.  |S_new| <= |S_old| + 64 max|v| because kh <= 1.
+  int* const s_rmax = const_cast<int*>(s_flags) + 2;   // [2]
+  int* const s_vmax = s_rmax + 2;                      // [2]
+  int* const s_sbound = s_rmax + 4;                    // [2]
+  int* const s_smax = s_rmax + 6;                      // [1]
+  volatile int* const s_abort = s_flags + 1;
+  auto bar = [&](int i) -> uint32_t { return sb + OFF_BAR + 8 * i; };
+  auto vec = [&](int parity, int which) -> float* {  // which: 0 bm, 1 ft, 2 e63
+    return reinterpret_cast<float*>(sg + OFF_VEC + parity * 1536 + which * 512);
+  };
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int seg = blockIdx.x % a.grid_nseg;
   const int bh = blockIdx.x / a.grid_nseg;
   const int h = bh % a.H, b = bh / a.H;
   const int G = a.H / a.Hkv, j = h / G;
   const int t_begin = seg * a.seg_len;
   const int t_end = min(a.T, t_begin + a.seg_len);
-  const int nchunks = (t_end - t_begin + C - 1) / C;
+  const int nchunks = max(0, (t_end - t_begin + C - 1) / C);
   const size_t seg_idx = (size_t)bh * a.nseg + seg;
   const size_t in_idx = a.seg_in ? seg_idx : (size_t)bh, out_idx = a.seg_out ? seg_idx : (size_t)bh;
-  float dsum = 0.f;  // gate threads: log2 of this channel's total decay over the segment
+
+  if ((sb & 1023u) != 0) {  // the swizzled tiles need a 1024-byte aligned base
+    if (tid == 0 && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_CUDA);
+    return;
+  }
 
   // ---- one-time setup --------------------------------------------------------------------------------------------
   if (tid == 0) {
-    mbar_init(bar_load, 1);
-    mbar_init(bar_mma, 1);
+    const int nphi = MODE == 0 ? 128 : 64;  // threads of the phi pass: all row threads, or the key rows only
+    mbar_init(bar(B_RAW_FULL), 1);
+    mbar_init(bar(B_G_FULL), 1);
+    mbar_init(bar(B_V_FULL), 1);
+    mbar_init(bar(B_G_FREE), PREP_THREADS);
+    mbar_init(bar(B_U_FULL), PREP_THREADS);
+    mbar_init(bar(B_X_FULL), PREP_THREADS);
+    mbar_init(bar(B_VH_FULL), PREP_THREADS);
+    mbar_init(bar(B_MMA1), 1);
+    mbar_init(bar(B_Y_FREE), nphi);
+    mbar_init(bar(B_X_FREE), nphi + 128);  // the phi threads and the state threads (which read bm, ft)
+    mbar_init(bar(B_QK_FULL), nphi);
+    mbar_init(bar(B_SBF_FULL), 128);
+    mbar_init(bar(B_MMA2), 1);
+    mbar_init(bar(B_PH_FULL), 64);
+    mbar_init(bar(B_MMA3), 1);
+    mbar_init(bar(B_O_FREE), 64);
     mbar_fence_init();
     s_flags[1] = 0;
-    *s_rmax = 0; *s_smax = 0; *s_vmax = 0; *s_sbound = 0;
+    for (int i = 0; i < 7; ++i) s_rmax[i] = 0;
     tma_prefetch_desc(&tm_q); tma_prefetch_desc(&tm_k); tma_prefetch_desc(&tm_v); tma_prefetch_desc(&tm_g);
-    tma_prefetch_desc(&tm_o);
   }
-  if (warp == 0) {
-    __syncwarp();
-    tmem_alloc(sb + OFF_BAR + 32, TMEM_COLS);
+  if (warp == MMA_WARP) {
+    tmem_alloc(sb + OFF_BAR + 8 * NUM_BARS, TMEM_COLS);
     tmem_relinquish();
   }
   // W_h^T into its K-major slabs as fp16: row e holds W[h][c][e] over c
@@ -194,20 +263,23 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
   // constant "ones" operand and a zeroed z operand (unswizzled 8x8 core matrices)
   for (int i = tid; i < (4096 + 2048) / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_SZ)[i] = 0u;
+  // raw rows in front of the segment: earlier tokens, or the conv cache, or zeros (Section 4.1)
+  if (tid < 96) {
+    const int st = tid / 48, r = (tid % 48) / 16, oc = tid % 16;
+    const int NH = st ? a.Hkv : a.H, head = st ? j : h;
+    const int t = t_begin - HALO + r;  // token of halo row r
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (t >= 0) {
+      v = *reinterpret_cast<const uint4*>((st ? a.k : a.q) + ((size_t)b * a.T + t) * NH * D + head * D + oc * 8);
+    } else {
+      const bf16* cache = st ? a.cache_k : a.cache_q;
+      const int ci = t + (a.K - 1);  // the cache holds tokens -(K-1) .. -1, oldest first
+      if (cache && ci >= 0) v = *reinterpret_cast<const uint4*>(cache + ((size_t)b * (a.K - 1) + ci) * NH * D + head * D + oc * 8);
+    }
+    *reinterpret_cast<uint4*>(sg + OFF_HALO + ((st * 3 + r) * 16 + oc) * 16) = v;
+  }
   __syncthreads();
   if (tid < C) *reinterpret_cast<__half*>(sg + OFF_ONES + (tid >> 3) * 128 + (tid & 7) * 16) = __float2half(1.f);
-  // conv taps of this thread's channel octet (see the conv pass below)
-  const int cv_stream = tid >> 7, cv_oct = tid & 15, cv_rg = (tid >> 4) & 7;
-  float cw[8][4];
-  {
-    const bf16* w = cv_stream ? a.w_k : a.w_q;
-    const int head = cv_stream ? j : h;
-#pragma unroll
-    for (int ch = 0; ch < 8; ++ch)
-#pragma unroll
-      for (int dl = 0; dl < 4; ++dl)
-        cw[ch][dl] = dl < a.K ? __bfloat162float(w[((size_t)head * D + cv_oct * 8 + ch) * a.K + dl]) : 0.f;
-  }
   fence_proxy_async();
   tc_fence_before_sync();
   __syncthreads();
@@ -215,21 +287,22 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t tmem = (uint32_t)s_flags[0];
   const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
-  // initial state into tensor memory: thread c owns row c of [S | z]
-  if (tid < D) {
+  // initial state into tensor memory: state thread c owns row c of [S | z]
+  if (warp >= STATE_WARP0 && warp < STATE_WARP0 + 4) {
+    const int c = tid - STATE_WARP0 * 32;
     const bool have = a.S0 != nullptr && (a.seg_in || seg == 0);
     float s[32], mx = 0.f;
 #pragma unroll 1
     for (int blk = 0; blk < 4; ++blk) {
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        s[i] = have ? a.S0[(in_idx * D + tid) * D + blk * 32 + i] : 0.f;
+        s[i] = have ? a.S0[(in_idx * D + c) * D + blk * 32 + i] : 0.f;
         mx = fmaxf(mx, fabsf(s[i]));
       }
       tmem_st32(lane_base + COL_S + blk * 32, s);
     }
     const bool havez = a.z0 != nullptr && (a.seg_in || seg == 0);
-    const float z0v = havez ? a.z0[in_idx * D + tid] : 0.f;
+    const float z0v = havez ? a.z0[in_idx * D + c] : 0.f;
     tmem_st1(lane_base + COL_SZ, z0v);
     tmem_wait_st();
     mx = fmaxf(mx, fabsf(z0v));
@@ -238,203 +311,271 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
   tc_fence_before_sync();
   __syncthreads();
+  tc_fence_after_sync();
 
-  uint32_t ph_load = 0, ph_mma = 0;
-  bool store_pending = false;
+#define WAIT(b, par)                                     \
+  if (!wait_or_abort(bar(b), (uint32_t)(par), s_abort)) break
+  // for roles with barriers of their own: remember the failure, skip the work, leave at the role's next OR-barrier
+#define WAITF(b, par)                                    \
+  if (!fail && !wait_or_abort(bar(b), (uint32_t)(par), s_abort)) fail = true
 
-#define LAWCAT_WAIT_ALL(bar, phase)               \
-  do {                                            \
-    if (!mbar_wait(bar, phase)) s_flags[1] = 1;   \
-    phase ^= 1u;                                  \
-    __syncthreads();                              \
-    if (s_flags[1]) goto done;                    \
-  } while (0)
-
-  // shared-memory descriptors of the MMA operands (all tiles sit at fixed addresses); a K step adds a constant
-  const uint64_t dsc_a = smem_desc(sb + OFF_A, 16, 1024, LAYOUT_SW128);                // stacked A, K-major
-  const uint64_t dsc_w = smem_desc(sb + OFF_W, 16, 1024, LAYOUT_SW128);                // W^T, K-major
-  const uint64_t dsc_ks = smem_desc(sb + OFF_A + 8192, 16, 1024, LAYOUT_SW128);        // rows 64-127 of the stacked A
-  const uint64_t dsc_s = smem_desc(sb + OFF_SBF, 16384, 1024, LAYOUT_SW128);           // state operand, MN-major
-  const uint64_t dsc_sz = smem_desc(sb + OFF_SZ, 128, 2048, LAYOUT_NONE);
-  const uint64_t dsc_kh = smem_desc(sb + OFF_KH, 16, 1024, LAYOUT_SW128);              // kh^T, K-major
-  const uint64_t dsc_v = smem_desc(sb + OFF_V, 8192, 1024, LAYOUT_SW128);              // v, MN-major
-  const uint64_t dsc_one = smem_desc(sb + OFF_ONES, 128, 1024, LAYOUT_NONE);
-  const uint64_t dsc_p = smem_desc(sb + OFF_QRAW, 16, 1024, LAYOUT_SW128);             // masked scores, K-major
-  // start-address field steps (units of 16 bytes): K-major operand 32 B per K step, the second 64-column slab 16 KB
-  // further; MN-major swizzled operand 2048 B per K step; unswizzled [rows x 16] operand 256 B per K step
-  auto kmajor_step = [](int k) -> uint64_t { return (uint64_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2); };
-
-  for (int n = 0; n < nchunks; ++n) {
-    const int t0 = t_begin + n * C;
-    const int nvalid = min(C, t_end - t0);
-
-    // ---- TMA: raw q, k (with halo), gate, v -----------------------------------------------------------------------
-    if (tid == 0) {
-      if (store_pending) tma_store_wait_read();  // the output staging aliases the raw k tile
-      mbar_arrive_expect_tx(bar_load, MODE == 0 ? LOAD_BYTES : LOAD_BYTES - 2 * RAW_ROWS * 128);
+  if (warp == TMA_WARP) {
+    // ================================================================================================ TMA producer
+    if (lane == 0) {
+      int ar_raw = -1, ar_g = -1, ar_v = -1;  // last chunk whose copies were started, per tile
+      for (int n = 0; n < nchunks; ++n) {
+        const int t0 = t_begin + n * C;
+        const uint32_t pp = (uint32_t)((n - 1) & 1);
+        if (n > 0) WAIT(B_MMA1, pp);  // MMA 1 of the previous chunk has read the in-place conv output
+        mbar_arrive_expect_tx(bar(B_RAW_FULL), MODE == 0 ? 32768u : 16384u);
 #pragma unroll 1
-      for (int s = 0; s < 2; ++s) {
-        if (MODE == 0) tma_load_4d(sb + OFF_QRAW + s * RAW_SLAB, &tm_q, bar_load, s * 64, h, t0 - HALO, b);
-        tma_load_4d(sb + OFF_KRAW + s * RAW_SLAB, &tm_k, bar_load, s * 64, j, t0 - HALO, b);
-        tma_load_4d(sb + OFF_G + s * 8192, &tm_g, bar_load, s * 64, h, t0, b);
-        tma_load_4d(sb + OFF_V + s * 8192, &tm_v, bar_load, s * 64, j, t0, b);
-      }
-    }
-    store_pending = false;
-    LAWCAT_WAIT_ALL(bar_load, ph_load);
-    if (tid == 0) *s_rmax = 0;
-
-    // rows before the first token of the sequence come from the conv cache (TMA zero-filled them)
-    if (t0 == 0 && a.K > 1 && (a.cache_q || a.cache_k)) {
-      if (tid < 96) {
-        const int st = tid / 48, r = (tid % 48) / 16, oc = tid % 16;
-        const bf16* cache = st ? a.cache_k : a.cache_q;
-        const int ci = r - (HALO + 1) + a.K;  // cache row of token r - HALO
-        if (cache && ci >= 0 && (MODE == 0 || st == 1)) {
-          const int NH = st ? a.Hkv : a.H, head = st ? j : h;
-          const uint4 v = *reinterpret_cast<const uint4*>(cache + ((size_t)b * (a.K - 1) + ci) * NH * D + head * D + oc * 8);
-          sts128(sb + (st ? OFF_KRAW : OFF_QRAW) + (oc >> 3) * RAW_SLAB + sw128(r, oc & 7), v);
+        for (int s = 0; s < 2; ++s) {
+          if (MODE == 0) tma_load_4d(sb + OFF_AU + s * 16384, &tm_q, bar(B_RAW_FULL), s * 64, h, t0, b);
+          tma_load_4d(sb + OFF_AU + s * 16384 + 8192, &tm_k, bar(B_RAW_FULL), s * 64, j, t0, b);
         }
+        ar_raw = n;
+        if (n > 0) WAIT(B_G_FREE, pp);
+        mbar_arrive_expect_tx(bar(B_G_FULL), 16384u);
+        tma_load_4d(sb + OFF_G, &tm_g, bar(B_G_FULL), 0, h, t0, b);
+        tma_load_4d(sb + OFF_G + 8192, &tm_g, bar(B_G_FULL), 64, h, t0, b);
+        ar_g = n;
+        if (n > 0) WAIT(MODE == 0 ? B_MMA3 : B_MMA2, pp);  // the last MMA that reads v
+        mbar_arrive_expect_tx(bar(B_V_FULL), 16384u);
+        tma_load_4d(sb + OFF_V, &tm_v, bar(B_V_FULL), 0, j, t0, b);
+        tma_load_4d(sb + OFF_V + 8192, &tm_v, bar(B_V_FULL), 64, j, t0, b);
+        ar_v = n;
       }
-      __syncthreads();
-    }
-
-    // ---- conv: thread = (stream, channel octet, 8 consecutive tokens), sliding window over the raw rows -------------
-    if (MODE == 0 || cv_stream == 1) {
-      const uint32_t raw = sb + (cv_stream ? OFF_KRAW : OFF_QRAW) + (cv_oct >> 3) * RAW_SLAB;
-      const uint32_t dst = sb + OFF_A + (cv_oct >> 3) * 16384;
-      const int jc = cv_oct & 7, r0 = cv_rg * 8;
-      float x1[8], x2[8], x3[8], x0[8];
-      unpack8(lds128(raw + sw128(r0 + 0, jc)), x3);
-      unpack8(lds128(raw + sw128(r0 + 1, jc)), x2);
-      unpack8(lds128(raw + sw128(r0 + 2, jc)), x1);
-#pragma unroll 2
-      for (int i = 0; i < 8; ++i) {
-        unpack8(lds128(raw + sw128(r0 + 3 + i, jc)), x0);
-        float u[8];
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-          u[ch] = fmaf(cw[ch][0], x0[ch], fmaf(cw[ch][1], x1[ch], fmaf(cw[ch][2], x2[ch], cw[ch][3] * x3[ch])));
-        sts128(dst + sw128(cv_stream * 64 + r0 + i, jc), pack8(u, true));
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) { x3[ch] = x2[ch]; x2[ch] = x1[ch]; x1[ch] = x0[ch]; }
+      if (*s_abort) {
+        // leaving early: give the copies that are still in flight a bounded time to land before the CTA exits
+        if (ar_raw >= 0) mbar_wait(bar(B_RAW_FULL), (uint32_t)(ar_raw & 1));
+        if (ar_g >= 0) mbar_wait(bar(B_G_FULL), (uint32_t)(ar_g & 1));
+        if (ar_v >= 0) mbar_wait(bar(B_V_FULL), (uint32_t)(ar_v & 1));
       }
     }
-
-    __syncthreads();  // the raw q, k tiles are dead from here on: the exponents x take their place
-
-    // ---- gate: thread = (key channel, half of the chunk). Exponents x_t = b_t - b_mid, scanned outwards from MID. ------
-    {
-      const int c = tid & 127, half = tid >> 7, jc = (c & 63) >> 3;
-      const uint8_t* gcol = sg + OFF_G + (c >> 6) * 8192 + (c & 7) * 2;
-      // x[t][c] fp32, 512-byte rows whose 16-byte chunks are XOR-swizzled with t & 7 (conflict-free for this
-      // column-wise writer and for the row-wise readers of the phi pass)
-      float* const xcol = reinterpret_cast<float*>(sg + OFF_X) + (c & 3);
-      auto putx = [&](int t, float x) { xcol[t * 128 + (((c >> 2) ^ (t & 7)) << 2)] = x; };
-      float g[32];  // log-decays of tokens [32 half, 32 half + 32): all loaded and evaluated before the serial scan
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const int t = half * 32 + i;
-        const uint32_t raw = *reinterpret_cast<const uint16_t*>(gcol + sw128(t, jc));
-        g[i] = t < nvalid ? log2_decay(__uint_as_float(raw << 16), a.gate_mode, a.inv_tau) : 0.f;
-      }
-      float acc = 0.f;
-      if (half) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          acc += g[i];
-          putx(32 + i, fmaxf(acc, -120.f));
-        }
-        s_ft[c] = acc;
-      } else {
-        putx(MID, 0.f);
-#pragma unroll
-        for (int i = MID - 1; i >= 0; --i) {
-          acc += g[i + 1];
-          putx(i, fminf(-acc, 120.f));
-        }
-        s_bm[c] = acc + g[0];
-      }
-      // exponents are clamped to +-120 so that no factor overflows or vanishes; a clamp is reported
-      if (-acc > 120.f && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_NUMERIC);
-      const float am = warp_max(-acc);
-      if ((tid & 31) == 0) atomicMax(s_rmax, __float_as_int(am));  // g <= 0: the largest exponent magnitude
-    }
-    // ---- v: bf16 -> fp16 in place (exact for |v| in the fp16 normal range) --------------------------------------------
-    {
-      float vm = 0.f;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t ad = sb + OFF_V + (uint32_t)(tid + THREADS * i) * 16;
-        float x[8];
-        unpack8(lds128(ad), x);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) vm = fmaxf(vm, fabsf(x[e]));
-        sts128(ad, pack8(x, true));
-      }
-      vm = warp_max(vm);
-      if ((tid & 31) == 0) atomicMax(s_vmax, __float_as_int(vm < 3.0e38f ? vm : 3.0e38f));
-    }
-    fence_proxy_async();
-    __syncthreads();
-    // Operand type of this chunk (see the header): fp16 while the exponents and the state stay in range, else bf16.
-    const bool f16 = __int_as_float(*s_rmax) <= RMAX_F16 && __int_as_float(*s_sbound) < SMAX_F16;
-
-    // ---- MMA 1: Y = [u_q; u_k] W_h ------------------------------------------------------------------------------------
-    if (tid == 0) {
-      tc_fence_after_sync();
-      constexpr uint32_t ID = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_K);
+  } else if (warp == MMA_WARP) {
+    // ================================================================================================ MMA issuer
+    if (lane == 0) {
+      // shared-memory descriptors of the operands (all tiles sit at fixed addresses); a K step adds a constant to the
+      // start-address field (units of 16 bytes): K-major operand 32 B per step and 16 KB to the second 64-column slab;
+      // MN-major swizzled operand 2048 B per step; unswizzled [rows x 16] operand 256 B per step
+      const uint64_t dsc_u = smem_desc(sb + OFF_AU, 16, 1024, LAYOUT_SW128);
+      const uint64_t dsc_w = smem_desc(sb + OFF_W, 16, 1024, LAYOUT_SW128);
+      const uint64_t dsc_qk = smem_desc(sb + OFF_QK, 16, 1024, LAYOUT_SW128);
+      const uint64_t dsc_ks = smem_desc(sb + OFF_QK + 8192, 16, 1024, LAYOUT_SW128);  // rows 64-127
+      const uint64_t dsc_s = smem_desc(sb + OFF_SBF, 16384, 1024, LAYOUT_SW128);
+      const uint64_t dsc_sz = smem_desc(sb + OFF_SZ, 128, 2048, LAYOUT_NONE);
+      const uint64_t dsc_kh = smem_desc(sb + OFF_KH, 16, 1024, LAYOUT_SW128);
+      const uint64_t dsc_v = smem_desc(sb + OFF_V, 8192, 1024, LAYOUT_SW128);
+      const uint64_t dsc_one = smem_desc(sb + OFF_ONES, 128, 1024, LAYOUT_NONE);
+      const uint64_t dsc_p = smem_desc(sb + OFF_PH, 16, 1024, LAYOUT_SW128);
+      auto kstep = [](int k) -> uint64_t { return (uint64_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2); };
+      auto issue_mma1 = [&]() {
+        constexpr uint32_t ID = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_K);
 #pragma unroll 1
-      for (int k = 0; k < 8; ++k) mma_f16(tmem + COL_Y, dsc_a + kmajor_step(k), dsc_w + kmajor_step(k), ID, k > 0);
-      mma_commit(bar_mma);
-    }
-
-    // ---- state pass (overlaps MMA 1): operand 2^b_mid * [S|z] in 16 bit, accumulator [S|z] *= 2^b_C -----------------
-    if (tid < D) {
-      const int c = tid;
-      const float bm = s_bm[c], ft = s_ft[c];
-      const float dm = ex2f(bm), dC = ex2f(bm + ft);
-      s_e63[c] = ex2f(fmaxf(ft, -120.f));
-      dsum += bm + ft;
-      float s[32], mx = 0.f;
-#pragma unroll 1
-      for (int blk = 0; blk < 4; ++blk) {
-        tmem_ld32(lane_base + COL_S + blk * 32, s);
-        tmem_wait_ld();
+        for (int k = 0; k < 8; ++k) mma_f16(tmem + COL_Y, dsc_u + kstep(k), dsc_w + kstep(k), ID, k > 0);
+        mma_commit(bar(B_MMA1));
+      };
+      bool ok = nchunks > 0;
+      if (ok) ok = wait_or_abort(bar(B_U_FULL), 0u, s_abort);
+      if (ok) {
+        tc_fence_after_sync();
+        issue_mma1();
+      }
+      for (int n = 0; ok && n < nchunks; ++n) {
+        const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
+        WAIT(B_QK_FULL, p);
+        WAIT(B_SBF_FULL, p);
+        WAIT(B_VH_FULL, p);
+        if (MODE == 0 && n > 0) WAIT(B_O_FREE, pp);
+        tc_fence_after_sync();
         if (MODE == 0) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(s[i]));
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            float w[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) w[i] = dm * s[8 * q4 + i];
-            sts128(sb + OFF_SBF + (blk >> 1) * 16384 + sw128(c, (blk & 1) * 4 + q4), pack8(w, f16));
+          const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
+          const int fmt = f16 ? FMT_F16 : FMT_BF16;
+          const uint32_t ID_P = instr_desc(128, 64, fmt, MAJOR_K, MAJOR_K);
+          const uint32_t ID_O = instr_desc(128, 128, fmt, MAJOR_K, MAJOR_MN);
+          const uint32_t ID_OZ = instr_desc(128, 16, fmt, MAJOR_K, MAJOR_MN);
+#pragma unroll 1
+          for (int k = 0; k < 8; ++k) {
+            const uint64_t ad = dsc_qk + kstep(k);
+            mma_f16(tmem + COL_P, ad, dsc_ks + kstep(k), ID_P, k > 0);
+            mma_f16(tmem + COL_O, ad, dsc_s + (uint64_t)(k * (2048 >> 4)), ID_O, k > 0);
+            mma_f16(tmem + COL_OZ, ad, dsc_sz + (uint64_t)(k * (256 >> 4)), ID_OZ, k > 0);
           }
         }
-#pragma unroll
-        for (int i = 0; i < 32; ++i) s[i] *= dC;
-        tmem_st32(lane_base + COL_S + blk * 32, s);
+        {
+          constexpr uint32_t ID_S = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
+          constexpr uint32_t ID_SZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
+#pragma unroll 1
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t ad = dsc_kh + (uint64_t)(k * 2);
+            mma_f16(tmem + COL_S, ad, dsc_v + (uint64_t)(k * (2048 >> 4)), ID_S, 1);
+            mma_f16(tmem + COL_SZ, ad, dsc_one + (uint64_t)(k * (256 >> 4)), ID_SZ, 1);
+          }
+          mma_commit(bar(B_MMA2));
+        }
+        if (n + 1 < nchunks) {  // the mix of the next chunk, ahead of this chunk's last product
+          WAIT(B_U_FULL, pp);
+          WAIT(B_Y_FREE, p);
+          tc_fence_after_sync();
+          issue_mma1();
+        }
+        if (MODE == 0) {
+          WAIT(B_PH_FULL, p);
+          tc_fence_after_sync();
+          constexpr uint32_t ID_O = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
+          constexpr uint32_t ID_OZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
+#pragma unroll 1
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t ad = dsc_p + (uint64_t)(k * 2);
+            mma_f16(tmem + COL_O, ad, dsc_v + (uint64_t)(k * (2048 >> 4)), ID_O, 1);
+            mma_f16(tmem + COL_OZ, ad, dsc_one + (uint64_t)(k * (256 >> 4)), ID_OZ, 1);
+          }
+          mma_commit(bar(B_MMA3));
+        }
       }
-      const float z = tmem_ld1(lane_base + COL_SZ);
-      tmem_wait_ld();
-      if (MODE == 0) {
-        *reinterpret_cast<uint16_t*>(sg + OFF_SZ + (c >> 3) * 128 + (c & 7) * 16) = to16(dm * z, f16);
-        mx = warp_max(fmaxf(mx, fabsf(z)));
-        if ((tid & 31) == 0) atomicMax(s_smax, __float_as_int(mx < 3.0e38f ? mx : 3.0e38f));
-      }
-      tmem_st1(lane_base + COL_SZ, dC * z);
-      tmem_wait_st();
     }
-    LAWCAT_WAIT_ALL(bar_mma, ph_mma);
-    tc_fence_after_sync();
+  } else if (warp < ROW_WARP0) {
+    // ================================================================================================ prep warps
+    // conv mapping: thread = (stream, channel octet, 8 consecutive tokens); gate mapping: thread = (channel, half chunk)
+    const int cv_stream = tid >> 7, cv_oct = tid & 15, cv_rg = (tid >> 4) & 7;
+    const bool cv_on = MODE == 0 || cv_stream == 1;
+    float cw[8][4];
+    {
+      const bf16* w = cv_stream ? a.w_k : a.w_q;
+      const int head = cv_stream ? j : h;
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch)
+#pragma unroll
+        for (int dl = 0; dl < 4; ++dl)
+          cw[ch][dl] = dl < a.K ? __bfloat162float(w[((size_t)head * D + cv_oct * 8 + ch) * a.K + dl]) : 0.f;
+    }
+    const uint32_t au = sb + OFF_AU + (cv_oct >> 3) * 16384;  // this thread's 64-channel slab
+    const int cjc = cv_oct & 7, crow0 = cv_stream * 64 + cv_rg * 8;
+    const int gc = tid & 127, ghalf = tid >> 7, gjc = (gc & 63) >> 3;
+    bool fail = false;
+    for (int n = 0; n < nchunks; ++n) {
+      const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
+      const int nvalid = min(C, t_end - (t_begin + n * C));
+      // ---- conv, in place: the three rows in front of this thread's rows belong to another thread (or to the previous
+      // chunk), so they are read before the barrier and every row is overwritten only after it ------------------------
+      WAITF(B_RAW_FULL, p);
+      float x1[8], x2[8], x3[8], x0[8];
+      if (cv_on && !fail) {
+        if (cv_rg == 0) {
+          const uint4* hl = reinterpret_cast<const uint4*>(sg + OFF_HALO) + cv_stream * 48 + cv_oct;
+          unpack8(hl[0], x3); unpack8(hl[16], x2); unpack8(hl[32], x1);
+        } else {
+          unpack8(lds128(au + sw128(crow0 - 3, cjc)), x3);
+          unpack8(lds128(au + sw128(crow0 - 2, cjc)), x2);
+          unpack8(lds128(au + sw128(crow0 - 1, cjc)), x1);
+        }
+      }
+      if (tid == 0) { s_rmax[p] = 0; s_vmax[p] = 0; }
+      fail = named_bar_or(1, PREP_THREADS, fail);
+      if (fail) break;
+      if (cv_on) {
+#pragma unroll 2
+        for (int i = 0; i < 8; ++i) {
+          const uint32_t ad = au + sw128(crow0 + i, cjc);
+          unpack8(lds128(ad), x0);
+          float u[8];
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch)
+            u[ch] = fmaf(cw[ch][0], x0[ch], fmaf(cw[ch][1], x1[ch], fmaf(cw[ch][2], x2[ch], cw[ch][3] * x3[ch])));
+          sts128(ad, pack8(u, true));
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch) { x3[ch] = x2[ch]; x2[ch] = x1[ch]; x1[ch] = x0[ch]; }
+        }
+        if (cv_rg == 7) {  // the last three raw rows of the chunk are the next chunk's halo (bf16 values: exact repack)
+          uint4* hl = reinterpret_cast<uint4*>(sg + OFF_HALO) + cv_stream * 48 + cv_oct;
+          hl[0] = pack8(x3, false); hl[16] = pack8(x2, false); hl[32] = pack8(x1, false);
+        }
+      }
+      fence_proxy_async();
+      named_bar_sync(1, PREP_THREADS);
+      mbar_arrive(bar(B_U_FULL));
 
-    // ---- phi: one thread per row of Y, 32 columns at a time -------------------------------------------------------
-    if (tid < D && (MODE == 0 || tid >= C)) {
-      const float L2E = 1.4426950408889634f;
-      const int row = tid < C ? tid : tid - C;  // token of this row (query rows 0-63, key rows 64-127 of Y)
+      // ---- gate: exponents x_t = b_t - b_mid, scanned outwards from MID ------------------------------------------------
+      WAITF(B_G_FULL, p);
+      if (n > 0) WAITF(B_X_FREE, pp);
+      if (!fail) {
+        const uint8_t* gcol = sg + OFF_G + (gc >> 6) * 8192 + (gc & 7) * 2;
+        // x[t][c] fp32, 512-byte rows whose 16-byte chunks are XOR-swizzled with t & 7 (conflict-free for this
+        // column-wise writer and for the row-wise readers of the phi pass)
+        float* const xcol = reinterpret_cast<float*>(sg + OFF_X) + (gc & 3);
+        auto putx = [&](int t, float x) { xcol[t * 128 + (((gc >> 2) ^ (t & 7)) << 2)] = x; };
+        float g[32];  // log-decays of tokens [32 half, 32 half + 32): all evaluated before the serial scan
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int t = ghalf * 32 + i;
+          const uint32_t raw = *reinterpret_cast<const uint16_t*>(gcol + sw128(t, gjc));
+          g[i] = t < nvalid ? log2_decay(__uint_as_float(raw << 16), a.gate_mode, a.inv_tau) : 0.f;
+        }
+        float acc = 0.f;
+        if (ghalf) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            acc += g[i];
+            putx(32 + i, fmaxf(acc, -120.f));
+          }
+          vec(p, 1)[gc] = acc;                           // ft = b_C - b_mid
+          vec(p, 2)[gc] = ex2f(fmaxf(acc, -120.f));      // 2^ft
+        } else {
+          putx(MID, 0.f);
+#pragma unroll
+          for (int i = MID - 1; i >= 0; --i) {
+            acc += g[i + 1];
+            putx(i, fminf(-acc, 120.f));
+          }
+          vec(p, 0)[gc] = acc + g[0];                    // bm = b_mid
+        }
+        // exponents are clamped to +-120 so that no factor overflows or vanishes; a clamp is reported
+        if (-acc > 120.f && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_NUMERIC);
+        const float am = warp_max(-acc);
+        if (lane == 0) atomicMax(&s_rmax[p], __float_as_int(am));  // g <= 0: the largest exponent magnitude
+      }
+      mbar_arrive(bar(B_G_FREE));
+      mbar_arrive(bar(B_X_FULL));
+
+      // ---- v: bf16 -> fp16 in place (exact for |v| in the fp16 normal range) ------------------------------------------
+      WAITF(B_V_FULL, p);
+      if (!fail) {
+        float vm = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t ad = sb + OFF_V + (uint32_t)(tid + PREP_THREADS * i) * 16;
+          float x[8];
+          unpack8(lds128(ad), x);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) vm = fmaxf(vm, fabsf(x[e]));
+          sts128(ad, pack8(x, true));
+        }
+        vm = warp_max(vm);
+        if (lane == 0) atomicMax(&s_vmax[p], __float_as_int(vm < 3.0e38f ? vm : 3.0e38f));
+      }
+      fence_proxy_async();
+      mbar_arrive(bar(B_VH_FULL));
+    }
+  } else if (warp < STATE_WARP0) {
+    // ================================================================================================ row warps
+    // thread = one row of Y: rows 0-63 the query tokens (these threads also mask the scores and write the output),
+    // rows 64-127 the key tokens
+    const int rt = tid - ROW_WARP0 * 32;
+    const bool is_q = rt < C;
+    const int row = is_q ? rt : rt - C;
+    const float L2E = 1.4426950408889634f;
+    const bool need_qsum = a.eps != 0.f;  // the dropped softmax normalizer of the query rows only matters next to eps
+    for (int n = 0; n < nchunks && (MODE == 0 || !is_q); ++n) {
+      const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
+      const int t0 = t_begin + n * C;
+      const int nvalid = min(C, t_end - t0);
+      WAIT(B_X_FULL, p);
+      WAIT(B_MMA1, p);
+      if (n > 0) WAIT(B_MMA2, pp);  // qs / ks / kh of the previous chunk have been consumed
+      tc_fence_after_sync();
+      const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
       float y[32];
-      float m = -INFINITY;
+      float m = -INFINITY, qsum = 0.f;
 #pragma unroll 1
       for (int blk = 0; blk < 4; ++blk) {
         tmem_ld32(lane_base + COL_Y + blk * 32, y);
@@ -443,9 +584,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         for (int i = 0; i < 32; ++i) m = fmaxf(m, y[i]);
       }
       const float mb = m * L2E;
-      if (tid < C) {
-        float qsum = 0.f;
-        const bool need_qsum = a.eps != 0.f;  // the dropped normalizer only matters next to eps
+      if (is_q) {
 #pragma unroll 1
         for (int blk = 0; blk < 4; ++blk) {
           tmem_ld32(lane_base + COL_Y + blk * 32, y);
@@ -460,10 +599,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
               for (int i = 0; i < 8; ++i) qsum += ex2f(fmaf(y[q4 * 8 + i], L2E, -mb));
             }
-            sts128(sb + OFF_A + (blk >> 1) * 16384 + sw128(row, (blk & 1) * 4 + q4), pack8(v, f16));
+            sts128(sb + OFF_QK + (blk >> 1) * 16384 + sw128(row, (blk & 1) * 4 + q4), pack8(v, f16));
           }
         }
-        s_qsum[row] = qsum;
       } else {
         // key rows: a first sweep for the softmax sum, a second for ks = phi_k 2^-x and kh = ks 2^(b_C - b_mid)
         float sum = 0.f;
@@ -475,6 +613,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           for (int i = 0; i < 32; ++i) sum += ex2f(fmaf(y[i], L2E, -mb));
         }
         const float inv = row < nvalid ? 1.f / sum : 0.f;  // tokens past the end contribute nothing
+        const float* e63v = vec(p, 2);
 #pragma unroll 1
         for (int blk = 0; blk < 4; ++blk) {
           tmem_ld32(lane_base + COL_Y + blk * 32, y);
@@ -484,12 +623,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int jj = blk * 4 + q4;  // channels [8 jj, 8 jj + 8)
             float x[8], ks[8];
             load_x8(sb + OFF_X, row, jj, x);
-            const float4 ea = *reinterpret_cast<const float4*>(s_e63 + jj * 8);
-            const float4 eb = *reinterpret_cast<const float4*>(s_e63 + jj * 8 + 4);
+            const float4 ea = *reinterpret_cast<const float4*>(e63v + jj * 8);
+            const float4 eb = *reinterpret_cast<const float4*>(e63v + jj * 8 + 4);
             const float e63[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
 #pragma unroll
             for (int i = 0; i < 8; ++i) ks[i] = ex2f(fmaf(y[q4 * 8 + i], L2E, -mb - x[i])) * inv;
-            if (MODE == 0) sts128(sb + OFF_A + (jj >> 3) * 16384 + sw128(C + row, jj & 7), pack8(ks, f16));
+            if (MODE == 0) sts128(sb + OFF_QK + (jj >> 3) * 16384 + sw128(C + row, jj & 7), pack8(ks, f16));
             // kh^T: row = key channel, 64 tokens (128 bytes) per row, so that the state update reads a K-major A operand
 #pragma unroll
             for (int i = 0; i < 8; ++i)
@@ -498,140 +637,146 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
         }
       }
-    }
-    fence_proxy_async();
-    tc_fence_before_sync();
-    __syncthreads();
-
-    // ---- MMA 2: scores, inter-chunk read-out, state update ---------------------------------------------------------
-    if (tid == 0) {
-      tc_fence_after_sync();
-      if (MODE == 0) {
-        const int fmt = f16 ? FMT_F16 : FMT_BF16;
-        const uint32_t ID_P = instr_desc(128, 64, fmt, MAJOR_K, MAJOR_K);
-        const uint32_t ID_O = instr_desc(128, 128, fmt, MAJOR_K, MAJOR_MN);
-        const uint32_t ID_OZ = instr_desc(128, 16, fmt, MAJOR_K, MAJOR_MN);
-        // bound on the state after this chunk's update, for the next chunk's choice of operand type
-        *s_sbound = __float_as_int(__int_as_float(*s_smax) + 64.f * fmaxf(__int_as_float(*s_vmax), 1.f));
-        *s_smax = 0;
-        *s_vmax = 0;
-#pragma unroll 1
-        for (int k = 0; k < 8; ++k) {
-          const uint64_t ad = dsc_a + kmajor_step(k);
-          mma_f16(tmem + COL_P, ad, dsc_ks + kmajor_step(k), ID_P, k > 0);
-          mma_f16(tmem + COL_O, ad, dsc_s + (uint64_t)(k * (2048 >> 4)), ID_O, k > 0);
-          mma_f16(tmem + COL_OZ, ad, dsc_sz + (uint64_t)(k * (256 >> 4)), ID_OZ, k > 0);
-        }
-      }
-      constexpr uint32_t ID_S = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
-      constexpr uint32_t ID_SZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
-#pragma unroll 1
-      for (int k = 0; k < 4; ++k) {
-        const uint64_t ad = dsc_kh + (uint64_t)(k * 2);
-        mma_f16(tmem + COL_S, ad, dsc_v + (uint64_t)(k * (2048 >> 4)), ID_S, 1);
-        mma_f16(tmem + COL_SZ, ad, dsc_one + (uint64_t)(k * (256 >> 4)), ID_SZ, 1);
-      }
-      mma_commit(bar_mma);
-    }
-    LAWCAT_WAIT_ALL(bar_mma, ph_mma);
-    tc_fence_after_sync();
-
-    if (MODE == 0) {
-      // ---- causal mask, fp16 scores ---------------------------------------------------------------------------------
-      if (tid < C) {
-        const int t = tid;
-        float p[32];
+      fence_proxy_async();
+      tc_fence_before_sync();
+      mbar_arrive(bar(B_Y_FREE));
+      mbar_arrive(bar(B_X_FREE));
+      mbar_arrive(bar(B_QK_FULL));
+      if (MODE == 0 && is_q) {
+        // ---- causal mask, fp16 scores -------------------------------------------------------------------------------
+        WAIT(B_MMA2, p);
+        tc_fence_after_sync();
 #pragma unroll 1
         for (int blk = 0; blk < 2; ++blk) {
-          tmem_ld32(lane_base + COL_P + blk * 32, p);
+          tmem_ld32(lane_base + COL_P + blk * 32, y);
           tmem_wait_ld();
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) {
             float v[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = (blk * 32 + q4 * 8 + i <= t) ? p[q4 * 8 + i] : 0.f;
-            sts128(sb + OFF_QRAW + sw128(t, blk * 4 + q4), pack8(v, true));
+            for (int i = 0; i < 8; ++i) v[i] = (blk * 32 + q4 * 8 + i <= row) ? y[q4 * 8 + i] : 0.f;
+            sts128(sb + OFF_PH + sw128(row, blk * 4 + q4), pack8(v, true));
           }
         }
-      }
-      fence_proxy_async();
-      tc_fence_before_sync();
-      __syncthreads();
-
-      // ---- MMA 3: O' += P [v|1] ---------------------------------------------------------------------------------------
-      if (tid == 0) {
+        fence_proxy_async();
+        tc_fence_before_sync();
+        mbar_arrive(bar(B_PH_FULL));
+        // ---- normalize (Eq. 8) and store ------------------------------------------------------------------------------
+        WAIT(B_MMA3, p);
         tc_fence_after_sync();
-        constexpr uint32_t ID_O = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
-        constexpr uint32_t ID_OZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
-#pragma unroll 1
-        for (int k = 0; k < 4; ++k) {
-          const uint64_t ad = dsc_p + (uint64_t)(k * 2);
-          mma_f16(tmem + COL_O, ad, dsc_v + (uint64_t)(k * (2048 >> 4)), ID_O, 1);
-          mma_f16(tmem + COL_OZ, ad, dsc_one + (uint64_t)(k * (256 >> 4)), ID_OZ, 1);
-        }
-        mma_commit(bar_mma);
-      }
-      LAWCAT_WAIT_ALL(bar_mma, ph_mma);
-      tc_fence_after_sync();
-
-      // ---- normalize (Eq. 8), stage, store ----------------------------------------------------------------------------
-      if (tid < C) {
-        const int t = tid;
         const float den = tmem_ld1(lane_base + COL_OZ);
         tmem_wait_ld();
         // the query features went in scaled by qsum (unnormalized softmax), so eps scales the same way
-        const float inv = 1.f / (den + a.eps * s_qsum[t]);
-        float o[32];
+        const float inv = 1.f / (den + a.eps * qsum);
+        bf16* orow = a.o + (((size_t)b * a.T + t0 + row) * a.H + h) * D;
 #pragma unroll 1
         for (int blk = 0; blk < 4; ++blk) {
-          tmem_ld32(lane_base + COL_O + blk * 32, o);
+          tmem_ld32(lane_base + COL_O + blk * 32, y);
           tmem_wait_ld();
+          if (blk == 3) {  // O' is in registers: the next chunk's products may overwrite it
+            tc_fence_before_sync();
+            mbar_arrive(bar(B_O_FREE));
+          }
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] *= inv;
+          for (int i = 0; i < 32; ++i) y[i] *= inv;
+          if (row < nvalid) {
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4)
-            sts128(sb + OFF_KRAW + (blk >> 1) * 8192 + sw128(t, (blk & 1) * 4 + q4), pack8(o + 8 * q4, false));
+            for (int q4 = 0; q4 < 4; ++q4) *reinterpret_cast<uint4*>(orow + blk * 32 + q4 * 8) = pack8(y + 8 * q4, false);
+          }
         }
       }
+    }
+  } else {
+    // ================================================================================================ state warps
+    // thread c = row c of [S | z]: per chunk the 16-bit operand 2^b_mid [S|z] and the decay [S|z] *= 2^b_C
+    const int c = tid - STATE_WARP0 * 32;
+    float dsum = 0.f;  // log2 of this channel's total decay over the segment
+    bool fail = false;
+    for (int n = 0; n < nchunks; ++n) {
+      const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
+      WAITF(B_X_FULL, p);
+      if (n > 0) WAITF(B_MMA2, pp);  // the previous chunk's update has landed; its state operand has been consumed
+      if (!fail) {
+        tc_fence_after_sync();
+        const float bm = vec(p, 0)[c], ft = vec(p, 1)[c];
+        mbar_arrive(bar(B_X_FREE));
+        const float dm = ex2f(bm), dC = ex2f(bm + ft);
+        dsum += bm + ft;
+        const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
+        float s[32], mx = 0.f;
+#pragma unroll 1
+        for (int blk = 0; blk < 4; ++blk) {
+          tmem_ld32(lane_base + COL_S + blk * 32, s);
+          tmem_wait_ld();
+          if (MODE == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(s[i]));
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              float w[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) w[i] = dm * s[8 * q4 + i];
+              sts128(sb + OFF_SBF + (blk >> 1) * 16384 + sw128(c, (blk & 1) * 4 + q4), pack8(w, f16));
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) s[i] *= dC;
+          tmem_st32(lane_base + COL_S + blk * 32, s);
+        }
+        const float z = tmem_ld1(lane_base + COL_SZ);
+        tmem_wait_ld();
+        if (MODE == 0) {
+          *reinterpret_cast<uint16_t*>(sg + OFF_SZ + (c >> 3) * 128 + (c & 7) * 16) = to16(dm * z, f16);
+          mx = warp_max(fmaxf(mx, fabsf(z)));
+          if (lane == 0) atomicMax(s_smax, __float_as_int(mx < 3.0e38f ? mx : 3.0e38f));
+        }
+        tmem_st1(lane_base + COL_SZ, dC * z);
+        tmem_wait_st();
+      }
+      WAITF(B_VH_FULL, p);  // the chunk's max|v| is known
       fence_proxy_async();
       tc_fence_before_sync();
-      __syncthreads();
-      if (tid == 0) {
-        tma_store_4d(&tm_o, sb + OFF_KRAW, 0, h, t0, b);
-        tma_store_4d(&tm_o, sb + OFF_KRAW + 8192, 64, h, t0, b);
-        tma_store_commit();
+      fail = named_bar_or(2, 128, fail);
+      if (fail) break;
+      if (MODE == 0 && c == 0) {
+        // bound on the state after this chunk's update: the next chunk's choice of operand type
+        s_sbound[pp] = __float_as_int(__int_as_float(*s_smax) + 64.f * fmaxf(__int_as_float(s_vmax[p]), 1.f));
+        *s_smax = 0;
+        __threadfence_block();
       }
-      store_pending = true;
+      mbar_arrive(bar(B_SBF_FULL));
     }
-  }
-
-  // ---- final state ---------------------------------------------------------------------------------------------------
-  tc_fence_after_sync();
-  if (tid < D && a.dtot != nullptr) a.dtot[seg_idx * D + tid] = dsum;
-  if (tid < D && a.S_T != nullptr && (a.seg_out || seg == a.nseg - 1)) {
-    float s[32];
+    // ---- final state -------------------------------------------------------------------------------------------------
+    if (!fail && !*s_abort && (nchunks == 0 || wait_or_abort(bar(B_MMA2), (uint32_t)((nchunks - 1) & 1), s_abort))) {
+      tc_fence_after_sync();
+      if (a.dtot != nullptr) a.dtot[seg_idx * D + c] = dsum;
+      if (a.S_T != nullptr && (a.seg_out || seg == a.nseg - 1)) {
+        float s[32];
 #pragma unroll 1
-    for (int blk = 0; blk < 4; ++blk) {
-      tmem_ld32(lane_base + COL_S + blk * 32, s);
-      tmem_wait_ld();
+        for (int blk = 0; blk < 4; ++blk) {
+          tmem_ld32(lane_base + COL_S + blk * 32, s);
+          tmem_wait_ld();
 #pragma unroll
-      for (int i = 0; i < 32; i += 4)
-        *reinterpret_cast<float4*>(a.S_T + (out_idx * D + tid) * D + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
+          for (int i = 0; i < 32; i += 4)
+            *reinterpret_cast<float4*>(a.S_T + (out_idx * D + c) * D + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
+        }
+        const float z = tmem_ld1(lane_base + COL_SZ);
+        tmem_wait_ld();
+        if (a.z_T) a.z_T[out_idx * D + c] = z;
+      }
     }
-    const float z = tmem_ld1(lane_base + COL_SZ);
-    tmem_wait_ld();
-    if (a.z_T) a.z_T[out_idx * D + tid] = z;
   }
+#undef WAIT
+#undef WAITF
 
-done:
-  if (tid == 0) {
-    tma_store_wait_all();
-    if (s_flags[1] && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_TIMEOUT);
-  }
+  // ---- teardown --------------------------------------------------------------------------------------------------------
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
-#undef LAWCAT_WAIT_ALL
+  if (tid == 0 && *s_abort && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_TIMEOUT);
+  if (warp == MMA_WARP) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
 }
 
 }  // namespace tc
