@@ -138,13 +138,11 @@ __device__ __forceinline__ void load_x8(uint32_t base, int t, int jj, float* x) 
   x[4] = __uint_as_float(hi.x); x[5] = __uint_as_float(hi.y); x[6] = __uint_as_float(hi.z); x[7] = __uint_as_float(hi.w);
 }
 
-// log2 of the decay of one gate entry: LOGITS: log2(sigmoid(a)) / tau, LOGDECAY: a * log2(e).
-__device__ __forceinline__ float log2_decay(float a, int gate_mode, float inv_tau) {
-  const float L2E = 1.4426950408889634f;
-  if (gate_mode == LAWCAT_GATE_LOGDECAY) return a * L2E;
-  // -log2(1 + 2^x) with 2^x = exp(-a), branch-free: the clamp keeps 2^x finite, and beyond it log2(1 + 2^x) = x
-  const float x = -a * L2E;
-  return -fmaxf(x, lg2f(1.f + ex2f(fminf(x, 126.f)))) * inv_tau;
+// log2(sigmoid(a)) = -log2(1 + 2^x) with 2^x = exp(-a); branch-free: the clamp keeps 2^x finite, and beyond it
+// log2(1 + 2^x) = x to fp32 accuracy.
+__device__ __forceinline__ float log2_sigmoid(float a) {
+  const float x = -a * 1.4426950408889634f;
+  return -fmaxf(x, lg2f(1.f + ex2f(fminf(x, 126.f))));
 }
 
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
@@ -497,20 +495,37 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
       // ---- gate: exponents x_t = b_t - b_mid, scanned outwards from MID ------------------------------------------------
       WAITF(B_G_FULL, p);
-      if (n > 0) WAITF(B_X_FREE, pp);
-      if (!fail) {
+      {
         const uint8_t* gcol = sg + OFF_G + (gc >> 6) * 8192 + (gc & 7) * 2;
         // x[t][c] fp32, 512-byte rows whose 16-byte chunks are XOR-swizzled with t & 7 (conflict-free for this
         // column-wise writer and for the row-wise readers of the phi pass)
         float* const xcol = reinterpret_cast<float*>(sg + OFF_X) + (gc & 3);
         auto putx = [&](int t, float x) { xcol[t * 128 + (((gc >> 2) ^ (t & 7)) << 2)] = x; };
-        float g[32];  // log-decays of tokens [32 half, 32 half + 32): all evaluated before the serial scan
+        // log-decays of tokens [32 half, 32 half + 32): all evaluated before the serial scan. The mode and the ragged
+        // tail are decided outside the loops: a branch around each special-function instruction costs more than it.
+        float g[32];
+        const float L2E = 1.4426950408889634f;
+        if (a.gate_mode == LAWCAT_GATE_LOGDECAY) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int t = ghalf * 32 + i;
-          const uint32_t raw = *reinterpret_cast<const uint16_t*>(gcol + sw128(t, gjc));
-          g[i] = t < nvalid ? log2_decay(__uint_as_float(raw << 16), a.gate_mode, a.inv_tau) : 0.f;
+          for (int i = 0; i < 32; ++i) {
+            const uint32_t raw = *reinterpret_cast<const uint16_t*>(gcol + sw128(ghalf * 32 + i, gjc));
+            g[i] = __uint_as_float(raw << 16) * L2E;
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const uint32_t raw = *reinterpret_cast<const uint16_t*>(gcol + sw128(ghalf * 32 + i, gjc));
+            g[i] = log2_sigmoid(__uint_as_float(raw << 16)) * a.inv_tau;
+          }
         }
+        if (nvalid < C) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (ghalf * 32 + i >= nvalid) g[i] = 0.f;  // tokens past the end: no decay
+        }
+        // the exponent tile is free once the previous chunk's phi pass has read it; the log-decays above did not need it
+        mbar_arrive(bar(B_G_FREE));
+        if (n > 0) WAITF(B_X_FREE, pp);
         float acc = 0.f;
         if (ghalf) {
 #pragma unroll
@@ -534,7 +549,6 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const float am = warp_max(-acc);
         if (lane == 0) atomicMax(&s_rmax[p], __float_as_int(am));  // g <= 0: the largest exponent magnitude
       }
-      mbar_arrive(bar(B_G_FREE));
       mbar_arrive(bar(B_X_FULL));
 
       // ---- v: bf16 -> fp16 in place (exact for |v| in the fp16 normal range) ------------------------------------------
@@ -574,60 +588,85 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (n > 0) WAIT(B_MMA2, pp);  // qs / ks / kh of the previous chunk have been consumed
       tc_fence_after_sync();
       const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
+      // Y is read 16 columns at a time with the next load in flight while a block is processed
+      float ya[16], yb[16];
       float y[32];
       float m = -INFINITY, qsum = 0.f;
+      tmem_ld16(lane_base + COL_Y, ya);
 #pragma unroll 1
-      for (int blk = 0; blk < 4; ++blk) {
-        tmem_ld32(lane_base + COL_Y + blk * 32, y);
+      for (int b2 = 0; b2 < 4; ++b2) {
         tmem_wait_ld();
+        tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) m = fmaxf(m, y[i]);
+        for (int i = 0; i < 16; ++i) m = fmaxf(m, ya[i]);
+        tmem_wait_ld();
+        tmem_ld16(lane_base + COL_Y + ((b2 * 32 + 32) & 127), ya);  // wraps to column 0: the first block of the next sweep
+#pragma unroll
+        for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
       }
       const float mb = m * L2E;
       if (is_q) {
-#pragma unroll 1
-        for (int blk = 0; blk < 4; ++blk) {
-          tmem_ld32(lane_base + COL_Y + blk * 32, y);
-          tmem_wait_ld();
+        auto q_block = [&](const float* yy, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int jj = jj0 + h2;
             float x[8], v[8];
-            load_x8(sb + OFF_X, row, blk * 4 + q4, x);
+            load_x8(sb + OFF_X, row, jj, x);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = ex2f(fmaf(y[q4 * 8 + i], L2E, x[i] - mb));
+            for (int i = 0; i < 8; ++i) v[i] = ex2f(fmaf(yy[h2 * 8 + i], L2E, x[i] - mb));
             if (need_qsum) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i) qsum += ex2f(fmaf(y[q4 * 8 + i], L2E, -mb));
+              for (int i = 0; i < 8; ++i) qsum += ex2f(fmaf(yy[h2 * 8 + i], L2E, -mb));
             }
-            sts128(sb + OFF_QK + (blk >> 1) * 16384 + sw128(row, (blk & 1) * 4 + q4), pack8(v, f16));
+            sts128(sb + OFF_QK + (jj >> 3) * 16384 + sw128(row, jj & 7), pack8(v, f16));
           }
+        };
+#pragma unroll 1
+        for (int b2 = 0; b2 < 4; ++b2) {
+          tmem_wait_ld();
+          tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
+          q_block(ya, b2 * 4);
+          tmem_wait_ld();
+          if (b2 < 3) tmem_ld16(lane_base + COL_Y + b2 * 32 + 32, ya);
+          q_block(yb, b2 * 4 + 2);
         }
       } else {
-        // key rows: a first sweep for the softmax sum, a second for ks = phi_k 2^-x and kh = ks 2^(b_C - b_mid)
+        // key rows: one sweep forms e = exp(y - max) and its sum and parks e in Y's own columns; the last sweep
+        // writes ks = e 2^-x / sum and kh = ks 2^(b_C - b_mid)
         float sum = 0.f;
 #pragma unroll 1
-        for (int blk = 0; blk < 4; ++blk) {
-          tmem_ld32(lane_base + COL_Y + blk * 32, y);
+        for (int b2 = 0; b2 < 4; ++b2) {
           tmem_wait_ld();
+          tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) sum += ex2f(fmaf(y[i], L2E, -mb));
+          for (int i = 0; i < 16; ++i) {
+            ya[i] = ex2f(fmaf(ya[i], L2E, -mb));
+            sum += ya[i];
+          }
+          tmem_st16(lane_base + COL_Y + b2 * 32, ya);
+          tmem_wait_ld();
+          if (b2 < 3) tmem_ld16(lane_base + COL_Y + b2 * 32 + 32, ya);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            yb[i] = ex2f(fmaf(yb[i], L2E, -mb));
+            sum += yb[i];
+          }
+          tmem_st16(lane_base + COL_Y + b2 * 32 + 16, yb);
         }
+        tmem_wait_st();
         const float inv = row < nvalid ? 1.f / sum : 0.f;  // tokens past the end contribute nothing
         const float* e63v = vec(p, 2);
-#pragma unroll 1
-        for (int blk = 0; blk < 4; ++blk) {
-          tmem_ld32(lane_base + COL_Y + blk * 32, y);
-          tmem_wait_ld();
+        auto k_block = [&](const float* ee, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            const int jj = blk * 4 + q4;  // channels [8 jj, 8 jj + 8)
+          for (int h2 = 0; h2 < 2; ++h2) {
+            const int jj = jj0 + h2;  // channels [8 jj, 8 jj + 8)
             float x[8], ks[8];
             load_x8(sb + OFF_X, row, jj, x);
             const float4 ea = *reinterpret_cast<const float4*>(e63v + jj * 8);
             const float4 eb = *reinterpret_cast<const float4*>(e63v + jj * 8 + 4);
             const float e63[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
 #pragma unroll
-            for (int i = 0; i < 8; ++i) ks[i] = ex2f(fmaf(y[q4 * 8 + i], L2E, -mb - x[i])) * inv;
+            for (int i = 0; i < 8; ++i) ks[i] = ee[h2 * 8 + i] * inv * ex2f(-x[i]);
             if (MODE == 0) sts128(sb + OFF_QK + (jj >> 3) * 16384 + sw128(C + row, jj & 7), pack8(ks, f16));
             // kh^T: row = key channel, 64 tokens (128 bytes) per row, so that the state update reads a K-major A operand
 #pragma unroll
@@ -635,6 +674,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               *reinterpret_cast<__half*>(sg + OFF_KH + (jj * 8 + i) * 128 + (((row >> 3) ^ i) << 4) + (row & 7) * 2) =
                   __float2half_rn(ks[i] * e63[i]);
           }
+        };
+        tmem_ld16(lane_base + COL_Y, ya);
+#pragma unroll 1
+        for (int b2 = 0; b2 < 4; ++b2) {
+          tmem_wait_ld();
+          tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
+          k_block(ya, b2 * 4);
+          tmem_wait_ld();
+          if (b2 < 3) tmem_ld16(lane_base + COL_Y + b2 * 32 + 32, ya);
+          k_block(yb, b2 * 4 + 2);
         }
       }
       fence_proxy_async();
