@@ -12,10 +12,10 @@
 //               exponents x_t = b_t - b_mid (b the running sum of g) in fp32 (the middle reference keeps every factor
 //               2^x within 2^(+-32 max|g|)); v: bf16 -> fp16 in place (exact)
 //   MMA warp    MMA 1: Y = [u_q; u_k] W_h  (fp16 operands, fp32 accumulate in TMEM)
-//   row warps   phi: row softmax, one thread per token row, 32 columns at a time straight from tensor memory. Query rows
-//               keep exp(y - max) unnormalized: a positive per-token factor cancels in Eq. 8. The decay factors ride in
+//   row warps   (two threads per token row, 64 columns each, straight from tensor memory)
+//               phi: row softmax. Query rows keep exp(y - max) unnormalized: a positive per-token factor cancels in Eq. 8. The decay factors ride in
 //               the exponent of the softmax: qs = 2^(y' + x_t), ks = phi_k 2^(-x_i), kh = phi_k 2^(b_C - b_i) (<= phi_k)
-//   state warps 2^b_mid [S|z] as a 16-bit operand, accumulator [S|z] *= 2^b_C
+//   row warps   state pass: 2^b_mid [S|z] as a 16-bit operand, accumulator [S|z] *= 2^b_C
 //   MMA warp    MMA 2: P = qs ks^T ; O' = qs (2^b_mid [S|z]) ; [S|z] += kh^T [v|1]
 //   row warps   mask: P_ti = 0 for i > t, rounded to fp16
 //   MMA warp    MMA 3: O' += P [v|1]
@@ -41,9 +41,9 @@ constexpr int C = 64;        // tokens per chunk
 constexpr int MID = 31;      // reference token of the in-chunk decay factorization
 constexpr int HALO = 3;      // raw rows in front of a chunk that the conv needs (conv width up to 4)
 
-// warps: 0-7 prep, 8-11 row warps (TMEM quadrant = warp & 3), 12-15 state warps (same), 16 TMA, 17 MMA
+// warps: 0-7 prep, 8-15 row warps (TMEM quadrant = warp & 3, column half = (warp - 8) >> 2), 16 TMA, 17 MMA
 constexpr int PREP_THREADS = 256;
-constexpr int ROW_WARP0 = 8, STATE_WARP0 = 12, TMA_WARP = 16, MMA_WARP = 17;
+constexpr int ROW_WARP0 = 8, TMA_WARP = 16, MMA_WARP = 17;
 constexpr int THREADS = 18 * 32;
 
 // shared memory map (byte offsets from a 1024-byte aligned base)
@@ -52,7 +52,7 @@ constexpr uint32_t OFF_SBF = OFF_W + 32768;       // 2^b_mid * S, 16 bit, MN-maj
 constexpr uint32_t OFF_AU = OFF_SBF + 32768;      // raw q|k tile, then conv output in place: A of MMA 1, 2 slabs
 constexpr uint32_t OFF_QK = OFF_AU + 32768;       // qs (rows 0-63) | ks (rows 64-127), 16 bit, K-major, 2 slabs
 constexpr uint32_t OFF_X = OFF_QK + 32768;        // exponents x fp32 [64 x 128], XOR-swizzled 16-byte chunks
-constexpr uint32_t OFF_KH = OFF_X + 32768;        // kh^T fp16, K-major A of the state update, [128 channels x 64 tokens]
+constexpr uint32_t OFF_KH = OFF_X + 32768;        // kh fp16, MN-major A of the state update, 2 slabs x [64 tokens x 128 B]
 constexpr uint32_t OFF_G = OFF_KH + 16384;        // gate logits bf16, 2 slabs x [64 x 128 B]
 constexpr uint32_t OFF_V = OFF_G + 16384;         // v bf16, then fp16 in place, MN-major B, 2 slabs x [64 x 128 B]
 constexpr uint32_t OFF_PH = OFF_V + 16384;        // masked scores fp16, K-major, [64 x 128 B]; an M=128 MMA also reads
@@ -76,6 +76,7 @@ constexpr uint32_t COL_O = 256;    // [128 x 128] numerator (lanes 0-63 meaningf
 constexpr uint32_t COL_P = 384;    // [128 x 64] scores (lanes 0-63 meaningful)
 constexpr uint32_t COL_SZ = 448;   // [128 x 16] column 0: normalizer state z
 constexpr uint32_t COL_OZ = 464;   // [128 x 16] column 0: denominator
+constexpr uint32_t COL_MAIL = 480; // [128 x 2] per chunk parity: eps * (dropped query normalizer), row warps -> output pass
 constexpr uint32_t TMEM_COLS = 512;
 
 // mbarrier indices. "full": producer -> consumer, "free": consumer -> producer. Each completes once per chunk, so the
@@ -86,13 +87,13 @@ enum {
   B_V_FULL,        // TMA: v tile landed                             -> prep (v convert)
   B_G_FREE,        // prep: gate tile consumed                       -> TMA
   B_U_FULL,        // prep: conv output written                      -> MMA 1
-  B_X_FULL,        // prep: exponents, per-channel sums, range flags -> row warps, state warps
-  B_VH_FULL,       // prep: v converted                              -> MMA 2, state warps
+  B_X_FULL,        // prep: exponents, per-channel sums, range flags -> row warps
+  B_VH_FULL,       // prep: v converted                              -> MMA 2, row warps
   B_MMA1,          // MMA 1 complete: Y ready -> row warps; raw tile free -> TMA
   B_Y_FREE,        // row warps: Y consumed                          -> MMA 1 of the next chunk
   B_X_FREE,        // row warps: exponents consumed                  -> prep (gate of the next chunk)
   B_QK_FULL,       // row warps: qs, ks, kh written                  -> MMA 2
-  B_SBF_FULL,      // state warps: state operand written, S decayed  -> MMA 2
+  B_SBF_FULL,      // row warps: state operand written, S decayed    -> MMA 2
   B_MMA2,          // MMA 2 complete: P ready, state updated, qs/ks/kh/state operand free
   B_PH_FULL,       // row warps: masked scores written               -> MMA 3
   B_MMA3,          // MMA 3 complete: O' ready -> row warps; v tile free -> TMA
@@ -219,7 +220,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   // ---- one-time setup --------------------------------------------------------------------------------------------
   if (tid == 0) {
-    const int nphi = MODE == 0 ? 128 : 64;  // threads of the phi pass: all row threads, or the key rows only
+    const int nphi = MODE == 0 ? 256 : 128;  // threads of the phi pass: all row threads, or the key rows only
     mbar_init(bar(B_RAW_FULL), 1);
     mbar_init(bar(B_G_FULL), 1);
     mbar_init(bar(B_V_FULL), 1);
@@ -229,13 +230,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     mbar_init(bar(B_VH_FULL), PREP_THREADS);
     mbar_init(bar(B_MMA1), 1);
     mbar_init(bar(B_Y_FREE), nphi);
-    mbar_init(bar(B_X_FREE), nphi + 128);  // the phi threads and the state threads (which read bm, ft)
+    mbar_init(bar(B_X_FREE), 256);  // every row thread: it reads bm, ft and (phi threads) the exponents
     mbar_init(bar(B_QK_FULL), nphi);
-    mbar_init(bar(B_SBF_FULL), 128);
+    mbar_init(bar(B_SBF_FULL), 256);
     mbar_init(bar(B_MMA2), 1);
-    mbar_init(bar(B_PH_FULL), 64);
+    mbar_init(bar(B_PH_FULL), 128);
     mbar_init(bar(B_MMA3), 1);
-    mbar_init(bar(B_O_FREE), 64);
+    mbar_init(bar(B_O_FREE), 128);
     mbar_fence_init();
     s_flags[1] = 0;
     for (int i = 0; i < 7; ++i) s_rmax[i] = 0;
@@ -285,13 +286,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t tmem = (uint32_t)s_flags[0];
   const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
-  // initial state into tensor memory: state thread c owns row c of [S | z]
-  if (warp >= STATE_WARP0 && warp < STATE_WARP0 + 4) {
-    const int c = tid - STATE_WARP0 * 32;
+  // initial state into tensor memory: row thread (c, half) owns 64 columns of row c of [S | z]
+  if (warp >= ROW_WARP0 && warp < ROW_WARP0 + 8) {
+    const int tw = tid - ROW_WARP0 * 32, c = tw & 127, chh = tw >> 7;
     const bool have = a.S0 != nullptr && (a.seg_in || seg == 0);
     float s[32], mx = 0.f;
 #pragma unroll 1
-    for (int blk = 0; blk < 4; ++blk) {
+    for (int b2 = 0; b2 < 2; ++b2) {
+      const int blk = chh * 2 + b2;
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
         s[i] = have ? a.S0[(in_idx * D + c) * D + blk * 32 + i] : 0.f;
@@ -299,11 +301,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       tmem_st32(lane_base + COL_S + blk * 32, s);
     }
-    const bool havez = a.z0 != nullptr && (a.seg_in || seg == 0);
-    const float z0v = havez ? a.z0[in_idx * D + c] : 0.f;
-    tmem_st1(lane_base + COL_SZ, z0v);
+    if (chh == 1) {
+      const bool havez = a.z0 != nullptr && (a.seg_in || seg == 0);
+      const float z0v = havez ? a.z0[in_idx * D + c] : 0.f;
+      tmem_st1(lane_base + COL_SZ, z0v);
+      mx = fmaxf(mx, fabsf(z0v));
+    }
     tmem_wait_st();
-    mx = fmaxf(mx, fabsf(z0v));
     if (!(mx < 3.0e38f)) mx = 3.0e38f;  // NaN or inf in the given state: no fp16 operand
     atomicMax(s_sbound, __float_as_int(mx));
   }
@@ -362,15 +366,19 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint64_t dsc_ks = smem_desc(sb + OFF_QK + 8192, 16, 1024, LAYOUT_SW128);  // rows 64-127
       const uint64_t dsc_s = smem_desc(sb + OFF_SBF, 16384, 1024, LAYOUT_SW128);
       const uint64_t dsc_sz = smem_desc(sb + OFF_SZ, 128, 2048, LAYOUT_NONE);
-      const uint64_t dsc_kh = smem_desc(sb + OFF_KH, 16, 1024, LAYOUT_SW128);
+      const uint64_t dsc_kh = smem_desc(sb + OFF_KH, 8192, 1024, LAYOUT_SW128);
       const uint64_t dsc_v = smem_desc(sb + OFF_V, 8192, 1024, LAYOUT_SW128);
       const uint64_t dsc_one = smem_desc(sb + OFF_ONES, 128, 1024, LAYOUT_NONE);
       const uint64_t dsc_p = smem_desc(sb + OFF_PH, 16, 1024, LAYOUT_SW128);
-      auto kstep = [](int k) -> uint64_t { return (uint64_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2); };
+      // only the 14-bit start-address field (bits 0-13) moves, and it cannot carry: a 32-bit add on the low word
+      auto adv = [](uint64_t d, uint32_t off16) -> uint64_t {
+        return (d & 0xFFFFFFFF00000000ull) | (uint64_t)((uint32_t)d + off16);
+      };
+      auto kstep = [](int k) -> uint32_t { return (uint32_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2); };
       auto issue_mma1 = [&]() {
         constexpr uint32_t ID = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_K);
-#pragma unroll 1
-        for (int k = 0; k < 8; ++k) mma_f16(tmem + COL_Y, dsc_u + kstep(k), dsc_w + kstep(k), ID, k > 0);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) mma_f16(tmem + COL_Y, adv(dsc_u, kstep(k)), adv(dsc_w, kstep(k)), ID, k > 0);
         mma_commit(bar(B_MMA1));
       };
       bool ok = nchunks > 0;
@@ -392,22 +400,22 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const uint32_t ID_P = instr_desc(128, 64, fmt, MAJOR_K, MAJOR_K);
           const uint32_t ID_O = instr_desc(128, 128, fmt, MAJOR_K, MAJOR_MN);
           const uint32_t ID_OZ = instr_desc(128, 16, fmt, MAJOR_K, MAJOR_MN);
-#pragma unroll 1
+#pragma unroll
           for (int k = 0; k < 8; ++k) {
-            const uint64_t ad = dsc_qk + kstep(k);
-            mma_f16(tmem + COL_P, ad, dsc_ks + kstep(k), ID_P, k > 0);
-            mma_f16(tmem + COL_O, ad, dsc_s + (uint64_t)(k * (2048 >> 4)), ID_O, k > 0);
-            mma_f16(tmem + COL_OZ, ad, dsc_sz + (uint64_t)(k * (256 >> 4)), ID_OZ, k > 0);
+            const uint64_t ad = adv(dsc_qk, kstep(k));
+            mma_f16(tmem + COL_P, ad, adv(dsc_ks, kstep(k)), ID_P, k > 0);
+            mma_f16(tmem + COL_O, ad, adv(dsc_s, k * (2048 >> 4)), ID_O, k > 0);
+            mma_f16(tmem + COL_OZ, ad, adv(dsc_sz, k * (256 >> 4)), ID_OZ, k > 0);
           }
         }
         {
-          constexpr uint32_t ID_S = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
-          constexpr uint32_t ID_SZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
-#pragma unroll 1
+          constexpr uint32_t ID_S = instr_desc(128, 128, FMT_F16, MAJOR_MN, MAJOR_MN);
+          constexpr uint32_t ID_SZ = instr_desc(128, 16, FMT_F16, MAJOR_MN, MAJOR_MN);
+#pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const uint64_t ad = dsc_kh + (uint64_t)(k * 2);
-            mma_f16(tmem + COL_S, ad, dsc_v + (uint64_t)(k * (2048 >> 4)), ID_S, 1);
-            mma_f16(tmem + COL_SZ, ad, dsc_one + (uint64_t)(k * (256 >> 4)), ID_SZ, 1);
+            const uint64_t ad = adv(dsc_kh, k * (2048 >> 4));
+            mma_f16(tmem + COL_S, ad, adv(dsc_v, k * (2048 >> 4)), ID_S, 1);
+            mma_f16(tmem + COL_SZ, ad, adv(dsc_one, k * (256 >> 4)), ID_SZ, 1);
           }
           mma_commit(bar(B_MMA2));
         }
@@ -422,11 +430,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tc_fence_after_sync();
           constexpr uint32_t ID_O = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
           constexpr uint32_t ID_OZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
-#pragma unroll 1
+#pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const uint64_t ad = dsc_p + (uint64_t)(k * 2);
-            mma_f16(tmem + COL_O, ad, dsc_v + (uint64_t)(k * (2048 >> 4)), ID_O, 1);
-            mma_f16(tmem + COL_OZ, ad, dsc_one + (uint64_t)(k * (256 >> 4)), ID_OZ, 1);
+            const uint64_t ad = adv(dsc_p, k * 2);
+            mma_f16(tmem + COL_O, ad, adv(dsc_v, k * (2048 >> 4)), ID_O, 1);
+            mma_f16(tmem + COL_OZ, ad, adv(dsc_one, k * (256 >> 4)), ID_OZ, 1);
           }
           mma_commit(bar(B_MMA3));
         }
@@ -450,6 +458,37 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t au = sb + OFF_AU + (cv_oct >> 3) * 16384;  // this thread's 64-channel slab
     const int cjc = cv_oct & 7, crow0 = cv_stream * 64 + cv_rg * 8;
     const int gc = tid & 127, ghalf = tid >> 7, gjc = (gc & 63) >> 3;
+    // Output pass (threads of TMEM quadrants 0 and 1: 64 query rows x 2 column halves): o = O' / (denominator + eps),
+    // Eq. 8, straight from tensor memory to global memory.
+    auto out_pass = [&](int m) {
+      if ((warp & 3) >= 2) return;
+      const int orow_i = (warp & 3) * 32 + lane, och = tid >> 7;
+      const int ot0 = t_begin + m * C;
+      const int onvalid = min(C, t_end - ot0);
+      tc_fence_after_sync();
+      float den = tmem_ld1(lane_base + COL_OZ);
+      // the query features went in scaled by their dropped softmax normalizer, so eps arrives scaled the same way
+      if (a.eps != 0.f) den += tmem_ld1(lane_base + COL_MAIL + (m & 1));
+      tmem_wait_ld();
+      const float inv = 1.f / den;
+      bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * D + och * 64;
+      float y[32];
+#pragma unroll 1
+      for (int b2 = 0; b2 < 2; ++b2) {
+        tmem_ld32(lane_base + COL_O + och * 64 + b2 * 32, y);
+        tmem_wait_ld();
+        if (b2 == 1) {  // O' is in registers: the next chunk's products may overwrite it
+          tc_fence_before_sync();
+          mbar_arrive(bar(B_O_FREE));
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) y[i] *= inv;
+        if (orow_i < onvalid) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) *reinterpret_cast<uint4*>(orow + b2 * 32 + q4 * 8) = pack8(y + 8 * q4, false);
+        }
+      }
+    };
     bool fail = false;
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
@@ -551,6 +590,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       mbar_arrive(bar(B_X_FULL));
 
+      // ---- output of the previous chunk (its last product completes about now; the v tile is loaded after it) -----------
+      if (MODE == 0 && n > 0) {
+        WAITF(B_MMA3, pp);
+        if (!fail) out_pass(n - 1);
+      }
+
       // ---- v: bf16 -> fp16 in place (exact for |v| in the fp16 normal range) ------------------------------------------
       WAITF(B_V_FULL, p);
       if (!fail) {
@@ -570,248 +615,271 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       fence_proxy_async();
       mbar_arrive(bar(B_VH_FULL));
     }
-  } else if (warp < STATE_WARP0) {
+    if (MODE == 0 && nchunks > 0 && !fail && !*s_abort &&
+        wait_or_abort(bar(B_MMA3), (uint32_t)((nchunks - 1) & 1), s_abort))
+      out_pass(nchunks - 1);
+  } else {
     // ================================================================================================ row warps
-    // thread = one row of Y: rows 0-63 the query tokens (these threads also mask the scores and write the output),
-    // rows 64-127 the key tokens
-    const int rt = tid - ROW_WARP0 * 32;
-    const bool is_q = rt < C;
-    const int row = is_q ? rt : rt - C;
+    // 8 warps, two per TMEM quadrant. Thread = (row, half of the columns): rows 0-63 are the query tokens, rows 64-127 the
+    // key tokens of Y; the same threads own row c of [S | z] (state pass), and the query-row threads also mask the
+    // scores and write the output. The two threads of a row meet through shared memory (row max, softmax sum).
+    const int tw = tid - ROW_WARP0 * 32;
+    const int ch = tw >> 7;                       // column half: columns [64 ch, 64 ch + 64)
+    const int r128 = (tw & 127);                  // row of Y and of the state (= TMEM lane)
+    const bool is_q = r128 < C;
+    const int row = is_q ? r128 : r128 - C;       // token inside the chunk
+    const bool phi_on = MODE == 0 || !is_q;       // the state-only pass has no query rows
+    const int phi_bar = is_q ? 3 : 4;             // the query rows and the key rows meet among themselves (128 threads each)
     const float L2E = 1.4426950408889634f;
     const bool need_qsum = a.eps != 0.f;  // the dropped softmax normalizer of the query rows only matters next to eps
-    for (int n = 0; n < nchunks && (MODE == 0 || !is_q); ++n) {
-      const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
-      const int t0 = t_begin + n * C;
-      const int nvalid = min(C, t_end - t0);
-      WAIT(B_X_FULL, p);
-      WAIT(B_MMA1, p);
-      if (n > 0) WAIT(B_MMA2, pp);  // qs / ks / kh of the previous chunk have been consumed
-      tc_fence_after_sync();
-      const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
-      // Y is read 16 columns at a time with the next load in flight while a block is processed
-      float ya[16], yb[16];
-      float y[32];
-      float m = -INFINITY, qsum = 0.f;
-      tmem_ld16(lane_base + COL_Y, ya);
-#pragma unroll 1
-      for (int b2 = 0; b2 < 4; ++b2) {
-        tmem_wait_ld();
-        tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) m = fmaxf(m, ya[i]);
-        tmem_wait_ld();
-        tmem_ld16(lane_base + COL_Y + ((b2 * 32 + 32) & 127), ya);  // wraps to column 0: the first block of the next sweep
-#pragma unroll
-        for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
-      }
-      const float mb = m * L2E;
-      if (is_q) {
-        auto q_block = [&](const float* yy, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
-#pragma unroll
-          for (int h2 = 0; h2 < 2; ++h2) {
-            const int jj = jj0 + h2;
-            float x[8], v[8];
-            load_x8(sb + OFF_X, row, jj, x);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = ex2f(fmaf(yy[h2 * 8 + i], L2E, x[i] - mb));
-            if (need_qsum) {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) qsum += ex2f(fmaf(yy[h2 * 8 + i], L2E, -mb));
-            }
-            sts128(sb + OFF_QK + (jj >> 3) * 16384 + sw128(row, jj & 7), pack8(v, f16));
-          }
-        };
-#pragma unroll 1
-        for (int b2 = 0; b2 < 4; ++b2) {
-          tmem_wait_ld();
-          tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
-          q_block(ya, b2 * 4);
-          tmem_wait_ld();
-          if (b2 < 3) tmem_ld16(lane_base + COL_Y + b2 * 32 + 32, ya);
-          q_block(yb, b2 * 4 + 2);
-        }
-      } else {
-        // key rows: one sweep forms e = exp(y - max) and its sum and parks e in Y's own columns; the last sweep
-        // writes ks = e 2^-x / sum and kh = ks 2^(b_C - b_mid)
-        float sum = 0.f;
-#pragma unroll 1
-        for (int b2 = 0; b2 < 4; ++b2) {
-          tmem_wait_ld();
-          tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            ya[i] = ex2f(fmaf(ya[i], L2E, -mb));
-            sum += ya[i];
-          }
-          tmem_st16(lane_base + COL_Y + b2 * 32, ya);
-          tmem_wait_ld();
-          if (b2 < 3) tmem_ld16(lane_base + COL_Y + b2 * 32 + 32, ya);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            yb[i] = ex2f(fmaf(yb[i], L2E, -mb));
-            sum += yb[i];
-          }
-          tmem_st16(lane_base + COL_Y + b2 * 32 + 16, yb);
-        }
-        tmem_wait_st();
-        const float inv = row < nvalid ? 1.f / sum : 0.f;  // tokens past the end contribute nothing
-        const float* e63v = vec(p, 2);
-        auto k_block = [&](const float* ee, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
-#pragma unroll
-          for (int h2 = 0; h2 < 2; ++h2) {
-            const int jj = jj0 + h2;  // channels [8 jj, 8 jj + 8)
-            float x[8], ks[8];
-            load_x8(sb + OFF_X, row, jj, x);
-            const float4 ea = *reinterpret_cast<const float4*>(e63v + jj * 8);
-            const float4 eb = *reinterpret_cast<const float4*>(e63v + jj * 8 + 4);
-            const float e63[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ks[i] = ee[h2 * 8 + i] * inv * ex2f(-x[i]);
-            if (MODE == 0) sts128(sb + OFF_QK + (jj >> 3) * 16384 + sw128(C + row, jj & 7), pack8(ks, f16));
-            // kh^T: row = key channel, 64 tokens (128 bytes) per row, so that the state update reads a K-major A operand
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-              *reinterpret_cast<__half*>(sg + OFF_KH + (jj * 8 + i) * 128 + (((row >> 3) ^ i) << 4) + (row & 7) * 2) =
-                  __float2half_rn(ks[i] * e63[i]);
-          }
-        };
-        tmem_ld16(lane_base + COL_Y, ya);
-#pragma unroll 1
-        for (int b2 = 0; b2 < 4; ++b2) {
-          tmem_wait_ld();
-          tmem_ld16(lane_base + COL_Y + b2 * 32 + 16, yb);
-          k_block(ya, b2 * 4);
-          tmem_wait_ld();
-          if (b2 < 3) tmem_ld16(lane_base + COL_Y + b2 * 32 + 32, ya);
-          k_block(yb, b2 * 4 + 2);
-        }
-      }
-      fence_proxy_async();
-      tc_fence_before_sync();
-      mbar_arrive(bar(B_Y_FREE));
-      mbar_arrive(bar(B_X_FREE));
-      mbar_arrive(bar(B_QK_FULL));
-      if (MODE == 0 && is_q) {
-        // ---- causal mask, fp16 scores -------------------------------------------------------------------------------
-        WAIT(B_MMA2, p);
-        tc_fence_after_sync();
-#pragma unroll 1
-        for (int blk = 0; blk < 2; ++blk) {
-          tmem_ld32(lane_base + COL_P + blk * 32, y);
-          tmem_wait_ld();
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = (blk * 32 + q4 * 8 + i <= row) ? y[q4 * 8 + i] : 0.f;
-            sts128(sb + OFF_PH + sw128(row, blk * 4 + q4), pack8(v, true));
-          }
-        }
-        fence_proxy_async();
-        tc_fence_before_sync();
-        mbar_arrive(bar(B_PH_FULL));
-        // ---- normalize (Eq. 8) and store ------------------------------------------------------------------------------
-        WAIT(B_MMA3, p);
-        tc_fence_after_sync();
-        const float den = tmem_ld1(lane_base + COL_OZ);
-        tmem_wait_ld();
-        // the query features went in scaled by qsum (unnormalized softmax), so eps scales the same way
-        const float inv = 1.f / (den + a.eps * qsum);
-        bf16* orow = a.o + (((size_t)b * a.T + t0 + row) * a.H + h) * D;
-#pragma unroll 1
-        for (int blk = 0; blk < 4; ++blk) {
-          tmem_ld32(lane_base + COL_O + blk * 32, y);
-          tmem_wait_ld();
-          if (blk == 3) {  // O' is in registers: the next chunk's products may overwrite it
-            tc_fence_before_sync();
-            mbar_arrive(bar(B_O_FREE));
-          }
-#pragma unroll
-          for (int i = 0; i < 32; ++i) y[i] *= inv;
-          if (row < nvalid) {
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) *reinterpret_cast<uint4*>(orow + blk * 32 + q4 * 8) = pack8(y + 8 * q4, false);
-          }
-        }
-      }
-    }
-  } else {
-    // ================================================================================================ state warps
-    // thread c = row c of [S | z]: per chunk the 16-bit operand 2^b_mid [S|z] and the decay [S|z] *= 2^b_C
-    const int c = tid - STATE_WARP0 * 32;
-    float dsum = 0.f;  // log2 of this channel's total decay over the segment
+    // row max / softmax sum of the two column halves. Key rows: the first 1 KB of the kh tile, which nobody uses before
+    // the key rows' last sweep (the previous chunk's update has completed, this chunk's kh is not written yet). Query
+    // rows: the first 1 KB of the score tile (the previous chunk's MMA 3 has completed, the mask pass comes later).
+    float* const s_pmax = reinterpret_cast<float*>(sg + (is_q ? OFF_PH : OFF_KH));  // [2][64]
+    float* const s_psum = s_pmax + 128;                                             // [2][64]
+    float dsum = 0.f;  // log2 of this state row's total decay over the segment
     bool fail = false;
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
+      const int t0 = t_begin + n * C;
+      const int nvalid = min(C, t_end - t0);
       WAITF(B_X_FULL, p);
-      if (n > 0) WAITF(B_MMA2, pp);  // the previous chunk's update has landed; its state operand has been consumed
+      if (n > 0) WAITF(B_MMA2, pp);  // the previous chunk's update has landed; qs / ks / kh / state operand are free
+      tc_fence_after_sync();
+      const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
+      float y[32];
+      // ---- state pass: 16-bit operand 2^b_mid [S|z], accumulator [S|z] *= 2^b_C (this thread: 64 columns of row r128)
       if (!fail) {
-        tc_fence_after_sync();
+        const int c = r128;
         const float bm = vec(p, 0)[c], ft = vec(p, 1)[c];
-        mbar_arrive(bar(B_X_FREE));
         const float dm = ex2f(bm), dC = ex2f(bm + ft);
-        dsum += bm + ft;
-        const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
-        float s[32], mx = 0.f;
+        if (ch == 0) dsum += bm + ft;
+        float mx = 0.f;
 #pragma unroll 1
-        for (int blk = 0; blk < 4; ++blk) {
-          tmem_ld32(lane_base + COL_S + blk * 32, s);
+        for (int b2 = 0; b2 < 2; ++b2) {
+          const int blk = ch * 2 + b2;
+          tmem_ld32(lane_base + COL_S + blk * 32, y);
           tmem_wait_ld();
           if (MODE == 0) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(s[i]));
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(y[i]));
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
               float w[8];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) w[i] = dm * s[8 * q4 + i];
-              sts128(sb + OFF_SBF + (blk >> 1) * 16384 + sw128(c, (blk & 1) * 4 + q4), pack8(w, f16));
+              for (int i = 0; i < 8; ++i) w[i] = dm * y[8 * q4 + i];
+              sts128(sb + OFF_SBF + ch * 16384 + sw128(c, b2 * 4 + q4), pack8(w, f16));
             }
           }
 #pragma unroll
-          for (int i = 0; i < 32; ++i) s[i] *= dC;
-          tmem_st32(lane_base + COL_S + blk * 32, s);
+          for (int i = 0; i < 32; ++i) y[i] *= dC;
+          tmem_st32(lane_base + COL_S + blk * 32, y);
         }
-        const float z = tmem_ld1(lane_base + COL_SZ);
-        tmem_wait_ld();
+        if (ch == 1) {
+          const float z = tmem_ld1(lane_base + COL_SZ);
+          tmem_wait_ld();
+          if (MODE == 0) {
+            *reinterpret_cast<uint16_t*>(sg + OFF_SZ + (c >> 3) * 128 + (c & 7) * 16) = to16(dm * z, f16);
+            mx = fmaxf(mx, fabsf(z));
+          }
+          tmem_st1(lane_base + COL_SZ, dC * z);
+        }
         if (MODE == 0) {
-          *reinterpret_cast<uint16_t*>(sg + OFF_SZ + (c >> 3) * 128 + (c & 7) * 16) = to16(dm * z, f16);
-          mx = warp_max(fmaxf(mx, fabsf(z)));
+          mx = warp_max(mx);
           if (lane == 0) atomicMax(s_smax, __float_as_int(mx < 3.0e38f ? mx : 3.0e38f));
         }
-        tmem_st1(lane_base + COL_SZ, dC * z);
         tmem_wait_st();
+        if (!phi_on) mbar_arrive(bar(B_X_FREE));  // (state-only pass) this thread has read bm, ft and reads no exponents
       }
+      // ---- phi ------------------------------------------------------------------------------------------------------
+      float qsum = 0.f;
+      if (phi_on) {
+        WAITF(B_MMA1, p);
+        // the score tile (scratch of the query rows below, then this chunk's masked scores) was the previous chunk's
+        // MMA 3 operand
+        if (MODE == 0 && is_q && n > 0) WAITF(B_MMA3, pp);
+        tc_fence_after_sync();
+        const uint32_t ycol = lane_base + COL_Y + ch * 64;
+        float ya[16], yb[16];  // 16 columns at a time, the next load in flight while a block is processed
+        float m = -INFINITY;
+        if (!fail) {
+          tmem_ld16(ycol, ya);
+#pragma unroll 1
+          for (int b2 = 0; b2 < 2; ++b2) {
+            tmem_wait_ld();
+            tmem_ld16(ycol + b2 * 32 + 16, yb);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) m = fmaxf(m, ya[i]);
+            tmem_wait_ld();
+            tmem_ld16(ycol + ((b2 * 32 + 32) & 63), ya);  // wraps to the first block: the next sweep starts there
+#pragma unroll
+            for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
+          }
+          s_pmax[ch * 64 + row] = m;
+        }
+        named_bar_sync(phi_bar, 128);
+        m = fmaxf(s_pmax[row], s_pmax[64 + row]);
+        const float mb = m * L2E;
+        if (is_q) {
+          if (!fail) {
+            auto q_block = [&](const float* yy, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
+#pragma unroll
+              for (int h2 = 0; h2 < 2; ++h2) {
+                const int jj = jj0 + h2;
+                float x[8], v[8];
+                load_x8(sb + OFF_X, row, jj, x);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = ex2f(fmaf(yy[h2 * 8 + i], L2E, x[i] - mb));
+                if (need_qsum) {
+#pragma unroll
+                  for (int i = 0; i < 8; ++i) qsum += ex2f(fmaf(yy[h2 * 8 + i], L2E, -mb));
+                }
+                sts128(sb + OFF_QK + ch * 16384 + sw128(row, jj & 7), pack8(v, f16));
+              }
+            };
+#pragma unroll 1
+            for (int b2 = 0; b2 < 2; ++b2) {
+              tmem_wait_ld();
+              tmem_ld16(ycol + b2 * 32 + 16, yb);
+              q_block(ya, ch * 8 + b2 * 4);
+              tmem_wait_ld();
+              if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
+              q_block(yb, ch * 8 + b2 * 4 + 2);
+            }
+            if (need_qsum) s_psum[ch * 64 + row] = qsum;
+          }
+          if (need_qsum) {
+            named_bar_sync(phi_bar, 128);
+            qsum = s_psum[row] + s_psum[64 + row];
+            if (ch == 0 && !fail) {  // eps times the dropped normalizer travels to the output pass through tensor memory
+              tmem_st1(lane_base + COL_MAIL + p, a.eps * qsum);
+              tmem_wait_st();
+            }
+          }
+        } else {
+          // key rows: one sweep forms e = exp(y - max) and its sum and parks e in Y's own columns; the last sweep
+          // writes ks = e 2^-x / sum and kh = ks 2^(b_C - b_mid)
+          float sum = 0.f;
+          if (!fail) {
+#pragma unroll 1
+            for (int b2 = 0; b2 < 2; ++b2) {
+              tmem_wait_ld();
+              tmem_ld16(ycol + b2 * 32 + 16, yb);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                ya[i] = ex2f(fmaf(ya[i], L2E, -mb));
+                sum += ya[i];
+              }
+              tmem_st16(ycol + b2 * 32, ya);
+              tmem_wait_ld();
+              if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                yb[i] = ex2f(fmaf(yb[i], L2E, -mb));
+                sum += yb[i];
+              }
+              tmem_st16(ycol + b2 * 32 + 16, yb);
+            }
+            tmem_wait_st();
+            s_psum[ch * 64 + row] = sum;
+          }
+          named_bar_sync(phi_bar, 128);
+          sum = s_psum[row] + s_psum[64 + row];
+          // every key-row thread has the maxima and sums it needs: from here on the kh tile may be written
+          named_bar_sync(phi_bar, 128);
+          if (!fail) {
+            const float inv = row < nvalid ? 1.f / sum : 0.f;  // tokens past the end contribute nothing
+            const float* e63v = vec(p, 2);
+            auto k_block = [&](const float* ee, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
+#pragma unroll
+              for (int h2 = 0; h2 < 2; ++h2) {
+                const int jj = jj0 + h2;  // channels [8 jj, 8 jj + 8)
+                float x[8], ks[8];
+                load_x8(sb + OFF_X, row, jj, x);
+                const float4 ea = *reinterpret_cast<const float4*>(e63v + jj * 8);
+                const float4 eb = *reinterpret_cast<const float4*>(e63v + jj * 8 + 4);
+                const float e63[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
+#pragma unroll
+                for (int i = 0; i < 8; ++i) ks[i] = ee[h2 * 8 + i] * inv * ex2f(-x[i]);
+                if (MODE == 0) sts128(sb + OFF_QK + ch * 16384 + sw128(C + row, jj & 7), pack8(ks, f16));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) ks[i] *= e63[i];
+                // kh: row = token, MN-major A operand of the state update (slab = column half)
+                sts128(sb + OFF_KH + ch * 8192 + sw128(row, jj & 7), pack8(ks, true));
+              }
+            };
+            tmem_ld16(ycol, ya);
+#pragma unroll 1
+            for (int b2 = 0; b2 < 2; ++b2) {
+              tmem_wait_ld();
+              tmem_ld16(ycol + b2 * 32 + 16, yb);
+              k_block(ya, ch * 8 + b2 * 4);
+              tmem_wait_ld();
+              if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
+              k_block(yb, ch * 8 + b2 * 4 + 2);
+            }
+          }
+        }
+      }
+      // ---- hand-over to MMA 2: state operand, qs / ks / kh, and the bound on the state for the next chunk ------------
       WAITF(B_VH_FULL, p);  // the chunk's max|v| is known
       fence_proxy_async();
       tc_fence_before_sync();
-      fail = named_bar_or(2, 128, fail);
+      fail = named_bar_or(2, 256, fail);
       if (fail) break;
-      if (MODE == 0 && c == 0) {
-        // bound on the state after this chunk's update: the next chunk's choice of operand type
+      if (MODE == 0 && tw == 0) {
+        // |S_new| <= |S_old| + 64 max|v|: the next chunk's choice of operand type
         s_sbound[pp] = __float_as_int(__int_as_float(*s_smax) + 64.f * fmaxf(__int_as_float(s_vmax[p]), 1.f));
         *s_smax = 0;
         __threadfence_block();
       }
       mbar_arrive(bar(B_SBF_FULL));
+      if (phi_on) {
+        mbar_arrive(bar(B_Y_FREE));
+        mbar_arrive(bar(B_X_FREE));
+        mbar_arrive(bar(B_QK_FULL));
+      }
+      if (MODE == 0 && is_q) {
+        // ---- causal mask, fp16 scores: this thread's 32 columns of row `row` -------------------------------------------
+        WAITF(B_MMA2, p);
+        if (!fail) {
+          tc_fence_after_sync();
+          tmem_ld32(lane_base + COL_P + ch * 32, y);
+          tmem_wait_ld();
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = (ch * 32 + q4 * 8 + i <= row) ? y[q4 * 8 + i] : 0.f;
+            sts128(sb + OFF_PH + sw128(row, ch * 4 + q4), pack8(v, true));
+          }
+          fence_proxy_async();
+          tc_fence_before_sync();
+          mbar_arrive(bar(B_PH_FULL));
+        }
+      }
     }
     // ---- final state -------------------------------------------------------------------------------------------------
     if (!fail && !*s_abort && (nchunks == 0 || wait_or_abort(bar(B_MMA2), (uint32_t)((nchunks - 1) & 1), s_abort))) {
       tc_fence_after_sync();
-      if (a.dtot != nullptr) a.dtot[seg_idx * D + c] = dsum;
+      const int c = r128;
+      if (a.dtot != nullptr && ch == 0) a.dtot[seg_idx * D + c] = dsum;
       if (a.S_T != nullptr && (a.seg_out || seg == a.nseg - 1)) {
         float s[32];
 #pragma unroll 1
-        for (int blk = 0; blk < 4; ++blk) {
+        for (int b2 = 0; b2 < 2; ++b2) {
+          const int blk = ch * 2 + b2;
           tmem_ld32(lane_base + COL_S + blk * 32, s);
           tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 32; i += 4)
             *reinterpret_cast<float4*>(a.S_T + (out_idx * D + c) * D + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
         }
-        const float z = tmem_ld1(lane_base + COL_SZ);
-        tmem_wait_ld();
-        if (a.z_T) a.z_T[out_idx * D + c] = z;
+        if (ch == 1 && a.z_T) {
+          const float z = tmem_ld1(lane_base + COL_SZ);
+          tmem_wait_ld();
+          a.z_T[out_idx * D + c] = z;
+        }
       }
     }
   }
