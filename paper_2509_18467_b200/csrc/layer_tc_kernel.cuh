@@ -76,7 +76,9 @@ constexpr uint32_t COL_O = 256;    // [128 x 128] numerator (lanes 0-63 meaningf
 constexpr uint32_t COL_P = 384;    // [128 x 64] scores (lanes 0-63 meaningful)
 constexpr uint32_t COL_SZ = 448;   // [128 x 16] column 0: normalizer state z
 constexpr uint32_t COL_OZ = 464;   // [128 x 16] column 0: denominator
-constexpr uint32_t COL_MAIL = 480; // [128 x 2] per chunk parity: eps * (dropped query normalizer), row warps -> output pass
+constexpr uint32_t COL_MAIL = 480; // spare columns used as per-row mailboxes between threads of one TMEM lane:
+                                   // +2, +3: row max / softmax sum of the two column halves; +4 p + half (p = chunk
+                                   // parity): eps * (dropped query normalizer) of that half, row warps -> output pass
 constexpr uint32_t TMEM_COLS = 512;
 
 // mbarrier indices. "full": producer -> consumer, "free": consumer -> producer. Each completes once per chunk, so the
@@ -389,6 +391,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       for (int n = 0; ok && n < nchunks; ++n) {
         const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
+        if (n + 1 < nchunks) {
+          // the mix of the next chunk goes first: its phi pass starts reading Y while this chunk's MMA 2 executes
+          WAIT(B_U_FULL, pp);
+          WAIT(B_Y_FREE, p);
+          tc_fence_after_sync();
+          issue_mma1();
+        }
         WAIT(B_QK_FULL, p);
         WAIT(B_SBF_FULL, p);
         WAIT(B_VH_FULL, p);
@@ -418,12 +427,6 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             mma_f16(tmem + COL_SZ, ad, adv(dsc_one, k * (256 >> 4)), ID_SZ, 1);
           }
           mma_commit(bar(B_MMA2));
-        }
-        if (n + 1 < nchunks) {  // the mix of the next chunk, ahead of this chunk's last product
-          WAIT(B_U_FULL, pp);
-          WAIT(B_Y_FREE, p);
-          tc_fence_after_sync();
-          issue_mma1();
         }
         if (MODE == 0) {
           WAIT(B_PH_FULL, p);
@@ -468,7 +471,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_after_sync();
       float den = tmem_ld1(lane_base + COL_OZ);
       // the query features went in scaled by their dropped softmax normalizer, so eps arrives scaled the same way
-      if (a.eps != 0.f) den += tmem_ld1(lane_base + COL_MAIL + (m & 1));
+      if (a.eps != 0.f) den += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1)) + tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
       tmem_wait_ld();
       const float inv = 1.f / den;
       bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * D + och * 64;
@@ -622,7 +625,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ================================================================================================ row warps
     // 8 warps, two per TMEM quadrant. Thread = (row, half of the columns): rows 0-63 are the query tokens, rows 64-127 the
     // key tokens of Y; the same threads own row c of [S | z] (state pass), and the query-row threads also mask the
-    // scores and write the output. The two threads of a row meet through shared memory (row max, softmax sum).
+    // scores. The two threads of a row share a TMEM lane and meet through two spare TMEM columns (row max, softmax sum).
+    // Order inside a chunk: the sweeps of phi that only READ (row max; key rows: exp and its sum) run while the previous
+    // chunk's MMA 2 is still executing; the state pass and the sweep that writes qs / ks / kh wait for it.
     const int tw = tid - ROW_WARP0 * 32;
     const int ch = tw >> 7;                       // column half: columns [64 ch, 64 ch + 64)
     const int r128 = (tw & 127);                  // row of Y and of the state (= TMEM lane)
@@ -632,22 +637,82 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int phi_bar = is_q ? 3 : 4;             // the query rows and the key rows meet among themselves (128 threads each)
     const float L2E = 1.4426950408889634f;
     const bool need_qsum = a.eps != 0.f;  // the dropped softmax normalizer of the query rows only matters next to eps
-    // row max / softmax sum of the two column halves. Key rows: the first 1 KB of the kh tile, which nobody uses before
-    // the key rows' last sweep (the previous chunk's update has completed, this chunk's kh is not written yet). Query
-    // rows: the first 1 KB of the score tile (the previous chunk's MMA 3 has completed, the mask pass comes later).
-    float* const s_pmax = reinterpret_cast<float*>(sg + (is_q ? OFF_PH : OFF_KH));  // [2][64]
-    float* const s_psum = s_pmax + 128;                                             // [2][64]
+    const uint32_t mail_mine = lane_base + COL_MAIL + 2 + ch, mail_other = lane_base + COL_MAIL + 2 + (ch ^ 1);
+    const uint32_t ycol = lane_base + COL_Y + ch * 64;
     float dsum = 0.f;  // log2 of this state row's total decay over the segment
     bool fail = false;
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
-      const int t0 = t_begin + n * C;
-      const int nvalid = min(C, t_end - t0);
+      const int nvalid = min(C, t_end - (t_begin + n * C));
+      float y[32], ya[16], yb[16];
+      float mb = 0.f, sum = 0.f;
+      // ---- phi, reading sweeps ----------------------------------------------------------------------------------------
+      if (phi_on) {
+        WAITF(B_MMA1, p);
+        tc_fence_after_sync();
+        float m = -INFINITY;
+        if (!fail) {
+          tmem_ld16(ycol, ya);  // 16 columns at a time, the next load in flight while a block is processed
+#pragma unroll 1
+          for (int b2 = 0; b2 < 2; ++b2) {
+            tmem_wait_ld();
+            tmem_ld16(ycol + b2 * 32 + 16, yb);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) m = fmaxf(m, ya[i]);
+            tmem_wait_ld();
+            tmem_ld16(ycol + ((b2 * 32 + 32) & 63), ya);  // wraps to the first block: the next sweep starts there
+#pragma unroll
+            for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
+          }
+          tmem_st1(mail_mine, m);
+          tmem_wait_st();
+        }
+        named_bar_sync(phi_bar, 128);
+        if (!fail) {
+          m = fmaxf(m, tmem_ld1(mail_other));  // (the load of `ya` issued above completes with this wait as well)
+          tmem_wait_ld();
+        }
+        mb = m * L2E;
+        if (!is_q) {
+          // key rows: e = exp(y - max) and its sum; e is parked in Y's own columns for the writing sweep
+          if (!fail) {
+#pragma unroll 1
+            for (int b2 = 0; b2 < 2; ++b2) {
+              tmem_wait_ld();
+              tmem_ld16(ycol + b2 * 32 + 16, yb);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                ya[i] = ex2f(fmaf(ya[i], L2E, -mb));
+                sum += ya[i];
+              }
+              tmem_st16(ycol + b2 * 32, ya);
+              tmem_wait_ld();
+              if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                yb[i] = ex2f(fmaf(yb[i], L2E, -mb));
+                sum += yb[i];
+              }
+              tmem_st16(ycol + b2 * 32 + 16, yb);
+            }
+            named_bar_sync(phi_bar, 128);  // the partner has read the row max out of the mailbox
+            tmem_st1(mail_mine, sum);
+            tmem_wait_st();
+          } else {
+            named_bar_sync(phi_bar, 128);
+          }
+          named_bar_sync(phi_bar, 128);
+          if (!fail) {
+            sum += tmem_ld1(mail_other);
+            tmem_wait_ld();
+          }
+        }
+      }
+      // ---- the previous chunk's MMA 2 has completed: the state is updated; qs / ks / kh / state operand are free ---------
       WAITF(B_X_FULL, p);
-      if (n > 0) WAITF(B_MMA2, pp);  // the previous chunk's update has landed; qs / ks / kh / state operand are free
+      if (n > 0) WAITF(B_MMA2, pp);
       tc_fence_after_sync();
       const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
-      float y[32];
       // ---- state pass: 16-bit operand 2^b_mid [S|z], accumulator [S|z] *= 2^b_C (this thread: 64 columns of row r128)
       if (!fail) {
         const int c = r128;
@@ -691,133 +756,70 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tmem_wait_st();
         if (!phi_on) mbar_arrive(bar(B_X_FREE));  // (state-only pass) this thread has read bm, ft and reads no exponents
       }
-      // ---- phi ------------------------------------------------------------------------------------------------------
-      float qsum = 0.f;
-      if (phi_on) {
-        WAITF(B_MMA1, p);
-        // the score tile (scratch of the query rows below, then this chunk's masked scores) was the previous chunk's
-        // MMA 3 operand
-        if (MODE == 0 && is_q && n > 0) WAITF(B_MMA3, pp);
-        tc_fence_after_sync();
-        const uint32_t ycol = lane_base + COL_Y + ch * 64;
-        float ya[16], yb[16];  // 16 columns at a time, the next load in flight while a block is processed
-        float m = -INFINITY;
-        if (!fail) {
+      // ---- phi, writing sweep -------------------------------------------------------------------------------------------
+      if (phi_on && !fail) {
+        if (is_q) {
+          float qsum = 0.f;
+          auto q_block = [&](const float* yy, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              const int jj = jj0 + h2;
+              float x[8], v[8];
+              load_x8(sb + OFF_X, row, jj, x);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) v[i] = ex2f(fmaf(yy[h2 * 8 + i], L2E, x[i] - mb));
+              if (need_qsum) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) qsum += ex2f(fmaf(yy[h2 * 8 + i], L2E, -mb));
+              }
+              sts128(sb + OFF_QK + ch * 16384 + sw128(row, jj & 7), pack8(v, f16));
+            }
+          };
+          // (`ya` holds the first 16 columns since the row-max sweep)
+#pragma unroll 1
+          for (int b2 = 0; b2 < 2; ++b2) {
+            tmem_wait_ld();
+            tmem_ld16(ycol + b2 * 32 + 16, yb);
+            q_block(ya, ch * 8 + b2 * 4);
+            tmem_wait_ld();
+            if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
+            q_block(yb, ch * 8 + b2 * 4 + 2);
+          }
+          if (need_qsum) {
+            // eps times the dropped normalizer travels to the output pass through tensor memory: each half adds its part
+            tmem_st1(lane_base + COL_MAIL + 4 * p + ch, a.eps * qsum);
+            tmem_wait_st();
+          }
+        } else {
+          const float inv = row < nvalid ? 1.f / sum : 0.f;  // tokens past the end contribute nothing
+          const float* e63v = vec(p, 2);
+          auto k_block = [&](const float* ee, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              const int jj = jj0 + h2;  // channels [8 jj, 8 jj + 8)
+              float x[8], ks[8];
+              load_x8(sb + OFF_X, row, jj, x);
+              const float4 ea = *reinterpret_cast<const float4*>(e63v + jj * 8);
+              const float4 eb = *reinterpret_cast<const float4*>(e63v + jj * 8 + 4);
+              const float e63[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
+#pragma unroll
+              for (int i = 0; i < 8; ++i) ks[i] = ee[h2 * 8 + i] * inv * ex2f(-x[i]);
+              if (MODE == 0) sts128(sb + OFF_QK + ch * 16384 + sw128(C + row, jj & 7), pack8(ks, f16));
+#pragma unroll
+              for (int i = 0; i < 8; ++i) ks[i] *= e63[i];
+              // kh: row = token, MN-major A operand of the state update (slab = column half)
+              sts128(sb + OFF_KH + ch * 8192 + sw128(row, jj & 7), pack8(ks, true));
+            }
+          };
           tmem_ld16(ycol, ya);
 #pragma unroll 1
           for (int b2 = 0; b2 < 2; ++b2) {
             tmem_wait_ld();
             tmem_ld16(ycol + b2 * 32 + 16, yb);
-#pragma unroll
-            for (int i = 0; i < 16; ++i) m = fmaxf(m, ya[i]);
+            k_block(ya, ch * 8 + b2 * 4);
             tmem_wait_ld();
-            tmem_ld16(ycol + ((b2 * 32 + 32) & 63), ya);  // wraps to the first block: the next sweep starts there
-#pragma unroll
-            for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
-          }
-          s_pmax[ch * 64 + row] = m;
-        }
-        named_bar_sync(phi_bar, 128);
-        m = fmaxf(s_pmax[row], s_pmax[64 + row]);
-        const float mb = m * L2E;
-        if (is_q) {
-          if (!fail) {
-            auto q_block = [&](const float* yy, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
-#pragma unroll
-              for (int h2 = 0; h2 < 2; ++h2) {
-                const int jj = jj0 + h2;
-                float x[8], v[8];
-                load_x8(sb + OFF_X, row, jj, x);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = ex2f(fmaf(yy[h2 * 8 + i], L2E, x[i] - mb));
-                if (need_qsum) {
-#pragma unroll
-                  for (int i = 0; i < 8; ++i) qsum += ex2f(fmaf(yy[h2 * 8 + i], L2E, -mb));
-                }
-                sts128(sb + OFF_QK + ch * 16384 + sw128(row, jj & 7), pack8(v, f16));
-              }
-            };
-#pragma unroll 1
-            for (int b2 = 0; b2 < 2; ++b2) {
-              tmem_wait_ld();
-              tmem_ld16(ycol + b2 * 32 + 16, yb);
-              q_block(ya, ch * 8 + b2 * 4);
-              tmem_wait_ld();
-              if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
-              q_block(yb, ch * 8 + b2 * 4 + 2);
-            }
-            if (need_qsum) s_psum[ch * 64 + row] = qsum;
-          }
-          if (need_qsum) {
-            named_bar_sync(phi_bar, 128);
-            qsum = s_psum[row] + s_psum[64 + row];
-            if (ch == 0 && !fail) {  // eps times the dropped normalizer travels to the output pass through tensor memory
-              tmem_st1(lane_base + COL_MAIL + p, a.eps * qsum);
-              tmem_wait_st();
-            }
-          }
-        } else {
-          // key rows: one sweep forms e = exp(y - max) and its sum and parks e in Y's own columns; the last sweep
-          // writes ks = e 2^-x / sum and kh = ks 2^(b_C - b_mid)
-          float sum = 0.f;
-          if (!fail) {
-#pragma unroll 1
-            for (int b2 = 0; b2 < 2; ++b2) {
-              tmem_wait_ld();
-              tmem_ld16(ycol + b2 * 32 + 16, yb);
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                ya[i] = ex2f(fmaf(ya[i], L2E, -mb));
-                sum += ya[i];
-              }
-              tmem_st16(ycol + b2 * 32, ya);
-              tmem_wait_ld();
-              if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                yb[i] = ex2f(fmaf(yb[i], L2E, -mb));
-                sum += yb[i];
-              }
-              tmem_st16(ycol + b2 * 32 + 16, yb);
-            }
-            tmem_wait_st();
-            s_psum[ch * 64 + row] = sum;
-          }
-          named_bar_sync(phi_bar, 128);
-          sum = s_psum[row] + s_psum[64 + row];
-          // every key-row thread has the maxima and sums it needs: from here on the kh tile may be written
-          named_bar_sync(phi_bar, 128);
-          if (!fail) {
-            const float inv = row < nvalid ? 1.f / sum : 0.f;  // tokens past the end contribute nothing
-            const float* e63v = vec(p, 2);
-            auto k_block = [&](const float* ee, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
-#pragma unroll
-              for (int h2 = 0; h2 < 2; ++h2) {
-                const int jj = jj0 + h2;  // channels [8 jj, 8 jj + 8)
-                float x[8], ks[8];
-                load_x8(sb + OFF_X, row, jj, x);
-                const float4 ea = *reinterpret_cast<const float4*>(e63v + jj * 8);
-                const float4 eb = *reinterpret_cast<const float4*>(e63v + jj * 8 + 4);
-                const float e63[8] = {ea.x, ea.y, ea.z, ea.w, eb.x, eb.y, eb.z, eb.w};
-#pragma unroll
-                for (int i = 0; i < 8; ++i) ks[i] = ee[h2 * 8 + i] * inv * ex2f(-x[i]);
-                if (MODE == 0) sts128(sb + OFF_QK + ch * 16384 + sw128(C + row, jj & 7), pack8(ks, f16));
-#pragma unroll
-                for (int i = 0; i < 8; ++i) ks[i] *= e63[i];
-                // kh: row = token, MN-major A operand of the state update (slab = column half)
-                sts128(sb + OFF_KH + ch * 8192 + sw128(row, jj & 7), pack8(ks, true));
-              }
-            };
-            tmem_ld16(ycol, ya);
-#pragma unroll 1
-            for (int b2 = 0; b2 < 2; ++b2) {
-              tmem_wait_ld();
-              tmem_ld16(ycol + b2 * 32 + 16, yb);
-              k_block(ya, ch * 8 + b2 * 4);
-              tmem_wait_ld();
-              if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
-              k_block(yb, ch * 8 + b2 * 4 + 2);
-            }
+            if (b2 < 1) tmem_ld16(ycol + b2 * 32 + 32, ya);
+            k_block(yb, ch * 8 + b2 * 4 + 2);
           }
         }
       }
@@ -842,6 +844,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (MODE == 0 && is_q) {
         // ---- causal mask, fp16 scores: this thread's 32 columns of row `row` -------------------------------------------
         WAITF(B_MMA2, p);
+        if (n > 0) WAITF(B_MMA3, pp);  // the score tile was the previous chunk's MMA 3 operand
         if (!fail) {
           tc_fence_after_sync();
           tmem_ld32(lane_base + COL_P + ch * 32, y);
