@@ -124,6 +124,19 @@ __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
   f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
   f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
 }
+// 8 bf16 values -> 4 packed pairs of fp32
+__device__ __forceinline__ void unpack8p(const uint4& v, uint64_t* f) {
+  f[0] = f2_pack(bf16_lo(v.x), bf16_hi(v.x)); f[1] = f2_pack(bf16_lo(v.y), bf16_hi(v.y));
+  f[2] = f2_pack(bf16_lo(v.z), bf16_hi(v.z)); f[3] = f2_pack(bf16_lo(v.w), bf16_hi(v.w));
+}
+// 4 packed pairs of fp32 -> 8 packed 16-bit values, fp16 or bf16
+__device__ __forceinline__ uint4 pack8p(const uint64_t* v, bool f16) {
+  float f[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) f2_unpack(v[i], f[2 * i], f[2 * i + 1]);
+  return f16 ? make_uint4(pack_f16(f[0], f[1]), pack_f16(f[2], f[3]), pack_f16(f[4], f[5]), pack_f16(f[6], f[7]))
+             : make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+}
 // 8 values -> 8 packed 16-bit values, fp16 or bf16
 __device__ __forceinline__ uint4 pack8(const float* v, bool f16) {
   return f16 ? make_uint4(pack_f16(v[0], v[1]), pack_f16(v[2], v[3]), pack_f16(v[4], v[5]), pack_f16(v[6], v[7]))
@@ -448,15 +461,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // conv mapping: thread = (stream, channel octet, 8 consecutive tokens); gate mapping: thread = (channel, half chunk)
     const int cv_stream = tid >> 7, cv_oct = tid & 15, cv_rg = (tid >> 4) & 7;
     const bool cv_on = MODE == 0 || cv_stream == 1;
-    float cw[8][4];
+    uint64_t cw[4][4];  // [channel pair][tap], packed pairs of fp32
     {
       const bf16* w = cv_stream ? a.w_k : a.w_q;
       const int head = cv_stream ? j : h;
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch)
+      for (int cp = 0; cp < 4; ++cp)
 #pragma unroll
-        for (int dl = 0; dl < 4; ++dl)
-          cw[ch][dl] = dl < a.K ? __bfloat162float(w[((size_t)head * D + cv_oct * 8 + ch) * a.K + dl]) : 0.f;
+        for (int dl = 0; dl < 4; ++dl) {
+          const size_t i0 = ((size_t)head * D + cv_oct * 8 + 2 * cp) * a.K + dl;
+          cw[cp][dl] = dl < a.K ? f2_pack(__bfloat162float(w[i0]), __bfloat162float(w[i0 + a.K])) : f2_pack(0.f, 0.f);
+        }
     }
     const uint32_t au = sb + OFF_AU + (cv_oct >> 3) * 16384;  // this thread's 64-channel slab
     const int cjc = cv_oct & 7, crow0 = cv_stream * 64 + cv_rg * 8;
@@ -499,36 +514,36 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // ---- conv, in place: the three rows in front of this thread's rows belong to another thread (or to the previous
       // chunk), so they are read before the barrier and every row is overwritten only after it ------------------------
       WAITF(B_RAW_FULL, p);
-      float x1[8], x2[8], x3[8], x0[8];
+      uint64_t x1[4], x2[4], x3[4], x0[4];  // sliding window of raw rows, packed pairs of fp32
       if (cv_on && !fail) {
         if (cv_rg == 0) {
           const uint4* hl = reinterpret_cast<const uint4*>(sg + OFF_HALO) + cv_stream * 48 + cv_oct;
-          unpack8(hl[0], x3); unpack8(hl[16], x2); unpack8(hl[32], x1);
+          unpack8p(hl[0], x3); unpack8p(hl[16], x2); unpack8p(hl[32], x1);
         } else {
-          unpack8(lds128(au + sw128(crow0 - 3, cjc)), x3);
-          unpack8(lds128(au + sw128(crow0 - 2, cjc)), x2);
-          unpack8(lds128(au + sw128(crow0 - 1, cjc)), x1);
+          unpack8p(lds128(au + sw128(crow0 - 3, cjc)), x3);
+          unpack8p(lds128(au + sw128(crow0 - 2, cjc)), x2);
+          unpack8p(lds128(au + sw128(crow0 - 1, cjc)), x1);
         }
       }
       if (tid == 0) { s_rmax[p] = 0; s_vmax[p] = 0; }
       fail = named_bar_or(1, PREP_THREADS, fail);
       if (fail) break;
       if (cv_on) {
-#pragma unroll 2
+#pragma unroll 4
         for (int i = 0; i < 8; ++i) {
           const uint32_t ad = au + sw128(crow0 + i, cjc);
-          unpack8(lds128(ad), x0);
-          float u[8];
+          unpack8p(lds128(ad), x0);
+          uint64_t u[4];
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch)
-            u[ch] = fmaf(cw[ch][0], x0[ch], fmaf(cw[ch][1], x1[ch], fmaf(cw[ch][2], x2[ch], cw[ch][3] * x3[ch])));
-          sts128(ad, pack8(u, true));
+          for (int cp = 0; cp < 4; ++cp)
+            u[cp] = f2_fma(cw[cp][0], x0[cp], f2_fma(cw[cp][1], x1[cp], f2_fma(cw[cp][2], x2[cp], f2_mul(cw[cp][3], x3[cp]))));
+          sts128(ad, pack8p(u, true));
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) { x3[ch] = x2[ch]; x2[ch] = x1[ch]; x1[ch] = x0[ch]; }
+          for (int cp = 0; cp < 4; ++cp) { x3[cp] = x2[cp]; x2[cp] = x1[cp]; x1[cp] = x0[cp]; }
         }
         if (cv_rg == 7) {  // the last three raw rows of the chunk are the next chunk's halo (bf16 values: exact repack)
           uint4* hl = reinterpret_cast<uint4*>(sg + OFF_HALO) + cv_stream * 48 + cv_oct;
-          hl[0] = pack8(x3, false); hl[16] = pack8(x2, false); hl[32] = pack8(x1, false);
+          hl[0] = pack8p(x3, false); hl[16] = pack8p(x2, false); hl[32] = pack8p(x1, false);
         }
       }
       fence_proxy_async();
@@ -728,16 +743,20 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (MODE == 0) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(y[i]));
+            const uint64_t dm2 = f2_pack(dm, dm);
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
-              float w[8];
+              uint64_t w[4];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) w[i] = dm * y[8 * q4 + i];
-              sts128(sb + OFF_SBF + ch * 16384 + sw128(c, b2 * 4 + q4), pack8(w, f16));
+              for (int i = 0; i < 4; ++i) w[i] = f2_mul(dm2, f2_pack(y[8 * q4 + 2 * i], y[8 * q4 + 2 * i + 1]));
+              sts128(sb + OFF_SBF + ch * 16384 + sw128(c, b2 * 4 + q4), pack8p(w, f16));
             }
           }
+          {
+            const uint64_t dC2 = f2_pack(dC, dC);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) y[i] *= dC;
+            for (int i = 0; i < 32; i += 2) f2_unpack(f2_mul(dC2, f2_pack(y[i], y[i + 1])), y[i], y[i + 1]);
+          }
           tmem_st32(lane_base + COL_S + blk * 32, y);
         }
         if (ch == 1) {
