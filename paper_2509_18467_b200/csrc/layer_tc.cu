@@ -34,13 +34,14 @@ static bool make_map(CUtensorMap* m, const void* ptr, int heads, int T, int B, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// State at the start of every segment from the per-segment end states (computed from zero) and total decays:
-// start[0] = given state; start[s] = decay[s-1] * start[s-1] + local[s-1]  (Eq. 4 unrolled over whole segments).
+// State at the start of every segment from the end states of its pieces (each computed from a zero state) and their
+// total decays: running state cur = given state; after piece i: cur = decay[i] * cur + local[i] (Eq. 4 unrolled over
+// whole pieces); start[seg] = cur in front of the segment's first piece.
 // One thread per state entry (the d_k x d_v entries of S, then the d_k entries of z) of one (batch, head).
 __global__ void segment_scan_kernel(const float* __restrict__ S0, const float* __restrict__ z0,
                                     const float* __restrict__ loc_S, const float* __restrict__ loc_z,
                                     const float* __restrict__ dtot, float* __restrict__ start_S,
-                                    float* __restrict__ start_z, int BH, int nseg) {
+                                    float* __restrict__ start_z, int BH, int nseg, int nsub) {
   const int per = D * D + D;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= BH * per) return;
@@ -50,11 +51,14 @@ __global__ void segment_scan_kernel(const float* __restrict__ S0, const float* _
   const int e = isz ? 0 : r % D;
   float cur = isz ? (z0 ? z0[(size_t)bh * D + c] : 0.f) : (S0 ? S0[((size_t)bh * D + c) * D + e] : 0.f);
   for (int sgm = 0; sgm < nseg; ++sgm) {
-    const size_t si = (size_t)bh * nseg + sgm;
-    if (isz) start_z[si * D + c] = cur; else start_S[(si * D + c) * D + e] = cur;
+    const size_t so = (size_t)bh * nseg + sgm;
+    if (isz) start_z[so * D + c] = cur; else start_S[(so * D + c) * D + e] = cur;
     if (sgm + 1 < nseg) {
-      const float loc = isz ? loc_z[si * D + c] : loc_S[(si * D + c) * D + e];
-      cur = fmaf(exp2f(dtot[si * D + c]), cur, loc);
+      for (int sb = 0; sb < nsub; ++sb) {
+        const size_t si = so * nsub + sb;
+        const float loc = isz ? loc_z[si * D + c] : loc_S[(si * D + c) * D + e];
+        cur = fmaf(exp2f(dtot[si * D + c]), cur, loc);
+      }
     }
   }
 }
@@ -69,10 +73,25 @@ int layer_tc_segments(const lawcat_params& p) {
   return n < 1 ? 1 : n;
 }
 
+// Pieces per segment in the state-only pre-pass: its thread blocks are independent, so cutting the segments finer lets
+// them fill the SMs in whole waves. Picks the split with the fewest chunks per SM (a small charge per extra piece).
+static int layer_tc_pieces(const lawcat_params& p, int nseg) {
+  const int chunks = (p.T + tc::C - 1) / tc::C;
+  const int cps = (chunks + nseg - 1) / nseg;
+  int best = 1, best_cost = 1 << 30;
+  for (int ns = 1; ns <= 8 && ns * 4 <= cps; ++ns) {
+    const int ctas = p.B * p.H * (nseg - 1) * ns;
+    const int cost = ((ctas + 147) / 148) * ((cps + ns - 1) / ns + 2);
+    if (cost < best_cost) { best_cost = cost; best = ns; }
+  }
+  return best;
+}
+
 size_t layer_tc_workspace_bytes(const lawcat_params& p) {
   const int nseg = layer_tc_segments(p);
   if (nseg == 1) return 0;
-  return sizeof(float) * (size_t)p.B * p.H * nseg * (2 * (tc::D * tc::D + tc::D) + tc::D);
+  const size_t pieces = (size_t)nseg * layer_tc_pieces(p, nseg);
+  return sizeof(float) * (size_t)p.B * p.H * ((pieces + nseg) * (tc::D * tc::D + tc::D) + pieces * tc::D);
 }
 
 bool layer_tc_supported(const lawcat_params& p) {
@@ -106,7 +125,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   const int BH = p.B * p.H;
   if (nseg == 1) {
     a.S0 = S0; a.z0 = z0; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
-    a.grid_nseg = 1; a.seg_in = 0; a.seg_out = 0;
+    a.grid_nseg = 1; a.nsub = 1; a.seg_in = 0; a.seg_out = 0;
     LaunchScope _ls("layer_tc", c.stream);
     layer_tc_kernel<0><<<BH, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
     LAWCAT_CHECK_LAUNCH();
@@ -115,28 +134,29 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   // Several segments per sequence: (1) every segment but the last computes its end state from a zero state, and the
   // total decay of the segment; (2) a scan over the segments turns these into the state at each segment's start;
   // (3) the layer runs on all segments at once, each from its start state.
+  const int nsub = layer_tc_pieces(p, nseg);
   const size_t nS = (size_t)BH * nseg * D * D, nz = (size_t)BH * nseg * D;
-  float* loc_S = (float*)ws;
-  float* loc_z = loc_S + nS;
-  float* dtot = loc_z + nz;
-  float* start_S = dtot + nz;
-  float* start_z = start_S + nS;
+  float* loc_S = (float*)ws;              // [BH, nseg, nsub, D, D]
+  float* loc_z = loc_S + nS * nsub;       // [BH, nseg, nsub, D]
+  float* dtot = loc_z + nz * nsub;        // [BH, nseg, nsub, D]
+  float* start_S = dtot + nz * nsub;      // [BH, nseg, D, D]
+  float* start_z = start_S + nS;          // [BH, nseg, D]
   {
     TcArgs b1 = a;
     b1.S0 = nullptr; b1.z0 = nullptr; b1.S_T = loc_S; b1.z_T = loc_z; b1.dtot = dtot;
-    b1.grid_nseg = nseg - 1; b1.seg_in = 1; b1.seg_out = 1;
+    b1.grid_nseg = nseg - 1; b1.nsub = nsub; b1.seg_in = 1; b1.seg_out = 1;
     LaunchScope _ls("layer_tc_state", c.stream);
-    layer_tc_kernel<1><<<BH * (nseg - 1), THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, b1);
+    layer_tc_kernel<1><<<BH * (nseg - 1) * nsub, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, b1);
     LAWCAT_CHECK_LAUNCH();
   }
   {
     const int total = BH * (D * D + D);
     LaunchScope _ls("segment_scan", c.stream);
-    segment_scan_kernel<<<(total + 255) / 256, 256, 0, c.stream>>>(S0, z0, loc_S, loc_z, dtot, start_S, start_z, BH, nseg);
+    segment_scan_kernel<<<(total + 255) / 256, 256, 0, c.stream>>>(S0, z0, loc_S, loc_z, dtot, start_S, start_z, BH, nseg, nsub);
     LAWCAT_CHECK_LAUNCH();
   }
   a.S0 = start_S; a.z0 = start_z; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
-  a.grid_nseg = nseg; a.seg_in = 1; a.seg_out = 0;
+  a.grid_nseg = nseg; a.nsub = 1; a.seg_in = 1; a.seg_out = 0;
   LaunchScope _ls("layer_tc", c.stream);
   layer_tc_kernel<0><<<BH * nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
   LAWCAT_CHECK_LAUNCH();

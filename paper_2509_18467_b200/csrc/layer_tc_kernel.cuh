@@ -114,8 +114,9 @@ struct TcArgs {
   int T, H, Hkv, K;
   int nseg, seg_len;     // segments per sequence and tokens per segment (a multiple of C)
   int grid_nseg;         // segments of each sequence covered by this launch (the first grid_nseg of nseg)
-  int seg_in;            // 1: S0/z0 are indexed [b,h,seg]; 0: [b,h] and they apply to segment 0 only
-  int seg_out;           // 1: S_T/z_T are indexed [b,h,seg]; 0: [b,h] and only the last segment writes them
+  int nsub;              // pieces each segment is cut into by this launch (whole chunks; 1 = the segment itself)
+  int seg_in;            // 1: S0/z0 are indexed [b,h,seg*nsub+sub]; 0: [b,h] and they apply to segment 0 only
+  int seg_out;           // 1: S_T/z_T (and dtot) are indexed [b,h,seg*nsub+sub]; 0: [b,h], written by the last segment
   int gate_mode;
   float inv_tau, eps;
 };
@@ -218,14 +219,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int seg = blockIdx.x % a.grid_nseg;
-  const int bh = blockIdx.x / a.grid_nseg;
+  const int sub = blockIdx.x % a.nsub;
+  const int seg = (blockIdx.x / a.nsub) % a.grid_nseg;
+  const int bh = blockIdx.x / (a.nsub * a.grid_nseg);
   const int h = bh % a.H, b = bh / a.H;
   const int G = a.H / a.Hkv, j = h / G;
-  const int t_begin = seg * a.seg_len;
-  const int t_end = min(a.T, t_begin + a.seg_len);
+  const int cps = a.seg_len / C;  // chunks per segment; piece `sub` covers chunks [sub cps / nsub, (sub + 1) cps / nsub)
+  const int t_begin = min(a.T, seg * a.seg_len + (sub * cps / a.nsub) * C);
+  const int t_end = min(a.T, seg * a.seg_len + ((sub + 1) * cps / a.nsub) * C);
   const int nchunks = max(0, (t_end - t_begin + C - 1) / C);
-  const size_t seg_idx = (size_t)bh * a.nseg + seg;
+  const size_t seg_idx = ((size_t)bh * a.nseg + seg) * a.nsub + sub;
   const size_t in_idx = a.seg_in ? seg_idx : (size_t)bh, out_idx = a.seg_out ? seg_idx : (size_t)bh;
 
   if ((sb & 1023u) != 0) {  // the swizzled tiles need a 1024-byte aligned base
