@@ -144,18 +144,45 @@ def run_reference(args):
         "gpu_launches": 0}))
 
 
+def dist_setup(backend: str, device=None):
+    """(world, rank, local rank) from the launcher's environment; joins the process group when world > 1. The replicas
+    exchange nothing on the data path: the group only serves the barrier and the max over ranks of the timed region."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        kw = {"device_id": device} if device is not None else {}
+        dist.init_process_group(backend, **kw)
+    return world, rank, local
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's value (every rank gets it)."""
+    if world <= 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64 if str(device) == "cpu" else torch.float32, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: int, steps: int, world: int, ms: float) -> float:
+    """Units per second of the whole job: every rank processes units_per_rank per step (weak scaling)."""
+    return world * units_per_rank * steps / (ms / 1e3)
+
+
 def run_ours(args):
     import torch
     from paper_2509_18467_b200 import api
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    world, rank, local = dist_setup("nccl", dev)
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
     api.lib()
 
     s = I.CONFIGS[args.workload]
@@ -200,12 +227,9 @@ def run_ours(args):
         step()
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, dev)
     tokens = s.B * s.T
-    value = world * tokens * args.steps / (ms / 1e3)
+    value = whole_job_value(tokens, args.steps, world, ms)
 
     # per-kernel device time over the same K steps (CUDA events on the launch stream, bracketing each kernel)
     api.trace_begin()
@@ -248,13 +272,9 @@ def run_ours(args):
         api.lawcat_layer_fwd_host(p, *[hp[n] for n in LAYER_NAMES], h_o, arena)
     e1.record()
     barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
     h2d = sum(hp[n].numel() * hp[n].element_size() for n in LAYER_NAMES)
-    e2e = {"value": world * tokens * e2e_steps / (ms_e2e / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": whole_job_value(tokens, e2e_steps, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": h_o.numel() * h_o.element_size(), "steps": e2e_steps}
     same = bool(torch.equal(h_o.to(dev), o))
 
