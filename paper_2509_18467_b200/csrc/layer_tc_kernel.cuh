@@ -13,13 +13,14 @@
 //               2^x within 2^(+-32 max|g|)); v: bf16 -> fp16 in place (exact)
 //   MMA warp    MMA 1: Y = [u_q; u_k] W_h  (fp16 operands, fp32 accumulate in TMEM)
 //   row warps   (two threads per token row, 64 columns each, straight from tensor memory)
-//               phi: row softmax. Query rows keep exp(y - max) unnormalized: a positive per-token factor cancels in Eq. 8. The decay factors ride in
-//               the exponent of the softmax: qs = 2^(y' + x_t), ks = phi_k 2^(-x_i), kh = phi_k 2^(b_C - b_i) (<= phi_k)
+//               phi: row softmax. Query rows keep exp(y - max) unnormalized: a positive per-token factor cancels in
+//               Eq. 8. The decay factors ride in the exponent of the softmax: qs = 2^(y' + x_t), ks = phi_k 2^(-x_i),
+//               kh = phi_k 2^(b_C - b_i) (<= phi_k)
 //   row warps   state pass: 2^b_mid [S|z] as a 16-bit operand, accumulator [S|z] *= 2^b_C
 //   MMA warp    MMA 2: P = qs ks^T ; O' = qs (2^b_mid [S|z]) ; [S|z] += kh^T [v|1]
 //   row warps   mask: P_ti = 0 for i > t, rounded to fp16
 //   MMA warp    MMA 3: O' += P [v|1]
-//   row warps   o_t = O'_t[:d_v] / (O'_t[d_v] + eps) -> bf16 -> global memory
+//   prep warps  o_t = O'_t[:d_v] / (O'_t[d_v] + eps) -> bf16 -> global memory (the warps of TMEM quadrants 0-1)
 // Operand precision: qs, ks and the state operand are fp16 (11-bit mantissa) while the chunk's x stay within
 // +-8 and the state within +-3e4 -- the usual case -- and bf16 otherwise (range first). bf16 score weights would
 // cost up to 2^-9 relative error per weight, which the first tokens of a sequence do not average out.
@@ -619,11 +620,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
       // ---- v: bf16 -> fp16 in place (exact for |v| in the fp16 normal range) ------------------------------------------
       WAITF(B_V_FULL, p);
-      if (!fail) {
+      // (layer mode: by the warps of TMEM quadrants 2-3 only; those of quadrants 0-1 carry the output pass)
+      if (!fail && (MODE == 1 || (warp & 3) >= 2)) {
+        const int vthreads = MODE == 1 ? PREP_THREADS : PREP_THREADS / 2;
+        const int vt = MODE == 1 ? tid : (tid >> 7) * 64 + ((warp & 3) - 2) * 32 + lane;
         float vm = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint32_t ad = sb + OFF_V + (uint32_t)(tid + PREP_THREADS * i) * 16;
+#pragma unroll 4
+        for (int i = 0; i < 1024 / vthreads; ++i) {
+          const uint32_t ad = sb + OFF_V + (uint32_t)(vt + vthreads * i) * 16;
           float x[8];
           unpack8(lds128(ad), x);
 #pragma unroll
