@@ -18,7 +18,7 @@
 //               kh = phi_k 2^(b_C - b_i) (<= phi_k)
 //   row warps   state pass: 2^b_mid [S|z] as a 16-bit operand, accumulator [S|z] *= 2^b_C
 //   MMA warp    MMA 2: P = qs ks^T ; O' = qs (2^b_mid [S|z]) ; [S|z] += kh^T [v|1]
-//   row warps   mask: P_ti = 0 for i > t, rounded to fp16
+//   row warps   mask: P_ti = 0 for i > t, rounded to fp16 (behind the reading sweeps of the next chunk)
 //   MMA warp    MMA 3: O' += P [v|1]
 //   prep warps  o_t = O'_t[:d_v] / (O'_t[d_v] + eps) -> bf16 -> global memory (the warps of TMEM quadrants 0-1)
 // Operand precision: qs, ks and the state operand are fp16 (11-bit mantissa) while the chunk's x stay within
@@ -197,6 +197,38 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
   }
 }
 
+// Warp-collective bounded wait on a SET of mbarriers: lane l polls barrier l of the set, so the whole set costs one
+// round of polling. (A wait that is already satisfied still takes a few hundred cycles of latency here, and waits issued
+// one after the other add up on the critical path of a chunk.) `mask` selects the barriers, bit l of `parities` is the
+// parity barrier l is waited with. All 32 lanes must call it together. A lane stops polling once its barrier's phase has
+// completed: the barrier may run on into its next phase while the other lanes still wait.
+__device__ __forceinline__ bool wait_set_or_abort(uint32_t bar0, uint32_t mask, uint32_t parities, int lane,
+                                                  volatile int* abort_flag) {
+  const uint32_t b = bar0 + 8u * (uint32_t)lane, par = (parities >> lane) & 1u;
+  bool ok = ((mask >> lane) & 1u) == 0u || mbar_try_wait(b, par);
+  if (__all_sync(0xffffffffu, ok)) {
+    __syncwarp();
+    return true;
+  }
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i) {
+      if (!ok) ok = mbar_try_wait(b, par);
+      if (__all_sync(0xffffffffu, ok)) {
+        __syncwarp();
+        return true;
+      }
+    }
+    bool stop = *abort_flag != 0;
+    if (!stop && clock64() - t0 > 4000000000LL) {
+      *abort_flag = 1;
+      stop = true;
+    }
+    if (__any_sync(0xffffffffu, stop)) return false;
+  }
+}
+
 // MODE 0: the layer forward. MODE 1: state only (no query stream, no output): the end state of a segment that starts
 // from the given state, used to hand the state across segments of one sequence.
 template <int MODE>
@@ -339,6 +371,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // for roles with barriers of their own: remember the failure, skip the work, leave at the role's next OR-barrier
 #define WAITF(b, par)                                    \
   if (!fail && !wait_or_abort(bar(b), (uint32_t)(par), s_abort)) fail = true
+  // several barriers at once (whole warp): BIT(barrier) selects, PAR(barrier, parity) gives its parity
+#define BIT(b) (1u << (b))
+#define PAR(b, par) ((uint32_t)(par) << (b))
+#define WAITSET(mask, pars)                              \
+  if (!wait_set_or_abort(bar(0), (mask), (pars), lane, s_abort)) break
+#define WAITSETF(mask, pars)                             \
+  if (!fail && !wait_set_or_abort(bar(0), (mask), (pars), lane, s_abort)) fail = true
 
   if (warp == TMA_WARP) {
     // ================================================================================================ TMA producer
@@ -375,7 +414,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
   } else if (warp == MMA_WARP) {
     // ================================================================================================ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loop and waits (one lane per barrier of a set); lane 0 issues.
+    {
       // shared-memory descriptors of the operands (all tiles sit at fixed addresses); a K step adds a constant to the
       // start-address field (units of 16 bytes): K-major operand 32 B per step and 16 KB to the second 64-column slab;
       // MN-major swizzled operand 2048 B per step; unswizzled [rows x 16] operand 256 B per step
@@ -401,8 +441,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mma_commit(bar(B_MMA1));
       };
       bool ok = nchunks > 0;
-      if (ok) ok = wait_or_abort(bar(B_U_FULL), 0u, s_abort);
-      if (ok) {
+      if (ok) ok = wait_set_or_abort(bar(0), BIT(B_U_FULL), 0u, lane, s_abort);
+      if (ok && lane == 0) {
         tc_fence_after_sync();
         issue_mma1();
       }
@@ -410,15 +450,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
         if (n + 1 < nchunks) {
           // the mix of the next chunk goes first: its phi pass starts reading Y while this chunk's MMA 2 executes
-          WAIT(B_U_FULL, pp);
-          WAIT(B_Y_FREE, p);
-          tc_fence_after_sync();
-          issue_mma1();
+          WAITSET(BIT(B_U_FULL) | BIT(B_Y_FREE), PAR(B_U_FULL, pp) | PAR(B_Y_FREE, p));
+          if (lane == 0) {
+            tc_fence_after_sync();
+            issue_mma1();
+          }
         }
-        WAIT(B_QK_FULL, p);
-        WAIT(B_SBF_FULL, p);
-        WAIT(B_VH_FULL, p);
-        if (MODE == 0 && n > 0) WAIT(B_O_FREE, pp);
+        WAITSET(BIT(B_QK_FULL) | BIT(B_SBF_FULL) | BIT(B_VH_FULL) | (MODE == 0 && n > 0 ? BIT(B_O_FREE) : 0u),
+                PAR(B_QK_FULL, p) | PAR(B_SBF_FULL, p) | PAR(B_VH_FULL, p) | PAR(B_O_FREE, pp));
+        if (lane == 0) {
         tc_fence_after_sync();
         if (MODE == 0) {
           const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
@@ -445,8 +485,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           mma_commit(bar(B_MMA2));
         }
+        }
         if (MODE == 0) {
-          WAIT(B_PH_FULL, p);
+          WAITSET(BIT(B_PH_FULL), PAR(B_PH_FULL, p));
+          if (lane == 0) {
           tc_fence_after_sync();
           constexpr uint32_t ID_O = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
           constexpr uint32_t ID_OZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
@@ -457,6 +499,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             mma_f16(tmem + COL_OZ, ad, adv(dsc_one, k * (256 >> 4)), ID_OZ, 1);
           }
           mma_commit(bar(B_MMA3));
+          }
         }
       }
     }
@@ -663,6 +706,27 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t ycol = lane_base + COL_Y + ch * 64;
     float dsum = 0.f;  // log2 of this state row's total decay over the segment
     bool fail = false;
+    // ---- causal mask of chunk m, fp16 scores: this (query-row) thread's 32 columns of row `row`. It runs behind the
+    // reading sweeps of chunk m + 1, which do not have to wait for MMA 2 of chunk m.
+    auto mask_chunk = [&](int m) {
+      // (MMA 3 of the chunk before: the score tile was its operand)
+      WAITSETF(BIT(B_MMA2) | (m > 0 ? BIT(B_MMA3) : 0u), PAR(B_MMA2, m & 1) | PAR(B_MMA3, (m - 1) & 1));
+      if (fail) return;
+      tc_fence_after_sync();
+      float s[32];
+      tmem_ld32(lane_base + COL_P + ch * 32, s);
+      tmem_wait_ld();
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = (ch * 32 + q4 * 8 + i <= row) ? s[q4 * 8 + i] : 0.f;
+        sts128(sb + OFF_PH + sw128(row, ch * 4 + q4), pack8(v, true));
+      }
+      fence_proxy_async();
+      tc_fence_before_sync();
+      mbar_arrive(bar(B_PH_FULL));
+    };
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
       const int nvalid = min(C, t_end - (t_begin + n * C));
@@ -731,8 +795,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       // ---- the previous chunk's MMA 2 has completed: the state is updated; qs / ks / kh / state operand are free ---------
-      WAITF(B_X_FULL, p);
-      if (n > 0) WAITF(B_MMA2, pp);
+      if (MODE == 0 && is_q && n > 0) mask_chunk(n - 1);
+      WAITSETF(BIT(B_X_FULL) | (n > 0 ? BIT(B_MMA2) : 0u), PAR(B_X_FULL, p) | PAR(B_MMA2, pp));
       tc_fence_after_sync();
       const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
       // ---- state pass: 16-bit operand 2^b_mid [S|z], accumulator [S|z] *= 2^b_C (this thread: 64 columns of row r128)
@@ -867,27 +931,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_arrive(bar(B_X_FREE));
         mbar_arrive(bar(B_QK_FULL));
       }
-      if (MODE == 0 && is_q) {
-        // ---- causal mask, fp16 scores: this thread's 32 columns of row `row` -------------------------------------------
-        WAITF(B_MMA2, p);
-        if (n > 0) WAITF(B_MMA3, pp);  // the score tile was the previous chunk's MMA 3 operand
-        if (!fail) {
-          tc_fence_after_sync();
-          tmem_ld32(lane_base + COL_P + ch * 32, y);
-          tmem_wait_ld();
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            float v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = (ch * 32 + q4 * 8 + i <= row) ? y[q4 * 8 + i] : 0.f;
-            sts128(sb + OFF_PH + sw128(row, ch * 4 + q4), pack8(v, true));
-          }
-          fence_proxy_async();
-          tc_fence_before_sync();
-          mbar_arrive(bar(B_PH_FULL));
-        }
-      }
     }
+    if (MODE == 0 && is_q && nchunks > 0) mask_chunk(nchunks - 1);
     // ---- final state -------------------------------------------------------------------------------------------------
     if (!fail && !*s_abort && (nchunks == 0 || wait_or_abort(bar(B_MMA2), (uint32_t)((nchunks - 1) & 1), s_abort))) {
       tc_fence_after_sync();
@@ -914,6 +959,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
 #undef WAIT
 #undef WAITF
+#undef WAITSET
+#undef WAITSETF
+#undef BIT
+#undef PAR
 
   // ---- teardown --------------------------------------------------------------------------------------------------------
   tc_fence_before_sync();
