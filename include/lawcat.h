@@ -169,6 +169,8 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
  *   S [B,H,d_k,d_v], z [B,H,d_k] fp32 and cache_q, cache_k (layout as above) are REQUIRED and updated IN PLACE:
  *   the state advances by one token, the caches drop their oldest row and append q_t, k_t.
  *   out: o_t [B,H,d_v]
+ *   ws: device scratch of lawcat_workspace_bytes(p, LAWCAT_OP_DECODE_STEP) bytes (the token's features, decays and
+ *   denominators, handed from the first launch of the step to the second); LAWCAT_ERR_WORKSPACE_TOO_SMALL otherwise.
  */
 int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t, const void* v_t,
                        const void* gate_t, const void* w_q, const void* w_k, const void* W, float* S, float* z,

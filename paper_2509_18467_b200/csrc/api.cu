@@ -74,6 +74,8 @@ size_t lawcat_workspace_bytes(const lawcat_params* p, int op) {
     case LAWCAT_OP_LAYER_FWD:
       if (layer_tc_supported(*p)) return align_up(layer_tc_workspace_bytes(*p), 256);
       return 2 * align_up(sizeof(float) * elems(p, p->H, p->d_k), 256);
+    case LAWCAT_OP_DECODE_STEP:
+      return align_up(decode_workspace_bytes(*p), 256);
     default:
       return 0;
   }
@@ -171,15 +173,16 @@ int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t,
                        const void* gate_t, const void* w_q, const void* w_k, const void* W, float* S, float* z,
                        void* cache_q, void* cache_k, void* o_t, void* ws, size_t ws_bytes, void* stream,
                        int* dev_status) {
-  (void)ws; (void)ws_bytes;
   int r = check_params(p, false);
   if (r) return r;
   const void* const req[] = {q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, o_t};
-  const void* const opt[] = {cache_q, cache_k};
+  const void* const opt[] = {cache_q, cache_k, ws};
   if ((r = check_ptrs(req, opt))) return r;
   if (p->conv_k > 1 && (!cache_q || !cache_k)) return LAWCAT_ERR_INVALID_ARG;
+  const size_t need = lawcat_workspace_bytes(p, LAWCAT_OP_DECODE_STEP);
+  if (need && (!ws || ws_bytes < need)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
   Ctx c{p, (cudaStream_t)stream, dev_status};
-  return launch_decode(c, q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cache_q, cache_k, o_t);
+  return launch_decode(c, q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cache_q, cache_k, o_t, ws);
 }
 
 // ---- host-buffer variant of the layer forward ---------------------------------------------------------------------

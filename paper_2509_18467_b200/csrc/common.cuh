@@ -65,7 +65,8 @@ int launch_gla_bwd_rec(const Ctx& c, const void* qdot, const void* kdot, const v
                        void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws);
 int launch_decode(const Ctx& c, const void* q_t, const void* k_t, const void* v_t, const void* gate_t,
                   const void* w_q, const void* w_k, const void* W, float* S, float* z, void* cache_q, void* cache_k,
-                  void* o_t);
+                  void* o_t, void* ws);
+size_t decode_workspace_bytes(const lawcat_params& p);
 
 // Host-side check of a parameter block (api.cu): LAWCAT_OK, LAWCAT_ERR_INVALID_ARG or LAWCAT_ERR_UNSUPPORTED.
 int validate_params(const lawcat_params* p, bool need_T);

@@ -65,11 +65,13 @@ __global__ void segment_scan_kernel(const float* __restrict__ S0, const float* _
 
 }  // namespace tc
 
-// Segments per sequence: enough thread blocks to fill the SMs (one block per SM), but at least 16 chunks per segment.
+// Segments per sequence: enough thread blocks to fill the SMs (one block per SM), but at least MIN_SEG_CHUNKS chunks per
+// segment (a thread block spends about three chunk times on its set-up and on filling its pipeline).
 int layer_tc_segments(const lawcat_params& p) {
+  constexpr int MIN_SEG_CHUNKS = 4;
   const int chunks = (p.T + tc::C - 1) / tc::C;
   int n = 148 / (p.B * p.H);
-  if (n > chunks / 16) n = chunks / 16;
+  if (n > chunks / MIN_SEG_CHUNKS) n = chunks / MIN_SEG_CHUNKS;
   return n < 1 ? 1 : n;
 }
 

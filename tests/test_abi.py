@@ -48,7 +48,8 @@ def test_version_and_status_strings(L):
 def test_workspace_bytes(L):
     p = api.params(2, 100, 8, 2, 64, 32)
     assert api.workspace_bytes(p, api.OP_CONV_FWD) == 0
-    assert api.workspace_bytes(p, api.OP_DECODE_STEP) == 0
+    # decode: the token's features and decays (3 d_k floats) and one denominator per (sequence, head)
+    assert api.workspace_bytes(p, api.OP_DECODE_STEP) >= 4 * 2 * 8 * (3 * 64 + 1)
     assert api.workspace_bytes(p, api.OP_GLA_BWD) >= 4 * 2 * 100 * 8 * 32
     assert api.workspace_bytes(p, api.OP_CONV_BWD) >= 4 * 2 * 100 * (8 + 2) * 64
     assert api.workspace_bytes(p, api.OP_LAYER_FWD) > 0
@@ -81,9 +82,10 @@ def test_null_and_misaligned_pointers_rejected_on_host(L):
     # workspace too small is reported before any launch
     a13 = [ok] * 4 + [None, None] + [ok] * 7
     assert L.lawcat_gla_bwd(ctypes.byref(p), *a13, None, 0, None, None) == 4
-    # decode needs its caches
+    # decode needs its caches, and its workspace
     a12 = [ok] * 9 + [None, None, ok]
     assert L.lawcat_decode_step(ctypes.byref(p), *a12, None, 0, None, None) == 1
+    assert L.lawcat_decode_step(ctypes.byref(p), *([ok] * 12), None, 0, None, None) == 4
 
 
 def test_missing_library_is_a_hard_error(monkeypatch):
