@@ -97,7 +97,7 @@ size_t layer_tc_workspace_bytes(const lawcat_params& p) {
 }
 
 bool layer_tc_supported(const lawcat_params& p) {
-  return p.dtype == LAWCAT_BF16 && p.d_k == tc::D && p.d_v == tc::D && p.gate_dim == p.d_k &&
+  return p.dtype == LAWCAT_BF16 && p.d_k == tc::D && p.d_v == tc::D && (p.gate_dim == p.d_k || p.gate_dim == 1) &&
          p.phi == LAWCAT_PHI_SOFTMAX && p.normalize == 1 && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
          (p.chunk == 0 || p.chunk == tc::C);
 }
@@ -109,10 +109,13 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   const lawcat_params& p = *c.p;
   CUtensorMap tq, tk, tv, tg;
   if (!make_map(&tq, q, p.H, p.T, p.B, C) || !make_map(&tk, k, p.H_kv, p.T, p.B, C) ||
-      !make_map(&tv, v, p.H_kv, p.T, p.B, C) || !make_map(&tg, gate, p.H, p.T, p.B, C))
+      !make_map(&tv, v, p.H_kv, p.T, p.B, C))
     return LAWCAT_ERR_CUDA;
+  if (p.gate_dim == 1) tg = tq;  // (never used: one logit per token and head is read without a tensor map)
+  else if (!make_map(&tg, gate, p.H, p.T, p.B, C)) return LAWCAT_ERR_CUDA;
   TcArgs a{};
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.o = (bf16*)o;
+  a.gate = (const bf16*)gate; a.gate_dim = p.gate_dim;
   a.w_q = (const bf16*)w_q; a.w_k = (const bf16*)w_k; a.W = (const bf16*)W;
   a.cache_q = (const bf16*)cache_q_in; a.cache_k = (const bf16*)cache_k_in;
   a.dev_status = c.dev_status;

@@ -106,6 +106,8 @@ enum {
 
 struct TcArgs {
   const bf16 *q, *k;     // raw streams (for the halo rows in front of a segment)
+  const bf16* gate;      // gate logits; read directly when there is one per token and head (gate_dim = 1)
+  int gate_dim;          // d_k: one decay per key channel (tile loads); 1: one per head, shared by all channels
   const bf16 *w_q, *w_k, *W, *cache_q, *cache_k;
   const float *S0, *z0;  // state before the first token of the CTA's segment
   float *S_T, *z_T;      // state after the last token of the CTA's segment
@@ -394,11 +396,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tma_load_4d(sb + OFF_AU + s * 16384 + 8192, &tm_k, bar(B_RAW_FULL), s * 64, j, t0, b);
         }
         ar_raw = n;
-        if (n > 0) WAIT(B_G_FREE, pp);
-        mbar_arrive_expect_tx(bar(B_G_FULL), 16384u);
-        tma_load_4d(sb + OFF_G, &tm_g, bar(B_G_FULL), 0, h, t0, b);
-        tma_load_4d(sb + OFF_G + 8192, &tm_g, bar(B_G_FULL), 64, h, t0, b);
-        ar_g = n;
+        if (a.gate_dim != 1) {
+          if (n > 0) WAIT(B_G_FREE, pp);
+          mbar_arrive_expect_tx(bar(B_G_FULL), 16384u);
+          tma_load_4d(sb + OFF_G, &tm_g, bar(B_G_FULL), 0, h, t0, b);
+          tma_load_4d(sb + OFF_G + 8192, &tm_g, bar(B_G_FULL), 64, h, t0, b);
+          ar_g = n;
+        }
         if (n > 0) WAIT(MODE == 0 ? B_MMA3 : B_MMA2, pp);  // the last MMA that reads v
         mbar_arrive_expect_tx(bar(B_V_FULL), 16384u);
         tma_load_4d(sb + OFF_V, &tm_v, bar(B_V_FULL), 0, j, t0, b);
@@ -554,6 +558,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
     };
+    // One decay per head (gate_dim = 1): thread t < C reads the logit of token t of the chunk straight from global memory,
+    // one chunk ahead, and the log-decays of the chunk go to the other threads through (the unused) gate tile.
+    float* const s_g1 = reinterpret_cast<float*>(sg + OFF_G);
+    auto gate1_load = [&](int m) -> float {
+      const int t = t_begin + m * C + tid;
+      return (a.gate_dim == 1 && tid < C && m < nchunks && t < t_end)
+                 ? __bfloat162float(a.gate[((size_t)b * a.T + t) * a.H + h]) : 0.f;
+    };
+    float g1_next = gate1_load(0);
     bool fail = false;
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
@@ -598,7 +611,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       mbar_arrive(bar(B_U_FULL));
 
       // ---- gate: exponents x_t = b_t - b_mid, scanned outwards from MID ------------------------------------------------
-      WAITF(B_G_FULL, p);
+      if (a.gate_dim != 1) WAITF(B_G_FULL, p);
       {
         const uint8_t* gcol = sg + OFF_G + (gc >> 6) * 8192 + (gc & 7) * 2;
         // x[t][c] fp32, 512-byte rows whose 16-byte chunks are XOR-swizzled with t & 7 (conflict-free for this
@@ -609,7 +622,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // tail are decided outside the loops: a branch around each special-function instruction costs more than it.
         float g[32];
         const float L2E = 1.4426950408889634f;
-        if (a.gate_mode == LAWCAT_GATE_LOGDECAY) {
+        if (a.gate_dim == 1) {
+          if (tid < C)
+            s_g1[tid] = a.gate_mode == LAWCAT_GATE_LOGDECAY ? g1_next * L2E : log2_sigmoid(g1_next) * a.inv_tau;
+          g1_next = gate1_load(n + 1);
+          fail = named_bar_or(1, PREP_THREADS, fail);
+          if (fail) break;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) g[i] = s_g1[ghalf * 32 + i];
+        } else if (a.gate_mode == LAWCAT_GATE_LOGDECAY) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const uint32_t raw = *reinterpret_cast<const uint16_t*>(gcol + sw128(ghalf * 32 + i, gjc));

@@ -89,6 +89,17 @@ def test_distillation_lengths(api, T):
     run_case(api, shape(1, T, 4, 2, 45), False)
 
 
+@pytest.mark.parametrize("T,with_state", [(1, False), (64, False), (65, True), (300, False), (1223, True), (8269, True)])
+def test_one_decay_per_head(api, T, with_state):
+    """gate_dim = 1: the decay of a token is shared by all key channels of a head (the scalar-gate reading of Section
+    4.2); short, ragged, carried-state and many-segment lengths."""
+    run_case(api, shape(1, T, 4, 2, 50, gate_dim=1), with_state)
+
+
+def test_one_decay_per_head_sharp_gate(api):
+    run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=1.0), False)
+
+
 def test_long_sequence_many_segments(api):
     """Long enough for the sequence to be split into segments whose states are handed across thread blocks."""
     e, _, _ = run_case(api, shape(1, 8192 + 77, 2, 1, 46), True)
