@@ -21,12 +21,12 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [B, T, heads, 128] bf16 tensor as a 4-D map (channel, head, token, batch) with boxes of 64 channels x rows tokens
-static bool make_map(CUtensorMap* m, const void* ptr, int heads, int T, int B, int rows) {
+// [B, T, heads, dh] bf16 tensor as a 4-D map (channel, head, token, batch) with boxes of 64 channels x rows tokens
+static bool make_map(CUtensorMap* m, const void* ptr, int heads, int T, int B, int rows, int dh) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)T, (cuuint64_t)B};
-  const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)heads * D * 2, (cuuint64_t)T * heads * D * 2};
+  const cuuint64_t dims[4] = {(cuuint64_t)dh, (cuuint64_t)heads, (cuuint64_t)T, (cuuint64_t)B};
+  const cuuint64_t strides[3] = {(cuuint64_t)dh * 2, (cuuint64_t)heads * dh * 2, (cuuint64_t)T * heads * dh * 2};
   const cuuint32_t box[4] = {64, 1, (cuuint32_t)rows, 1};
   const cuuint32_t es[4] = {1, 1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, es,
@@ -41,7 +41,8 @@ static bool make_map(CUtensorMap* m, const void* ptr, int heads, int T, int B, i
 __global__ void segment_scan_kernel(const float* __restrict__ S0, const float* __restrict__ z0,
                                     const float* __restrict__ loc_S, const float* __restrict__ loc_z,
                                     const float* __restrict__ dtot, float* __restrict__ start_S,
-                                    float* __restrict__ start_z, int BH, int nseg, int nsub) {
+                                    float* __restrict__ start_z, int BH, int nseg, int nsub, int dh) {
+  const int D = dh;  // (rows and columns of the state as stored)
   const int per = D * D + D;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= BH * per) return;
@@ -93,11 +94,12 @@ size_t layer_tc_workspace_bytes(const lawcat_params& p) {
   const int nseg = layer_tc_segments(p);
   if (nseg == 1) return 0;
   const size_t pieces = (size_t)nseg * layer_tc_pieces(p, nseg);
-  return sizeof(float) * (size_t)p.B * p.H * ((pieces + nseg) * (tc::D * tc::D + tc::D) + pieces * tc::D);
+  return sizeof(float) * (size_t)p.B * p.H * ((pieces + nseg) * ((size_t)p.d_k * p.d_k + p.d_k) + pieces * p.d_k);
 }
 
 bool layer_tc_supported(const lawcat_params& p) {
-  return p.dtype == LAWCAT_BF16 && p.d_k == tc::D && p.d_v == tc::D && (p.gate_dim == p.d_k || p.gate_dim == 1) &&
+  return p.dtype == LAWCAT_BF16 && (p.d_k == tc::D || p.d_k == 64) && p.d_v == p.d_k &&
+         (p.gate_dim == p.d_k || p.gate_dim == 1) &&
          p.phi == LAWCAT_PHI_SOFTMAX && p.normalize == 1 && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
          (p.chunk == 0 || p.chunk == tc::C);
 }
@@ -108,14 +110,15 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   using namespace tc;
   const lawcat_params& p = *c.p;
   CUtensorMap tq, tk, tv, tg;
-  if (!make_map(&tq, q, p.H, p.T, p.B, C) || !make_map(&tk, k, p.H_kv, p.T, p.B, C) ||
-      !make_map(&tv, v, p.H_kv, p.T, p.B, C))
+  const int dh = p.d_k;
+  if (!make_map(&tq, q, p.H, p.T, p.B, C, dh) || !make_map(&tk, k, p.H_kv, p.T, p.B, C, dh) ||
+      !make_map(&tv, v, p.H_kv, p.T, p.B, C, dh))
     return LAWCAT_ERR_CUDA;
   if (p.gate_dim == 1) tg = tq;  // (never used: one logit per token and head is read without a tensor map)
-  else if (!make_map(&tg, gate, p.H, p.T, p.B, C)) return LAWCAT_ERR_CUDA;
+  else if (!make_map(&tg, gate, p.H, p.T, p.B, C, dh)) return LAWCAT_ERR_CUDA;
   TcArgs a{};
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.o = (bf16*)o;
-  a.gate = (const bf16*)gate; a.gate_dim = p.gate_dim;
+  a.gate = (const bf16*)gate; a.gate_dim = p.gate_dim; a.dh = dh;
   a.w_q = (const bf16*)w_q; a.w_k = (const bf16*)w_k; a.W = (const bf16*)W;
   a.cache_q = (const bf16*)cache_q_in; a.cache_k = (const bf16*)cache_k_in;
   a.dev_status = c.dev_status;
@@ -140,7 +143,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   // total decay of the segment; (2) a scan over the segments turns these into the state at each segment's start;
   // (3) the layer runs on all segments at once, each from its start state.
   const int nsub = layer_tc_pieces(p, nseg);
-  const size_t nS = (size_t)BH * nseg * D * D, nz = (size_t)BH * nseg * D;
+  const size_t nS = (size_t)BH * nseg * dh * dh, nz = (size_t)BH * nseg * dh;
   float* loc_S = (float*)ws;              // [BH, nseg, nsub, D, D]
   float* loc_z = loc_S + nS * nsub;       // [BH, nseg, nsub, D]
   float* dtot = loc_z + nz * nsub;        // [BH, nseg, nsub, D]
@@ -155,9 +158,9 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
     LAWCAT_CHECK_LAUNCH();
   }
   {
-    const int total = BH * (D * D + D);
+    const int total = BH * (dh * dh + dh);
     LaunchScope _ls("segment_scan", c.stream);
-    segment_scan_kernel<<<(total + 255) / 256, 256, 0, c.stream>>>(S0, z0, loc_S, loc_z, dtot, start_S, start_z, BH, nseg, nsub);
+    segment_scan_kernel<<<(total + 255) / 256, 256, 0, c.stream>>>(S0, z0, loc_S, loc_z, dtot, start_S, start_z, BH, nseg, nsub, dh);
     LAWCAT_CHECK_LAUNCH();
   }
   a.S0 = start_S; a.z0 = start_z; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;

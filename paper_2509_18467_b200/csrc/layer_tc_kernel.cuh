@@ -108,6 +108,9 @@ struct TcArgs {
   const bf16 *q, *k;     // raw streams (for the halo rows in front of a segment)
   const bf16* gate;      // gate logits; read directly when there is one per token and head (gate_dim = 1)
   int gate_dim;          // d_k: one decay per key channel (tile loads); 1: one per head, shared by all channels
+  int dh;                // d_k = d_v of the tensors: 128, or 64. A 64-wide head runs as a 128-wide one whose upper 64
+                         // channels (of q, k, gate, v, W, the state) are zero: the tiles' second 64-channel slabs are
+                         // zeroed once and never loaded, and the feature map leaves the padded outputs out
   const bf16 *w_q, *w_k, *W, *cache_q, *cache_k;
   const float *S0, *z0;  // state before the first token of the CTA's segment
   float *S_T, *z_T;      // state after the last token of the CTA's segment
@@ -254,6 +257,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int dh = a.dh, nslab = a.dh >> 6;  // tensor width and its 64-channel slabs (1 or 2)
   const int sub = blockIdx.x % a.nsub;
   const int seg = (blockIdx.x / a.nsub) % a.grid_nseg;
   const int bh = blockIdx.x / (a.nsub * a.grid_nseg);
@@ -301,16 +305,27 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
   // W_h^T into its K-major slabs as fp16: row e holds W[h][c][e] over c
   {
-    const bf16* Wh = a.W + (size_t)h * D * D;
+    const bf16* Wh = a.W + (size_t)h * dh * dh;
 #pragma unroll 1
     for (int idx = tid; idx < 16 * D; idx += THREADS) {
       const int e = idx & (D - 1), oc = idx >> 7;
-      uint32_t w[4];
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      if (e < dh && oc * 8 < dh) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        w[i] = pack_f16(__bfloat162float(Wh[(size_t)(oc * 8 + 2 * i) * D + e]),
-                        __bfloat162float(Wh[(size_t)(oc * 8 + 2 * i + 1) * D + e]));
+        for (int i = 0; i < 4; ++i)
+          w[i] = pack_f16(__bfloat162float(Wh[(size_t)(oc * 8 + 2 * i) * dh + e]),
+                          __bfloat162float(Wh[(size_t)(oc * 8 + 2 * i + 1) * dh + e]));
+      }
       sts128(sb + OFF_W + (oc >> 3) * 16384 + sw128(e, oc & 7), make_uint4(w[0], w[1], w[2], w[3]));
+    }
+  }
+  // a 64-wide head: the second slabs of the raw, gate and v tiles stay zero for good (nothing is loaded into them; the
+  // conv and the v conversion map zeros to zeros)
+  if (nslab == 1) {
+    for (int i = tid; i < 16384 / 16; i += THREADS) reinterpret_cast<uint4*>(sg + OFF_AU + 16384)[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < 8192 / 16; i += THREADS) {
+      reinterpret_cast<uint4*>(sg + OFF_G + 8192)[i] = make_uint4(0u, 0u, 0u, 0u);
+      reinterpret_cast<uint4*>(sg + OFF_V + 8192)[i] = make_uint4(0u, 0u, 0u, 0u);
     }
   }
   // constant "ones" operand and a zeroed z operand (unswizzled 8x8 core matrices)
@@ -321,12 +336,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int NH = st ? a.Hkv : a.H, head = st ? j : h;
     const int t = t_begin - HALO + r;  // token of halo row r
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (t >= 0) {
-      v = *reinterpret_cast<const uint4*>((st ? a.k : a.q) + ((size_t)b * a.T + t) * NH * D + head * D + oc * 8);
+    if (oc * 8 >= dh) {
+      // padded channels: zero
+    } else if (t >= 0) {
+      v = *reinterpret_cast<const uint4*>((st ? a.k : a.q) + ((size_t)b * a.T + t) * NH * dh + head * dh + oc * 8);
     } else {
       const bf16* cache = st ? a.cache_k : a.cache_q;
       const int ci = t + (a.K - 1);  // the cache holds tokens -(K-1) .. -1, oldest first
-      if (cache && ci >= 0) v = *reinterpret_cast<const uint4*>(cache + ((size_t)b * (a.K - 1) + ci) * NH * D + head * D + oc * 8);
+      if (cache && ci >= 0) v = *reinterpret_cast<const uint4*>(cache + ((size_t)b * (a.K - 1) + ci) * NH * dh + head * dh + oc * 8);
     }
     *reinterpret_cast<uint4*>(sg + OFF_HALO + ((st * 3 + r) * 16 + oc) * 16) = v;
   }
@@ -349,14 +366,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int blk = chh * 2 + b2;
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        s[i] = have ? a.S0[(in_idx * D + c) * D + blk * 32 + i] : 0.f;
+        s[i] = (have && c < dh && blk * 32 < dh) ? a.S0[(in_idx * dh + c) * dh + blk * 32 + i] : 0.f;
         mx = fmaxf(mx, fabsf(s[i]));
       }
       tmem_st32(lane_base + COL_S + blk * 32, s);
     }
     if (chh == 1) {
       const bool havez = a.z0 != nullptr && (a.seg_in || seg == 0);
-      const float z0v = havez ? a.z0[in_idx * D + c] : 0.f;
+      const float z0v = (havez && c < dh) ? a.z0[in_idx * dh + c] : 0.f;
       tmem_st1(lane_base + COL_SZ, z0v);
       mx = fmaxf(mx, fabsf(z0v));
     }
@@ -389,24 +406,24 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int t0 = t_begin + n * C;
         const uint32_t pp = (uint32_t)((n - 1) & 1);
         if (n > 0) WAIT(B_MMA1, pp);  // MMA 1 of the previous chunk has read the in-place conv output
-        mbar_arrive_expect_tx(bar(B_RAW_FULL), MODE == 0 ? 32768u : 16384u);
+        mbar_arrive_expect_tx(bar(B_RAW_FULL), (MODE == 0 ? 16384u : 8192u) * (uint32_t)nslab);
 #pragma unroll 1
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < nslab; ++s) {
           if (MODE == 0) tma_load_4d(sb + OFF_AU + s * 16384, &tm_q, bar(B_RAW_FULL), s * 64, h, t0, b);
           tma_load_4d(sb + OFF_AU + s * 16384 + 8192, &tm_k, bar(B_RAW_FULL), s * 64, j, t0, b);
         }
         ar_raw = n;
         if (a.gate_dim != 1) {
           if (n > 0) WAIT(B_G_FREE, pp);
-          mbar_arrive_expect_tx(bar(B_G_FULL), 16384u);
+          mbar_arrive_expect_tx(bar(B_G_FULL), 8192u * (uint32_t)nslab);
           tma_load_4d(sb + OFF_G, &tm_g, bar(B_G_FULL), 0, h, t0, b);
-          tma_load_4d(sb + OFF_G + 8192, &tm_g, bar(B_G_FULL), 64, h, t0, b);
+          if (nslab == 2) tma_load_4d(sb + OFF_G + 8192, &tm_g, bar(B_G_FULL), 64, h, t0, b);
           ar_g = n;
         }
         if (n > 0) WAIT(MODE == 0 ? B_MMA3 : B_MMA2, pp);  // the last MMA that reads v
-        mbar_arrive_expect_tx(bar(B_V_FULL), 16384u);
+        mbar_arrive_expect_tx(bar(B_V_FULL), 8192u * (uint32_t)nslab);
         tma_load_4d(sb + OFF_V, &tm_v, bar(B_V_FULL), 0, j, t0, b);
-        tma_load_4d(sb + OFF_V + 8192, &tm_v, bar(B_V_FULL), 64, j, t0, b);
+        if (nslab == 2) tma_load_4d(sb + OFF_V + 8192, &tm_v, bar(B_V_FULL), 64, j, t0, b);
         ar_v = n;
       }
       if (*s_abort) {
@@ -520,8 +537,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       for (int cp = 0; cp < 4; ++cp)
 #pragma unroll
         for (int dl = 0; dl < 4; ++dl) {
-          const size_t i0 = ((size_t)head * D + cv_oct * 8 + 2 * cp) * a.K + dl;
-          cw[cp][dl] = dl < a.K ? f2_pack(__bfloat162float(w[i0]), __bfloat162float(w[i0 + a.K])) : f2_pack(0.f, 0.f);
+          const size_t i0 = ((size_t)head * dh + cv_oct * 8 + 2 * cp) * a.K + dl;
+          cw[cp][dl] = (dl < a.K && cv_oct * 8 < dh) ? f2_pack(__bfloat162float(w[i0]), __bfloat162float(w[i0 + a.K]))
+                                                    : f2_pack(0.f, 0.f);
         }
     }
     const uint32_t au = sb + OFF_AU + (cv_oct >> 3) * 16384;  // this thread's 64-channel slab
@@ -540,7 +558,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (a.eps != 0.f) den += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1)) + tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
       tmem_wait_ld();
       const float inv = 1.f / den;
-      bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * D + och * 64;
+      bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * dh + och * 64;
       float y[32];
 #pragma unroll 1
       for (int b2 = 0; b2 < 2; ++b2) {
@@ -552,7 +570,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
 #pragma unroll
         for (int i = 0; i < 32; ++i) y[i] *= inv;
-        if (orow_i < onvalid) {
+        if (orow_i < onvalid && och * 64 < dh) {
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4) *reinterpret_cast<uint4*>(orow + b2 * 32 + q4 * 8) = pack8(y + 8 * q4, false);
         }
@@ -648,6 +666,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           for (int i = 0; i < 32; ++i)
             if (ghalf * 32 + i >= nvalid) g[i] = 0.f;  // tokens past the end: no decay
         }
+        if (gc >= dh) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) g[i] = 0.f;     // padded channels of a 64-wide head
+        }
         // the exponent tile is free once the previous chunk's phi pass has read it; the log-decays above did not need it
         mbar_arrive(bar(B_G_FREE));
         if (n > 0) WAITF(B_X_FREE, pp);
@@ -720,6 +742,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const bool is_q = r128 < C;
     const int row = is_q ? r128 : r128 - C;       // token inside the chunk
     const bool phi_on = MODE == 0 || !is_q;       // the state-only pass has no query rows
+    const bool padded = ch >= nslab;              // this thread's 64 columns are the zero padding of a 64-wide head
     const int phi_bar = is_q ? 3 : 4;             // the query rows and the key rows meet among themselves (128 threads each)
     const float L2E = 1.4426950408889634f;
     const bool need_qsum = a.eps != 0.f;  // the dropped softmax normalizer of the query rows only matters next to eps
@@ -771,6 +794,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
           }
+          if (padded) m = -INFINITY;  // the padded outputs of a 64-wide head take no part in the softmax
           tmem_st1(mail_mine, m);
           tmem_wait_st();
         }
@@ -779,7 +803,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           m = fmaxf(m, tmem_ld1(mail_other));  // (the load of `ya` issued above completes with this wait as well)
           tmem_wait_ld();
         }
-        mb = m * L2E;
+        // (padded outputs: an infinite offset turns every exponential below into an exact zero)
+        mb = padded ? INFINITY : m * L2E;
         if (!is_q) {
           // key rows: e = exp(y - max) and its sum; e is parked in Y's own columns for the writing sweep
           if (!fail) {
@@ -958,7 +983,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (!fail && !*s_abort && (nchunks == 0 || wait_or_abort(bar(B_MMA2), (uint32_t)((nchunks - 1) & 1), s_abort))) {
       tc_fence_after_sync();
       const int c = r128;
-      if (a.dtot != nullptr && ch == 0) a.dtot[seg_idx * D + c] = dsum;
+      if (a.dtot != nullptr && ch == 0 && c < dh) a.dtot[seg_idx * dh + c] = dsum;
       if (a.S_T != nullptr && (a.seg_out || seg == a.nseg - 1)) {
         float s[32];
 #pragma unroll 1
@@ -966,14 +991,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const int blk = ch * 2 + b2;
           tmem_ld32(lane_base + COL_S + blk * 32, s);
           tmem_wait_ld();
+          if (c < dh && blk * 32 < dh) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 4)
-            *reinterpret_cast<float4*>(a.S_T + (out_idx * D + c) * D + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<float4*>(a.S_T + (out_idx * dh + c) * dh + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
+          }
         }
         if (ch == 1 && a.z_T) {
           const float z = tmem_ld1(lane_base + COL_SZ);
           tmem_wait_ld();
-          a.z_T[out_idx * D + c] = z;
+          if (c < dh) a.z_T[out_idx * dh + c] = z;
         }
       }
     }

@@ -100,6 +100,23 @@ def test_one_decay_per_head_sharp_gate(api):
     run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=1.0), False)
 
 
+def shape64(B, T, H, Hkv, cid, **kw):
+    return I.LayerShape(B, T, H, Hkv, 64, 64, dtype="bf16", config_id=cid, **kw)
+
+
+@pytest.mark.parametrize("T,with_state", [(1, False), (63, True), (64, False), (65, True), (200, False), (1300, True),
+                                          (4133, True)])
+def test_heads_of_width_64(api, T, with_state):
+    """d_k = d_v = 64 (the Llama-3.2-1B shape): the kernel runs such a head as a 128-wide one with zero upper channels;
+    the feature map, the outputs and the states must not see the padding."""
+    run_case(api, shape64(2, T, 4, 2, 52), with_state)
+
+
+@pytest.mark.parametrize("kw", [dict(gate_dim=1), dict(conv_k=2), dict(gate_tau=1.0)])
+def test_heads_of_width_64_variants(api, kw):
+    run_case(api, shape64(1, 333, 8, 2, 53, **kw), True)
+
+
 def test_long_sequence_many_segments(api):
     """Long enough for the sequence to be split into segments whose states are handed across thread blocks."""
     e, _, _ = run_case(api, shape(1, 8192 + 77, 2, 1, 46), True)

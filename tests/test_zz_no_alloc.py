@@ -17,9 +17,9 @@ from paper_2509_18467_b200 import inputs as I
 NAMES = ["q", "k", "v", "gate", "w_q", "w_k", "W"]
 
 
-def _p(api, s):
+def _p(api, s, **kw):
     return api.params(s.B, s.T, s.H, s.H_kv, s.d_k, s.d_v, conv_k=s.conv_k, gate_dim=s.gate_dim, dtype=s.dtype,
-                      gate_tau=s.gate_tau)
+                      gate_tau=s.gate_tau, **kw)
 
 
 @pytest.mark.gpu
@@ -34,7 +34,9 @@ def test_noalloc_matches_regular_entry_point_twice(dtype):
         x = I.make(s, NAMES + ["S0", "z0", "cache_q", "cache_k"])
         d = {n: api.to_device(v, "f32" if n in ("S0", "z0") else s.dtype) for n, v in x.items()}
         p = _p(api, s)
-        ref = api.lawcat_layer_fwd(p, *[d[n] for n in NAMES], d["cache_q"], d["cache_k"], d["S0"], d["z0"])
+        # the entry point runs the recurrent CUDA-core path; chunk = 1 selects the same path in the regular entry point
+        ref = api.lawcat_layer_fwd(_p(api, s, chunk=1), *[d[n] for n in NAMES], d["cache_q"], d["cache_k"], d["S0"],
+                                   d["z0"])
         out = {k: torch.full_like(v, float("nan")) for k, v in ref.items()}
         torch.cuda.synchronize()
         held = torch.cuda.memory_allocated()
