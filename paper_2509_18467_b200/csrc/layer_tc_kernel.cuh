@@ -258,6 +258,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int dh = a.dh, nslab = a.dh >> 6;  // tensor width and its 64-channel slabs (1 or 2)
+  const bool narrow = nslab == 1;          // 64-wide head: everything that belongs to the upper 64 channels is left out
   const int sub = blockIdx.x % a.nsub;
   const int seg = (blockIdx.x / a.nsub) % a.grid_nseg;
   const int bh = blockIdx.x / (a.nsub * a.grid_nseg);
@@ -319,15 +320,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       sts128(sb + OFF_W + (oc >> 3) * 16384 + sw128(e, oc & 7), make_uint4(w[0], w[1], w[2], w[3]));
     }
   }
-  // a 64-wide head: the second slabs of the raw, gate and v tiles stay zero for good (nothing is loaded into them; the
-  // conv and the v conversion map zeros to zeros)
-  if (nslab == 1) {
-    for (int i = tid; i < 16384 / 16; i += THREADS) reinterpret_cast<uint4*>(sg + OFF_AU + 16384)[i] = make_uint4(0u, 0u, 0u, 0u);
-    for (int i = tid; i < 8192 / 16; i += THREADS) {
-      reinterpret_cast<uint4*>(sg + OFF_G + 8192)[i] = make_uint4(0u, 0u, 0u, 0u);
-      reinterpret_cast<uint4*>(sg + OFF_V + 8192)[i] = make_uint4(0u, 0u, 0u, 0u);
-    }
-  }
+  // a 64-wide head: the products run over the first 64 channels / columns only (K = 64, N = 64), so the second slabs of
+  // the tiles are never read; the one exception is the kh operand of the state update, whose M = 128 rows are the key
+  // channels: its second slab is zeroed here and never written
+  if (narrow)
+    for (int i = tid; i < 8192 / 16; i += THREADS) reinterpret_cast<uint4*>(sg + OFF_KH + 8192)[i] = make_uint4(0u, 0u, 0u, 0u);
   // constant "ones" operand and a zeroed z operand (unswizzled 8x8 core matrices)
   for (int i = tid; i < (4096 + 2048) / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_SZ)[i] = 0u;
   // raw rows in front of the segment: earlier tokens, or the conv cache, or zeros (Section 4.1)
@@ -455,10 +452,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         return (d & 0xFFFFFFFF00000000ull) | (uint64_t)((uint32_t)d + off16);
       };
       auto kstep = [](int k) -> uint32_t { return (uint32_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2); };
+      // (a 64-wide head: 4 instead of 8 K steps over the channels, 64 instead of 128 output columns)
+      const int ksteps = narrow ? 4 : 8, NW = narrow ? 64 : 128;
       auto issue_mma1 = [&]() {
-        constexpr uint32_t ID = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_K);
+        const uint32_t ID = instr_desc(128, NW, FMT_F16, MAJOR_K, MAJOR_K);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) mma_f16(tmem + COL_Y, adv(dsc_u, kstep(k)), adv(dsc_w, kstep(k)), ID, k > 0);
+        for (int k = 0; k < 8; ++k)
+          if (k < ksteps) mma_f16(tmem + COL_Y, adv(dsc_u, kstep(k)), adv(dsc_w, kstep(k)), ID, k > 0);
         mma_commit(bar(B_MMA1));
       };
       bool ok = nchunks > 0;
@@ -485,18 +485,20 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
           const int fmt = f16 ? FMT_F16 : FMT_BF16;
           const uint32_t ID_P = instr_desc(128, 64, fmt, MAJOR_K, MAJOR_K);
-          const uint32_t ID_O = instr_desc(128, 128, fmt, MAJOR_K, MAJOR_MN);
+          const uint32_t ID_O = instr_desc(128, NW, fmt, MAJOR_K, MAJOR_MN);
           const uint32_t ID_OZ = instr_desc(128, 16, fmt, MAJOR_K, MAJOR_MN);
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
-            const uint64_t ad = adv(dsc_qk, kstep(k));
-            mma_f16(tmem + COL_P, ad, adv(dsc_ks, kstep(k)), ID_P, k > 0);
-            mma_f16(tmem + COL_O, ad, adv(dsc_s, k * (2048 >> 4)), ID_O, k > 0);
-            mma_f16(tmem + COL_OZ, ad, adv(dsc_sz, k * (256 >> 4)), ID_OZ, k > 0);
+            if (k < ksteps) {
+              const uint64_t ad = adv(dsc_qk, kstep(k));
+              mma_f16(tmem + COL_P, ad, adv(dsc_ks, kstep(k)), ID_P, k > 0);
+              mma_f16(tmem + COL_O, ad, adv(dsc_s, k * (2048 >> 4)), ID_O, k > 0);
+              mma_f16(tmem + COL_OZ, ad, adv(dsc_sz, k * (256 >> 4)), ID_OZ, k > 0);
+            }
           }
         }
         {
-          constexpr uint32_t ID_S = instr_desc(128, 128, FMT_F16, MAJOR_MN, MAJOR_MN);
+          const uint32_t ID_S = instr_desc(128, NW, FMT_F16, MAJOR_MN, MAJOR_MN);
           constexpr uint32_t ID_SZ = instr_desc(128, 16, FMT_F16, MAJOR_MN, MAJOR_MN);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
@@ -511,7 +513,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           WAITSET(BIT(B_PH_FULL), PAR(B_PH_FULL, p));
           if (lane == 0) {
           tc_fence_after_sync();
-          constexpr uint32_t ID_O = instr_desc(128, 128, FMT_F16, MAJOR_K, MAJOR_MN);
+          const uint32_t ID_O = instr_desc(128, NW, FMT_F16, MAJOR_K, MAJOR_MN);
           constexpr uint32_t ID_OZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
@@ -528,7 +530,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ================================================================================================ prep warps
     // conv mapping: thread = (stream, channel octet, 8 consecutive tokens); gate mapping: thread = (channel, half chunk)
     const int cv_stream = tid >> 7, cv_oct = tid & 15, cv_rg = (tid >> 4) & 7;
-    const bool cv_on = MODE == 0 || cv_stream == 1;
+    const bool cv_on = (MODE == 0 || cv_stream == 1) && cv_oct * 8 < dh;
     uint64_t cw[4][4];  // [channel pair][tap], packed pairs of fp32
     {
       const bf16* w = cv_stream ? a.w_k : a.w_q;
@@ -547,15 +549,26 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int gc = tid & 127, ghalf = tid >> 7, gjc = (gc & 63) >> 3;
     // Output pass (threads of TMEM quadrants 0 and 1: 64 query rows x 2 column halves): o = O' / (denominator + eps),
     // Eq. 8, straight from tensor memory to global memory.
+    auto warp_free_o = [&]() {
+      tc_fence_before_sync();
+      mbar_arrive(bar(B_O_FREE));
+    };
     auto out_pass = [&](int m) {
       if ((warp & 3) >= 2) return;
       const int orow_i = (warp & 3) * 32 + lane, och = tid >> 7;
+      if (och >= nslab) {  // 64-wide head: no such columns
+        warp_free_o();
+        return;
+      }
       const int ot0 = t_begin + m * C;
       const int onvalid = min(C, t_end - ot0);
       tc_fence_after_sync();
       float den = tmem_ld1(lane_base + COL_OZ);
       // the query features went in scaled by their dropped softmax normalizer, so eps arrives scaled the same way
-      if (a.eps != 0.f) den += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1)) + tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
+      if (a.eps != 0.f) {
+        den += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1));
+        if (!narrow) den += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
+      }
       tmem_wait_ld();
       const float inv = 1.f / den;
       bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * dh + och * 64;
@@ -640,6 +653,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // tail are decided outside the loops: a branch around each special-function instruction costs more than it.
         float g[32];
         const float L2E = 1.4426950408889634f;
+        const bool g_on = gc < dh;  // (warp-uniform) the upper channels of a 64-wide head have no gate and no exponents
         if (a.gate_dim == 1) {
           if (tid < C)
             s_g1[tid] = a.gate_mode == LAWCAT_GATE_LOGDECAY ? g1_next * L2E : log2_sigmoid(g1_next) * a.inv_tau;
@@ -648,6 +662,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (fail) break;
 #pragma unroll
           for (int i = 0; i < 32; ++i) g[i] = s_g1[ghalf * 32 + i];
+        } else if (!g_on) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) g[i] = 0.f;
         } else if (a.gate_mode == LAWCAT_GATE_LOGDECAY) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
@@ -666,15 +683,14 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           for (int i = 0; i < 32; ++i)
             if (ghalf * 32 + i >= nvalid) g[i] = 0.f;  // tokens past the end: no decay
         }
-        if (gc >= dh) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) g[i] = 0.f;     // padded channels of a 64-wide head
-        }
+
         // the exponent tile is free once the previous chunk's phi pass has read it; the log-decays above did not need it
         mbar_arrive(bar(B_G_FREE));
         if (n > 0) WAITF(B_X_FREE, pp);
         float acc = 0.f;
-        if (ghalf) {
+        if (!g_on) {
+          // nothing: nobody reads these channels' exponents or sums
+        } else if (ghalf) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             acc += g[i];
@@ -712,7 +728,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int vt = MODE == 1 ? tid : (tid >> 7) * 64 + ((warp & 3) - 2) * 32 + lane;
         float vm = 0.f;
 #pragma unroll 4
-        for (int i = 0; i < 1024 / vthreads; ++i) {
+        for (int i = 0; i < nslab * 512 / vthreads; ++i) {
           const uint32_t ad = sb + OFF_V + (uint32_t)(vt + vthreads * i) * 16;
           float x[8];
           unpack8(lds128(ad), x);
@@ -781,7 +797,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         WAITF(B_MMA1, p);
         tc_fence_after_sync();
         float m = -INFINITY;
-        if (!fail) {
+        // (64-wide head: the threads of the upper 64 columns have no outputs: they skip every sweep, and the two threads
+        // of a row have nothing to exchange)
+        if (!fail && !padded) {
           tmem_ld16(ycol, ya);  // 16 columns at a time, the next load in flight while a block is processed
 #pragma unroll 1
           for (int b2 = 0; b2 < 2; ++b2) {
@@ -794,20 +812,22 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
           }
-          if (padded) m = -INFINITY;  // the padded outputs of a 64-wide head take no part in the softmax
-          tmem_st1(mail_mine, m);
-          tmem_wait_st();
         }
-        named_bar_sync(phi_bar, 128);
-        if (!fail) {
-          m = fmaxf(m, tmem_ld1(mail_other));  // (the load of `ya` issued above completes with this wait as well)
-          tmem_wait_ld();
+        if (!narrow) {
+          if (!fail) {
+            tmem_st1(mail_mine, m);
+            tmem_wait_st();
+          }
+          named_bar_sync(phi_bar, 128);
+          if (!fail) {
+            m = fmaxf(m, tmem_ld1(mail_other));  // (the load of `ya` issued above completes with this wait as well)
+            tmem_wait_ld();
+          }
         }
-        // (padded outputs: an infinite offset turns every exponential below into an exact zero)
-        mb = padded ? INFINITY : m * L2E;
+        mb = m * L2E;
         if (!is_q) {
           // key rows: e = exp(y - max) and its sum; e is parked in Y's own columns for the writing sweep
-          if (!fail) {
+          if (!fail && !padded) {
 #pragma unroll 1
             for (int b2 = 0; b2 < 2; ++b2) {
               tmem_wait_ld();
@@ -827,16 +847,18 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               }
               tmem_st16(ycol + b2 * 32 + 16, yb);
             }
-            named_bar_sync(phi_bar, 128);  // the partner has read the row max out of the mailbox
-            tmem_st1(mail_mine, sum);
-            tmem_wait_st();
-          } else {
-            named_bar_sync(phi_bar, 128);
           }
-          named_bar_sync(phi_bar, 128);
-          if (!fail) {
-            sum += tmem_ld1(mail_other);
-            tmem_wait_ld();
+          if (!narrow) {
+            named_bar_sync(phi_bar, 128);  // the partner has read the row max out of the mailbox
+            if (!fail) {
+              tmem_st1(mail_mine, sum);
+              tmem_wait_st();
+            }
+            named_bar_sync(phi_bar, 128);
+            if (!fail) {
+              sum += tmem_ld1(mail_other);
+              tmem_wait_ld();
+            }
           }
         }
       }
@@ -846,7 +868,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_after_sync();
       const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
       // ---- state pass: 16-bit operand 2^b_mid [S|z], accumulator [S|z] *= 2^b_C (this thread: 64 columns of row r128)
-      if (!fail) {
+      // (64-wide head: only the rows and columns that exist)
+      const bool s_on = !narrow || (!padded && r128 < dh);
+      if (!fail && !s_on && !phi_on) mbar_arrive(bar(B_X_FREE));  // (see the end of the pass)
+      if (!fail && s_on) {
         const int c = r128;
         const float bm = vec(p, 0)[c], ft = vec(p, 1)[c];
         const float dm = ex2f(bm), dC = ex2f(bm + ft);
@@ -876,7 +901,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           tmem_st32(lane_base + COL_S + blk * 32, y);
         }
-        if (ch == 1) {
+        if (ch == (narrow ? 0 : 1)) {  // (the thread of the row's last existing column half also carries z)
           const float z = tmem_ld1(lane_base + COL_SZ);
           tmem_wait_ld();
           if (MODE == 0) {
@@ -893,7 +918,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!phi_on) mbar_arrive(bar(B_X_FREE));  // (state-only pass) this thread has read bm, ft and reads no exponents
       }
       // ---- phi, writing sweep -------------------------------------------------------------------------------------------
-      if (phi_on && !fail) {
+      if (phi_on && !fail && !padded) {
         if (is_q) {
           float qsum = 0.f;
           auto q_block = [&](const float* yy, int jj0) {  // 16 columns = channel groups jj0, jj0 + 1
