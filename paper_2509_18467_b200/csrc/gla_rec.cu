@@ -119,7 +119,7 @@ template <typename TQ, typename TS>
 static int gla_fwd_launch(const Ctx& c, GlaArgs& a) {
   const lawcat_params& p = *c.p;
   if (p.B * p.H == 0) return LAWCAT_OK;
-  const int RG = p.d_k >= 32 ? 2 : 1, R = p.d_k / RG;
+  const int RG = p.d_k >= 64 ? 4 : (p.d_k >= 32 ? 2 : 1), R = p.d_k / RG;  // (at most 4 x 160 threads)
   const int CW = (p.d_v + 1 + 31) / 32 * 32;
   const size_t smem = sizeof(float) * ((size_t)3 * TB * p.d_k + (size_t)TB * CW + (size_t)TB * RG * CW);
   const int threads = RG * CW;
@@ -413,15 +413,14 @@ static int gla_bwd_typed(const Ctx& c, GlaArgs& a, void* dv_out) {
   const lawcat_params& p = *c.p;
   const int dk = p.d_k, dv = p.d_v;
   const unsigned grid = p.B * p.H;
-  const int CS = dv >= 32 ? 32 : 16, NSEG = dv / CS;
+  const int CS = 16, NSEG = dv / CS;  // 16 state columns per thread: more, shorter dependent chains per token
   const size_t smem_row = sizeof(float) * ((size_t)6 * TB * dk + (size_t)TB * dv + (size_t)TB * (dv + 1));
-  const int RG = dk >= 32 ? 2 : 1, R = dk / RG;
+  const int RG = dk >= 64 ? 4 : (dk >= 32 ? 2 : 1), R = dk / RG;
   const size_t smem_col = sizeof(float) * ((size_t)3 * TB * dk + (size_t)TB * (dv + 1) + (size_t)TB * RG * dv);
   const int row_thr = (dk * NSEG + 31) / 32 * 32, col_thr = (RG * dv + 31) / 32 * 32;
   // sweep 1: dqdot (forward in time) ; sweep 2: per-head dv (backward in time) ; sweep 3: dkdot + dgate
   LAWCAT_LAUNCH("gla_bwd_row_fwd", c.stream,
-                if (CS == 32) gla_bwd_row_kernel<TS, 32, 0><<<grid, row_thr, smem_row, c.stream>>>(a);
-                else gla_bwd_row_kernel<TS, 16, 0><<<grid, row_thr, smem_row, c.stream>>>(a));
+                gla_bwd_row_kernel<TS, 16, 0><<<grid, row_thr, smem_row, c.stream>>>(a));
   LAWCAT_CHECK_LAUNCH();
   if (R != 16 && R != 32 && R != 64) return LAWCAT_ERR_UNSUPPORTED;
   LAWCAT_LAUNCH("gla_bwd_col", c.stream,
@@ -430,8 +429,7 @@ static int gla_bwd_typed(const Ctx& c, GlaArgs& a, void* dv_out) {
                 else gla_bwd_col_kernel<TS, 64><<<grid, col_thr, smem_col, c.stream>>>(a));
   LAWCAT_CHECK_LAUNCH();
   LAWCAT_LAUNCH("gla_bwd_row_rev", c.stream,
-                if (CS == 32) gla_bwd_row_kernel<TS, 32, 1><<<grid, row_thr, smem_row, c.stream>>>(a);
-                else gla_bwd_row_kernel<TS, 16, 1><<<grid, row_thr, smem_row, c.stream>>>(a));
+                gla_bwd_row_kernel<TS, 16, 1><<<grid, row_thr, smem_row, c.stream>>>(a));
   LAWCAT_CHECK_LAUNCH();
   const size_t total = (size_t)p.B * p.T * p.H_kv * dv;
   LAWCAT_LAUNCH("dv_group_reduce", c.stream,
