@@ -189,7 +189,7 @@ int launch_convmix_fwd(const Ctx& c, const void* q, const void* k, const void* w
 // the mix output, apply the phi Jacobian to the incoming gradient, then
 //   d(conv out) = dy W[h]^T   (query stream: stored per query head; key stream: summed over the group),
 //   dW[h]      += (conv out)^T dy   (registers across the span, one atomic add per entry at the end).
-constexpr int CB_SPAN = 256;
+constexpr int CB_SPAN = 64;
 
 struct ConvMixBwdArgs {
   const void *q, *k, *w_q, *w_k, *W, *cache_q, *cache_k, *d_qdot, *d_kdot;
@@ -204,7 +204,8 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_bwd_kernel(ConvMixBwdArgs 
   float* Ws = smem;                    // [D][D+1]
   float* us = Ws + D * LDW;            // [TT][D]
   float* dys = us + CM_TT * D;         // [TT][D]
-  constexpr int NDW = (D * D + CM_THREADS - 1) / CM_THREADS;
+  // dW is accumulated in 4 x 4 register blocks (two 16-byte shared-memory reads per 16 multiply-adds)
+  constexpr int DB = D / 4, NB = (DB * DB + CM_THREADS - 1) / CM_THREADS;
   constexpr int TPW = CM_TT / (CM_THREADS / 32);
   const int Tn = a.T, K = a.K, G = a.H / a.Hkv;
   const int spans = (Tn + CB_SPAN - 1) / CB_SPAN;
@@ -223,9 +224,11 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_bwd_kernel(ConvMixBwdArgs 
       const TI* w = (const TI*)(stream ? a.w_k : a.w_q);
       const TI* cache = (const TI*)(stream ? a.cache_k : a.cache_q);
       const TI* dout = (const TI*)(stream ? a.d_kdot : a.d_qdot);
-      float dWacc[NDW];
+      float dWacc[NB][16];
 #pragma unroll
-      for (int m = 0; m < NDW; ++m) dWacc[m] = 0.f;
+      for (int m = 0; m < NB; ++m)
+#pragma unroll
+        for (int i = 0; i < 16; ++i) dWacc[m][i] = 0.f;
       for (int t0 = span0; t0 < span1; t0 += CM_TT) {
         __syncthreads();
         for (int i = tid; i < CM_TT * D; i += CM_THREADS) {
@@ -318,22 +321,35 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_bwd_kernel(ConvMixBwdArgs 
         }
         // dW[ch][e] += sum_tl u[tl][ch] dy[tl][e]
 #pragma unroll
-        for (int m = 0; m < NDW; ++m) {
-          const int idx = tid + CM_THREADS * m;
-          if (idx < D * D) {
-            const int ch = idx / D, e = idx % D;
-            float s = 0.f;
-#pragma unroll 8
-            for (int tl = 0; tl < CM_TT; ++tl) s = fmaf(us[tl * D + ch], dys[tl * D + e], s);
-            dWacc[m] += s;
+        for (int m = 0; m < NB; ++m) {
+          const int blk = tid + CM_THREADS * m;
+          if (blk < DB * DB) {
+            const int cb = blk / DB, eb = blk % DB;
+#pragma unroll 4
+            for (int tl = 0; tl < CM_TT; ++tl) {
+              const float4 u4 = *reinterpret_cast<const float4*>(us + tl * D + 4 * cb);
+              const float4 d4 = *reinterpret_cast<const float4*>(dys + tl * D + 4 * eb);
+              const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, dd[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) dWacc[m][4 * i + jj] = fmaf(uu[i], dd[jj], dWacc[m][4 * i + jj]);
+            }
           }
         }
       }
       if (a.dW) {
 #pragma unroll
-        for (int m = 0; m < NDW; ++m) {
-          const int idx = tid + CM_THREADS * m;
-          if (idx < D * D) atomicAdd(a.dW + (size_t)h * D * D + idx, dWacc[m]);
+        for (int m = 0; m < NB; ++m) {
+          const int blk = tid + CM_THREADS * m;
+          if (blk < DB * DB) {
+            const int cb = blk / DB, eb = blk % DB;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int jj = 0; jj < 4; ++jj)
+                atomicAdd(a.dW + (size_t)h * D * D + (size_t)(4 * cb + i) * D + 4 * eb + jj, dWacc[m][4 * i + jj]);
+          }
         }
       }
     }
