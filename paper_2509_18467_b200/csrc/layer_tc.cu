@@ -127,15 +127,18 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   const int nseg = layer_tc_segments(p);
   a.nseg = nseg;
   a.seg_len = ((p.T + nseg - 1) / nseg + C - 1) / C * C;
-  if (cudaFuncSetAttribute(layer_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
-      cudaFuncSetAttribute(layer_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess)
+  const bool narrow = dh == 64;
+  auto* const k_layer = narrow ? layer_tc_kernel<0, true> : layer_tc_kernel<0, false>;
+  auto* const k_state = narrow ? layer_tc_kernel<1, true> : layer_tc_kernel<1, false>;
+  if (cudaFuncSetAttribute(k_layer, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+      cudaFuncSetAttribute(k_state, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess)
     return LAWCAT_ERR_CUDA;
   const int BH = p.B * p.H;
   if (nseg == 1) {
     a.S0 = S0; a.z0 = z0; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
     a.grid_nseg = 1; a.nsub = 1; a.seg_in = 0; a.seg_out = 0;
     LaunchScope _ls("layer_tc", c.stream);
-    layer_tc_kernel<0><<<BH, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
+    k_layer<<<BH, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
     LAWCAT_CHECK_LAUNCH();
     return LAWCAT_OK;
   }
@@ -154,7 +157,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
     b1.S0 = nullptr; b1.z0 = nullptr; b1.S_T = loc_S; b1.z_T = loc_z; b1.dtot = dtot;
     b1.grid_nseg = nseg - 1; b1.nsub = nsub; b1.seg_in = 1; b1.seg_out = 1;
     LaunchScope _ls("layer_tc_state", c.stream);
-    layer_tc_kernel<1><<<BH * (nseg - 1) * nsub, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, b1);
+    k_state<<<BH * (nseg - 1) * nsub, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, b1);
     LAWCAT_CHECK_LAUNCH();
   }
   {
@@ -166,7 +169,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   a.S0 = start_S; a.z0 = start_z; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
   a.grid_nseg = nseg; a.nsub = 1; a.seg_in = 1; a.seg_out = 0;
   LaunchScope _ls("layer_tc", c.stream);
-  layer_tc_kernel<0><<<BH * nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
+  k_layer<<<BH * nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }

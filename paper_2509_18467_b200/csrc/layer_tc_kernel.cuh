@@ -236,7 +236,9 @@ __device__ __forceinline__ bool wait_set_or_abort(uint32_t bar0, uint32_t mask, 
 
 // MODE 0: the layer forward. MODE 1: state only (no query stream, no output): the end state of a segment that starts
 // from the given state, used to hand the state across segments of one sequence.
-template <int MODE>
+// NARROW: heads of width 64 (a.dh == 64) instead of 128; a compile-time switch, so that the 128-wide kernel carries none
+// of its tests.
+template <int MODE, bool NARROW>
 __global__ void __launch_bounds__(THREADS, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g, const TcArgs a) {
@@ -257,8 +259,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int dh = a.dh, nslab = a.dh >> 6;  // tensor width and its 64-channel slabs (1 or 2)
-  const bool narrow = nslab == 1;          // 64-wide head: everything that belongs to the upper 64 channels is left out
+  constexpr int dh = NARROW ? 64 : 128, nslab = dh >> 6;  // tensor width and its 64-channel slabs (1 or 2)
+  constexpr bool narrow = NARROW;  // 64-wide head: everything that belongs to the upper 64 channels is left out
   const int sub = blockIdx.x % a.nsub;
   const int seg = (blockIdx.x / a.nsub) % a.grid_nseg;
   const int bh = blockIdx.x / (a.nsub * a.grid_nseg);
