@@ -233,8 +233,9 @@ def test_split_prefill_equals_one_call(api):
 
 # ------------------------------------------------------------------------------------------------ decode
 @pytest.mark.parametrize("s", [shape(3, 12, 4, 2, 32, 64, "f32"), shape(2, 10, 8, 2, 128, 128, "bf16"),
-                               shape(2, 9, 4, 4, 64, 16, "bf16", gate_dim=1), shape(1, 6, 2, 1, 16, 32, "f32", conv_k=1)],
-                         ids=["f32-d32x64", "bf16-d128", "bf16-g1", "f32-K1"])
+                               shape(2, 9, 4, 4, 64, 16, "bf16", gate_dim=1), shape(1, 6, 2, 1, 16, 32, "f32", conv_k=1),
+                               shape(2, 5, 2, 1, 128, 128, "f32", conv_k=8), shape(9, 4, 4, 2, 64, 64, "bf16")],
+                         ids=["f32-d32x64", "bf16-d128", "bf16-g1", "f32-K1", "f32-d128-K8", "bf16-d64-B9"])
 def test_decode_steps_against_oracle(api, s):
     """T decode steps from a state and caches; every step's output, and the final state and caches, match the oracle."""
     import torch
