@@ -91,6 +91,9 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_features_kernel(DecodeArgs
     const int c = lane + 32 * k, b = b0 + warp;
     zreg[k] = (c < dk && warp < DEC_SEQ && b < a.B) ? a.z[((size_t)b * H + h) * dk + c] : 0.f;
   }
+  // the blocks of decode_state may be scheduled from here on: they start with loads of S, which this kernel never
+  // touches, and wait for the end of this grid before they read anything it writes
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // ---- ... and into shared memory
   {
     uint4* dW = reinterpret_cast<uint4*>(s_W);
@@ -221,6 +224,9 @@ __global__ void __launch_bounds__(DEC_THREADS, 3) decode_state_kernel(DecodeArgs
     for (int i = 0; i < DEC_ROWS; ++i)
       if (i < nr) sreg[i] = __ldcs(reinterpret_cast<const float4*>(Sbh + (size_t)(rgv + RGv * i) * dv) + e4);
   }
+  // (launched with programmatic stream serialization: everything above ran beside decode_features; from here on that
+  // grid has completed, its writes are visible, and it reads the conv caches no more)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const float* in = a.vecs + (size_t)bh * 3 * dk;
   for (int i = tid; i < 3 * dk; i += DEC_THREADS) s_q[i] = in[i];
   for (int i = tid; i < dv; i += DEC_THREADS) s_v[i] = ldf((const T*)a.v_t + ((size_t)b * a.Hkv + j) * dv + i);
@@ -302,7 +308,19 @@ static int decode_typed(const Ctx& c, DecodeArgs& a) {
   if (smem2 > 48 * 1024 &&
       cudaFuncSetAttribute(decode_state_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
     return LAWCAT_ERR_CUDA;
-  LAWCAT_LAUNCH("decode_state", c.stream, decode_state_kernel<T><<<p.B * p.H, DEC_THREADS, smem2, c.stream>>>(a));
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.B * p.H));
+    cfg.blockDim = dim3(DEC_THREADS);
+    cfg.dynamicSmemBytes = smem2;
+    cfg.stream = c.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    LAWCAT_LAUNCH("decode_state", c.stream, cudaLaunchKernelEx(&cfg, decode_state_kernel<T>, a));
+  }
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }
