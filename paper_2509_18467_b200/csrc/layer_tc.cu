@@ -45,6 +45,8 @@ __global__ void segment_scan_kernel(const float* __restrict__ S0, const float* _
   const int D = dh;  // (rows and columns of the state as stored)
   const int per = D * D + D;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the layer kernel may start its set-up
+  asm volatile("griddepcontrol.wait;" ::: "memory");               // (this kernel itself: behind the state-only pass)
   if (idx >= BH * per) return;
   const int bh = idx / per, r = idx % per;
   const bool isz = r >= D * D;
@@ -163,13 +165,35 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   {
     const int total = BH * (dh * dh + dh);
     LaunchScope _ls("segment_scan", c.stream);
-    segment_scan_kernel<<<(total + 255) / 256, 256, 0, c.stream>>>(S0, z0, loc_S, loc_z, dtot, start_S, start_z, BH, nseg, nsub, dh);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((total + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = c.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, segment_scan_kernel, S0, z0, (const float*)loc_S, (const float*)loc_z, (const float*)dtot,
+                       start_S, start_z, BH, nseg, nsub, dh);
     LAWCAT_CHECK_LAUNCH();
   }
   a.S0 = start_S; a.z0 = start_z; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
   a.grid_nseg = nseg; a.nsub = 1; a.seg_in = 1; a.seg_out = 0;
   LaunchScope _ls("layer_tc", c.stream);
-  k_layer<<<BH * nseg, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(BH * nseg));
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = SMEM_ALLOC;
+    cfg.stream = c.stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, k_layer, tq, tk, tv, tg, a);
+  }
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }

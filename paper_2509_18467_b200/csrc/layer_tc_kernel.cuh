@@ -279,6 +279,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   }
 
   // ---- one-time setup --------------------------------------------------------------------------------------------
+  if (MODE == 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // (the scan may be scheduled behind)
   if (tid == 0) {
     const int nphi = MODE == 0 ? 256 : 128;  // threads of the phi pass: all row threads, or the key rows only
     mbar_init(bar(B_RAW_FULL), 1);
@@ -355,6 +356,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const uint32_t tmem = (uint32_t)s_flags[0];
   const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
 
+  // Launched with programmatic stream serialization: the set-up above may run beside the tail of the kernel in front
+  // (the scan over the segments, whose results are the start states read next); from here on that kernel has completed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // initial state into tensor memory: row thread (c, half) owns 64 columns of row c of [S | z]
   if (warp >= ROW_WARP0 && warp < ROW_WARP0 + 8) {
     const int tw = tid - ROW_WARP0 * 32, c = tw & 127, chh = tw >> 7;
