@@ -102,7 +102,7 @@ size_t layer_tc_workspace_bytes(const lawcat_params& p) {
 bool layer_tc_supported(const lawcat_params& p) {
   return p.dtype == LAWCAT_BF16 && (p.d_k == tc::D || p.d_k == 64) && p.d_v == p.d_k &&
          (p.gate_dim == p.d_k || p.gate_dim == 1) &&
-         p.phi == LAWCAT_PHI_SOFTMAX && p.normalize == 1 && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
+         p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
          (p.chunk == 0 || p.chunk == tc::C);
 }
 
@@ -125,7 +125,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   a.cache_q = (const bf16*)cache_q_in; a.cache_k = (const bf16*)cache_k_in;
   a.dev_status = c.dev_status;
   a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k;
-  a.gate_mode = p.gate_mode; a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps;
+  a.gate_mode = p.gate_mode; a.normalize = p.normalize; a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps;
   const int nseg = layer_tc_segments(p);
   a.nseg = nseg;
   a.seg_len = ((p.T + nseg - 1) / nseg + C - 1) / C * C;

@@ -79,7 +79,7 @@ constexpr uint32_t COL_SZ = 448;   // [128 x 16] column 0: normalizer state z
 constexpr uint32_t COL_OZ = 464;   // [128 x 16] column 0: denominator
 constexpr uint32_t COL_MAIL = 480; // spare columns used as per-row mailboxes between threads of one TMEM lane:
                                    // +2, +3: row max / softmax sum of the two column halves; +4 p + half (p = chunk
-                                   // parity): eps * (dropped query normalizer) of that half, row warps -> output pass
+                                   // parity): the dropped query normalizer (softmax sum) of that half, row warps -> output pass
 constexpr uint32_t TMEM_COLS = 512;
 
 // mbarrier indices. "full": producer -> consumer, "free": consumer -> producer. Each completes once per chunk, so the
@@ -124,6 +124,7 @@ struct TcArgs {
   int seg_in;            // 1: S0/z0 are indexed [b,h,seg*nsub+sub]; 0: [b,h] and they apply to segment 0 only
   int seg_out;           // 1: S_T/z_T (and dtot) are indexed [b,h,seg*nsub+sub]; 0: [b,h], written by the last segment
   int gate_mode;
+  int normalize;         // 1: Eq. 8; 0: the numerator alone (the query features then carry their softmax normalizer)
   float inv_tau, eps;
 };
 
@@ -570,13 +571,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int onvalid = min(C, t_end - ot0);
       tc_fence_after_sync();
       float den = tmem_ld1(lane_base + COL_OZ);
-      // the query features went in scaled by their dropped softmax normalizer, so eps arrives scaled the same way
-      if (a.eps != 0.f) {
-        den += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1));
-        if (!narrow) den += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
+      // The query features went in as exp(y - max), without their softmax normalizer: it cancels in Eq. 8 except next to
+      // eps, which therefore gets scaled by it; without normalization the numerator is divided by it.
+      float qs = 0.f;
+      if (a.eps != 0.f || !a.normalize) {
+        qs = tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1));
+        if (!narrow) qs += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
       }
       tmem_wait_ld();
-      const float inv = 1.f / den;
+      const float inv = 1.f / (a.normalize ? fmaf(a.eps, qs, den) : qs);
       bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * dh + och * 64;
       float y[32];
 #pragma unroll 1
@@ -767,7 +770,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const bool padded = ch >= nslab;              // this thread's 64 columns are the zero padding of a 64-wide head
     const int phi_bar = is_q ? 3 : 4;             // the query rows and the key rows meet among themselves (128 threads each)
     const float L2E = 1.4426950408889634f;
-    const bool need_qsum = a.eps != 0.f;  // the dropped softmax normalizer of the query rows only matters next to eps
+    // the dropped softmax normalizer of the query rows only matters next to eps, and without normalization
+    const bool need_qsum = a.eps != 0.f || !a.normalize;
     const uint32_t mail_mine = lane_base + COL_MAIL + 2 + ch, mail_other = lane_base + COL_MAIL + 2 + (ch ^ 1);
     const uint32_t ycol = lane_base + COL_Y + ch * 64;
     float dsum = 0.f;  // log2 of this state row's total decay over the segment
@@ -953,8 +957,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             q_block(yb, ch * 8 + b2 * 4 + 2);
           }
           if (need_qsum) {
-            // eps times the dropped normalizer travels to the output pass through tensor memory: each half adds its part
-            tmem_st1(lane_base + COL_MAIL + 4 * p + ch, a.eps * qsum);
+            // the dropped normalizer travels to the output pass through tensor memory: each half adds its part
+            tmem_st1(lane_base + COL_MAIL + 4 * p + ch, qsum);
             tmem_wait_st();
           }
         } else {

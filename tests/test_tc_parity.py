@@ -145,6 +145,21 @@ def test_eps_in_the_denominator(api):
     check(r["o"], ref["o"], "bf16", "o")
 
 
+@pytest.mark.parametrize("d", [128, 64])
+def test_without_normalization(api, d):
+    """normalize = 0 (the ablation without the normalizer, Section 5.4): the output is the numerator of Eq. 8, with the
+    query features properly normalized by their softmax sum."""
+    s = I.LayerShape(1, 300, 4, 2, d, d, dtype="bf16", config_id=54)
+    x = I.make(s, NAMES)
+    dv = {n: api.to_device(v, s.dtype) for n, v in x.items()}
+    api.trace_begin()
+    r = api.lawcat_layer_fwd(P(api, s, normalize=0), *[dv[n] for n in NAMES])
+    assert any(k.startswith("layer_tc") for k in api.trace_end())
+    ref = O.layer_fwd(oracle_params(s, normalize=0), *[x[n] for n in NAMES])
+    check(r["o"], ref["o"], "bf16", "o")
+    check(r["S_T"], ref["S_T"], "bf16", "S_T", f32_store=True)
+
+
 def test_agrees_with_exact_path_and_split_calls(api):
     """Tensor-core path vs the CUDA-core recurrent path (chunk = 1) on the same device inputs, and one call vs two calls
     that carry the state and the conv caches."""
