@@ -1,0 +1,62 @@
+"""Randomized parity of the tensor-core layer forward: 36 seeded draws of (head width, batch, length, head grouping,
+conv width, gate sharpness, gate width, carried state, normalizer on/off, eps) against the fp64 oracle, through the C ABI.
+
+Tolerance: 1e-2 of the RMS on every tensor, with one documented exception: with the plain sigmoid gate (tau = 1) and one
+decay per head the state is concentrated on the last few tokens, max|S_T| / rms(S_T) reaches 15, and the 2^-11 relative
+rounding of the fp16 operands (conv output into the mix, decayed key features into the state update) shows as up to
+1.5e-2 of the RMS in the strict max / RMS metric; the bound there is 2e-2. The outputs o meet 1e-2 everywhere."""
+import random
+
+import numpy as np
+import pytest
+
+from oracle import lawcat_oracle as O
+from paper_2509_18467_b200 import inputs as I
+from paper_2509_18467_b200.metrics import err_bf16
+
+pytestmark = pytest.mark.gpu
+
+NAMES = ["q", "k", "v", "gate", "w_q", "w_k", "W"]
+
+
+def draws():
+    rng = random.Random(7)
+    out = []
+    for it in range(36):
+        d = rng.choice([64, 128]); Hkv = rng.choice([1, 2, 3]); G = rng.choice([1, 2, 4])
+        B = rng.choice([1, 2, 3]); T = rng.choice([1, 7, 64, 100, 257, 513, 1000, 2100, 4500])
+        K = rng.choice([1, 2, 3, 4]); tau = rng.choice([1.0, 4.0, 16.0]); gd = rng.choice([0, 1])
+        state = rng.random() < 0.5
+        norm = rng.choice([1, 1, 0]); eps = rng.choice([0.0, 0.0, 0.3])
+        out.append((it, d, B, T, Hkv * G, Hkv, K, tau, gd, state, norm, eps))
+    return out
+
+
+@pytest.mark.parametrize("case", draws(), ids=lambda c: f"draw{c[0]}-d{c[1]}-T{c[3]}")
+def test_random_configuration(case):
+    import torch
+    from paper_2509_18467_b200 import api
+    it, d, B, T, H, Hkv, K, tau, gd, state, norm, eps = case
+    s = I.LayerShape(B, T, H, Hkv, d, d, dtype="bf16", config_id=900 + it, conv_k=K, gate_tau=tau, gate_dim=gd)
+    extra = (["S0", "z0"] + (["cache_q", "cache_k"] if K > 1 else [])) if state else []
+    x = I.make(s, NAMES + extra)
+    dv = {n: api.to_device(x[n], "f32" if n in ("S0", "z0") else "bf16") for n in x}
+    p = api.params(B, T, H, Hkv, d, d, conv_k=K, gate_tau=tau, gate_dim=s.gate_dim, normalize=norm, eps=eps)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.trace_begin()
+    r = api.lawcat_layer_fwd(p, *[dv[n] for n in NAMES], dv.get("cache_q"), dv.get("cache_k"), dv.get("S0"), dv.get("z0"),
+                             dev_status=status)
+    kernels = api.trace_end()
+    assert any(k.startswith("layer_tc") for k in kernels), kernels
+    assert int(status.item()) == 0
+    ref = O.layer_fwd(O.OracleParams(B, T, H, Hkv, d, d, conv_k=K, gate_tau=tau, gate_dim=s.gate_dim, normalize=norm,
+                                     eps=eps),
+                      *[x[n] for n in NAMES], x.get("cache_q"), x.get("cache_k"), x.get("S0"), x.get("z0"))
+    o = r["o"].float().cpu().numpy()
+    assert np.isfinite(o).all()
+    _, e_o = err_bf16(o, ref["o"])
+    assert e_o <= 1e-2, f"o: {e_o:.3e}"
+    rms = max(float(np.sqrt((ref["S_T"] ** 2).mean())), 1e-30)
+    e_S = float(np.abs(r["S_T"].cpu().numpy() - ref["S_T"]).max()) / rms
+    tol_S = 2e-2 if (tau == 1.0 and s.gate_dim == 1) else 1e-2
+    assert e_S <= tol_S, f"S_T: {e_S:.3e} > {tol_S}"
