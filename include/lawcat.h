@@ -155,6 +155,12 @@ int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, c
  *   cache_q_out [B,conv_k-1,H*d_k], cache_k_out [B,conv_k-1,H_kv*d_k] = the last conv_k-1 raw tokens seen
  *   (taken from the input caches when T < conv_k-1); S_T, z_T = the state after the last token. All nullable.
  * The *_out buffers must not alias the *_in buffers.
+ * bf16 storage with d_k = d_v in {64, 128}, the softmax feature map, conv_k <= 4 and chunk in {0, 64} run on the
+ * chunkwise tensor-core kernel (chunks of 64 tokens, 16-bit operands, fp32 accumulation: results within the bf16
+ * tolerance of the exact recurrence); chunk = 1 selects the exact fp32 recurrence for any supported shape.
+ * Asynchronous conditions arrive through dev_status (largest code wins): LAWCAT_ERR_NUMERIC, a decay exponent within
+ * half a chunk left the range +-120 and was clamped; LAWCAT_ERR_TIMEOUT, a bounded device-side wait ran out (the kernel
+ * has released its resources and returned; the outputs are undefined).
  */
 int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const void* v, const void* gate,
                      const void* w_q, const void* w_k, const void* W, const void* cache_q_in,
