@@ -160,6 +160,22 @@ def test_without_normalization(api, d):
     check(r["S_T"], ref["S_T"], "bf16", "S_T", f32_store=True)
 
 
+def test_exponent_clamp_is_reported(api):
+    """Gate logits so negative that the decay exponents within half a chunk leave +-120: the kernel clamps them, says so
+    through dev_status (LAWCAT_ERR_NUMERIC = 6) and still returns finite numbers; moderate logits report nothing."""
+    import torch
+    s = shape(1, 128, 2, 1, 55, gate_tau=1.0)
+    x = I.make(s, NAMES)
+    for scale, want in ((1.0, 0), (60.0, 6)):
+        g = I.round_to_bf16(-np.abs(x["gate"]) * np.float32(scale))
+        d = {n: api.to_device(g if n == "gate" else v, s.dtype) for n, v in x.items()}
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        r = api.lawcat_layer_fwd(P(api, s), *[d[n] for n in NAMES], dev_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == want
+        assert torch.isfinite(r["o"].float()).all() and torch.isfinite(r["S_T"]).all()
+
+
 def test_agrees_with_exact_path_and_split_calls(api):
     """Tensor-core path vs the CUDA-core recurrent path (chunk = 1) on the same device inputs, and one call vs two calls
     that carry the state and the conv caches."""
