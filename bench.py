@@ -191,7 +191,7 @@ def run_ours(args):
     x = I.make(s, LAYER_NAMES)
     d = {n: api.to_device(x[n], s.dtype, dev) for n in LAYER_NAMES}
     p = api.params(s.B, s.T, s.H, s.H_kv, s.d_k, s.d_v, conv_k=s.conv_k, gate_dim=s.gate_dim, dtype=s.dtype,
-                   gate_tau=s.gate_tau)
+                   gate_tau=s.gate_tau, chunk=args.chunk)
     o = torch.empty(s.B, s.T, s.H, s.d_v, dtype=api.torch_dtype(p), device=dev)
     nws = api.workspace_bytes(p, api.OP_LAYER_FWD)
     ws = torch.empty(max(nws, 16), dtype=torch.uint8, device=dev)
@@ -299,7 +299,7 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic (seeded)",
             "config": {"workload": s.name, "B": s.B, "T": s.T, "H": s.H, "H_kv": s.H_kv, "d_k": s.d_k, "d_v": s.d_v,
-                       "conv_k": s.conv_k, "gate_dim": s.gd, "gate_tau": s.gate_tau, "replicas": world,
+                       "conv_k": s.conv_k, "gate_dim": s.gd, "gate_tau": s.gate_tau, "chunk": args.chunk, "replicas": world,
                        "l2": "inputs larger than L2 (no flush)" if alg_bytes_per_token(s) * tokens > 126e6
                        else "inputs fit in L2"},
             "clocks": clocks, "e2e": e2e, "e2e_matches_device_path": same, "gpu_launches": launches,
@@ -316,6 +316,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3"])
     ap.add_argument("--gate-dim", type=int, default=0, help="override the gate width (1 = one decay per head)")
+    ap.add_argument("--chunk", type=int, default=0, choices=[0, 1, 64],
+                    help="0: the library chooses (tensor-core kernel where it applies); 1: the exact recurrent path")
     ap.add_argument("--cpu-tokens", type=int, default=16384, help="tokens of the workload the CPU oracle is timed on")
     ap.add_argument("--ref-tokens", type=int, default=2048, help="tokens per step of the reference arm")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
