@@ -10,9 +10,10 @@
  *   oracle_mix_phi       identity pass-through, softmax rows sum to 1, library matmul               (pinned)
  *   oracle_gla_fwd       quadratic form of Eq. 8 with J as an explicit running product, zero-decay
  *                        reduction to Eq. 2, alpha = 0 reduction to o_t = v_t, convex-combination
- *                        bounds, causality, split-call state hand-off                               (pinned)
- *   oracle_gla_bwd       central finite differences of oracle_gla_fwd, reverse-cumsum gate identity,
- *                        value-shift identity                                                       (pinned)
+ *                        bounds, causality, split-call state hand-off; eps against the explicit
+ *                        denominator of Eq. 8; S_T, z_T against the explicit sum of Eq. 7           (pinned)
+ *   oracle_gla_bwd       central finite differences of oracle_gla_fwd (eps = 0 and eps = 0.3),
+ *                        reverse-cumsum gate identity, value-shift identity                         (pinned)
  *   oracle_conv_bwd      central finite differences of oracle_conv + oracle_mix_phi                 (pinned)
  *   choice of phi, gate_tau, eps: the paper does not fix them -> parameters; parity unpinned by the paper.
  *

@@ -140,6 +140,55 @@ def test_recurrence_equals_quadratic_form(gate_dim, T):
     np.testing.assert_allclose(r0["o"][0, :, 1], o0, rtol=1e-11, atol=1e-13)
 
 
+@pytest.mark.parametrize("gate_dim", [0, 1])
+def test_eps_sits_in_the_denominator_of_eq8(gate_dim):
+    # Eq. 8 with eps: o_t = (sum_i w_ti v_i) / (sum_i w_ti + eps), w_ti = qdot_t . (J_{i,t} kdot_i); the weights are
+    # built here from the explicit running product of the gates, eps is added to the explicit denominator only
+    T, H, dk, dv, eps = 14, 2, 5, 4, 0.37
+    p = O.OracleParams(1, T, H, H, dk, dv, gate_dim=gate_dim, gate_tau=2.0, eps=eps)
+    qd, kd = np.abs(rnd(1, T, H, dk)), np.abs(rnd(1, T, H, dk))
+    v, a = rnd(1, T, H, dv), 2 * rnd(1, T, H, p.gd)
+    r = O.gla_fwd(p, qd, kd, v, a)
+    alpha = np.broadcast_to(np.exp(logsigmoid(a) / 2.0), (1, T, H, dk))
+    for h in range(H):
+        num, den = quadratic_form(qd[0, :, h], kd[0, :, h], v[0, :, h], alpha[0, :, h], normalize=False)
+        np.testing.assert_allclose(r["o"][0, :, h], num / (den + eps)[:, None], rtol=1e-11, atol=1e-13)
+        np.testing.assert_allclose(r["den"][0, :, h], den + eps, rtol=1e-11)
+    # a wrong place for eps (added to the numerator, or scaled by anything) would show against the eps = 0 result too
+    r0 = O.gla_fwd(O.OracleParams(1, T, H, H, dk, dv, gate_dim=gate_dim, gate_tau=2.0), qd, kd, v, a)
+    np.testing.assert_allclose(r["o"] * r["den"][..., None], r0["o"] * r0["den"][..., None], rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(r["den"] - r0["den"], eps, rtol=1e-10)
+
+
+@pytest.mark.parametrize("gate_dim,with_state", [(0, False), (1, True), (0, True)])
+def test_final_state_equals_eq7_explicit_sum(gate_dim, with_state):
+    # Eq. 7: S_T = J_{0,T} S_0 + sum_i J_{i,T} (kdot_i^T v_i), z_T likewise with 1 for v_i, where J_{i,T} is the
+    # explicit product of the gates of tokens i+1..T (Eq. 6); a given initial state is decayed by every gate
+    T, H, dk, dv = 11, 2, 4, 3
+    p = O.OracleParams(1, T, H, H, dk, dv, gate_dim=gate_dim, gate_tau=2.0)
+    qd, kd = np.abs(rnd(1, T, H, dk)), np.abs(rnd(1, T, H, dk))
+    v, a = rnd(1, T, H, dv), 2 * rnd(1, T, H, p.gd)
+    S0 = rnd(1, H, dk, dv) if with_state else None
+    z0 = np.abs(rnd(1, H, dk)) if with_state else None
+    r = O.gla_fwd(p, qd, kd, v, a, S0, z0)
+    alpha = np.broadcast_to(np.exp(logsigmoid(a) / 2.0), (1, T, H, dk))
+    for h in range(H):
+        S, z = np.zeros((dk, dv)), np.zeros(dk)
+        for i in range(-1, T):  # i = -1 stands for the given initial state
+            J = np.ones(dk)
+            for zz in range(i + 1, T):
+                J = J * alpha[0, zz, h]
+            if i < 0:
+                if with_state:
+                    S += J[:, None] * S0[0, h]
+                    z += J * z0[0, h]
+            else:
+                S += J[:, None] * np.outer(kd[0, i, h], v[0, i, h])
+                z += J * kd[0, i, h]
+        np.testing.assert_allclose(r["S_T"][0, h], S, rtol=1e-11, atol=1e-13)
+        np.testing.assert_allclose(r["z_T"][0, h], z, rtol=1e-11, atol=1e-13)
+
+
 def test_zero_decay_is_kernel_linear_attention():
     # all gates 1 -> Eq. 2 by direct double sum
     T, dk, dv = 19, 5, 4
@@ -278,6 +327,23 @@ def test_gla_bwd_finite_differences(gate_dim, gate_mode, normalize, with_state):
     f = lambda: O.gla_fwd(p, qd, kd, v, a, S0, z0)["o"]
     for name, x in (("d_qdot", qd), ("d_kdot", kd), ("dv", v), ("dgate", a)):
         np.testing.assert_allclose(g[name], _fd(f, x, dO), rtol=2e-6, atol=1e-8, err_msg=name)
+
+
+@pytest.mark.parametrize("gate_dim", [0, 1])
+def test_gla_bwd_finite_differences_with_eps(gate_dim):
+    # eps = 0.3 is of the size of the denominators here: a misplaced eps in the backward (in do' or in the
+    # -(dO . o) / d term) changes every gradient by tens of percent
+    B, T, H, Hkv, dk, dv = 1, 6, 2, 1, 4, 3
+    p = O.OracleParams(B, T, H, Hkv, dk, dv, gate_dim=gate_dim, gate_tau=2.0, eps=0.3)
+    qd, kd = np.abs(rnd(B, T, H, dk)) * 0.3 + 0.05, np.abs(rnd(B, T, H, dk)) * 0.3 + 0.05
+    v, dO, a = rnd(B, T, Hkv, dv), rnd(B, T, H, dv), rnd(B, T, H, p.gd)
+    S0, z0 = np.abs(rnd(B, H, dk, dv)) * 0.2, np.abs(rnd(B, H, dk)) * 0.2
+    g = O.gla_bwd(p, qd, kd, v, a, dO, S0, z0)
+    f = lambda: O.gla_fwd(p, qd, kd, v, a, S0, z0)["o"]
+    for name, x in (("d_qdot", qd), ("d_kdot", kd), ("dv", v), ("dgate", a)):
+        np.testing.assert_allclose(g[name], _fd(f, x, dO), rtol=2e-6, atol=1e-8, err_msg=name)
+    g0 = O.gla_bwd(O.OracleParams(B, T, H, Hkv, dk, dv, gate_dim=gate_dim, gate_tau=2.0), qd, kd, v, a, dO, S0, z0)
+    assert np.abs(g["d_qdot"] - g0["d_qdot"]).max() > 0.05 * np.abs(g0["d_qdot"]).max()  # eps matters at this size
 
 
 def test_gate_gradient_reverse_cumsum_identity():
