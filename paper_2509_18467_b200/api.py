@@ -197,8 +197,9 @@ def lawcat_layer_fwd(p: Params, q, k, v, gate, w_q, w_k, W, cache_q=None, cache_
     dt, dev = torch_dtype(p), q.device
     if o is None:
         o = torch.empty(p.B, p.T, p.H, p.d_v, dtype=dt, device=dev)
-    S_T = torch.empty(p.B, p.H, p.d_k, p.d_v, dtype=torch.float32, device=dev) if want_state else None
-    z_T = torch.empty(p.B, p.H, p.d_k, dtype=torch.float32, device=dev) if want_state else None
+    # want_state: True / False, or "S" / "z" for one of the two state outputs alone (each is optional on its own)
+    S_T = torch.empty(p.B, p.H, p.d_k, p.d_v, dtype=torch.float32, device=dev) if want_state in (True, "S") else None
+    z_T = torch.empty(p.B, p.H, p.d_k, dtype=torch.float32, device=dev) if want_state in (True, "z") else None
     cq = torch.empty(p.B, p.conv_k - 1, p.H * p.d_k, dtype=dt, device=dev) if want_cache else None
     ck = torch.empty(p.B, p.conv_k - 1, p.H_kv * p.d_k, dtype=dt, device=dev) if want_cache else None
     ws, nb = _ws(p, OP_LAYER_FWD, ws, dev)

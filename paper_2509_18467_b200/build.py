@@ -16,9 +16,9 @@ OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "liblawcat.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 
-FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--use_fast_math=false",
+# (no fast-math: the exact path relies on the precise division, exp and log of the default settings)
+FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
-FLAGS.remove("--use_fast_math=false")  # precise math is the default; the flag is listed above only as a reminder
 
 
 def sources():

@@ -1,4 +1,6 @@
 // Host side of the chunkwise tensor-core layer forward: tensor maps, segment split, launches.
+#include <mutex>
+
 #include "layer_tc_kernel.cuh"
 
 namespace lawcat {
@@ -68,40 +70,67 @@ __global__ void segment_scan_kernel(const float* __restrict__ S0, const float* _
 
 }  // namespace tc
 
-// Segments per sequence: enough thread blocks to fill the SMs (one block per SM), but at least MIN_SEG_CHUNKS chunks per
-// segment (a thread block spends about three chunk times on its set-up and on filling its pipeline).
-int layer_tc_segments(const lawcat_params& p) {
-  constexpr int MIN_SEG_CHUNKS = 4;
-  const int chunks = (p.T + tc::C - 1) / tc::C;
-  int n = 148 / (p.B * p.H);
-  if (n > chunks / MIN_SEG_CHUNKS) n = chunks / MIN_SEG_CHUNKS;
-  return n < 1 ? 1 : n;
+// Number of SMs of the current device (cached per device; 148 on a B200).
+static int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
 }
 
-// Pieces per segment in the state-only pre-pass: its thread blocks are independent, so cutting the segments finer lets
-// them fill the SMs in whole waves. Picks the split with the fewest chunks per SM (a small charge per extra piece).
-static int layer_tc_pieces(const lawcat_params& p, int nseg) {
+// How a sequence is cut: nseg segments of seg_len tokens (a multiple of the chunk; every segment holds tokens), and the
+// pieces per segment of the state-only pre-pass.
+struct TcPlan {
+  int nseg, seg_len, nsub;
+};
+
+// Segments per sequence: enough thread blocks to fill the SMs (one block per SM), but at least MIN_SEG_CHUNKS chunks per
+// segment (a thread block spends about three chunk times on its set-up and on filling its pipeline). Pieces per segment
+// in the state-only pre-pass: its thread blocks are independent, so cutting the segments finer lets them fill the SMs in
+// whole waves; the split with the fewest chunks per SM wins (a small charge per extra piece).
+static TcPlan layer_tc_plan(const lawcat_params& p) {
+  constexpr int MIN_SEG_CHUNKS = 4;
+  const int sms = sm_count();
   const int chunks = (p.T + tc::C - 1) / tc::C;
-  const int cps = (chunks + nseg - 1) / nseg;
+  int n = sms / (p.B * p.H);
+  if (n > chunks / MIN_SEG_CHUNKS) n = chunks / MIN_SEG_CHUNKS;
+  if (n < 1) n = 1;
+  TcPlan pl;
+  pl.seg_len = ((chunks + n - 1) / n) * tc::C;
+  pl.nseg = (p.T + pl.seg_len - 1) / pl.seg_len;  // (rounding the length up may leave fewer segments than asked for)
+  if (pl.nseg < 1) pl.nseg = 1;
+  const int cps = pl.seg_len / tc::C;
   int best = 1, best_cost = 1 << 30;
   for (int ns = 1; ns <= 8 && ns * 4 <= cps; ++ns) {
-    const int ctas = p.B * p.H * (nseg - 1) * ns;
-    const int cost = ((ctas + 147) / 148) * ((cps + ns - 1) / ns + 2);
+    const int ctas = p.B * p.H * (pl.nseg - 1) * ns;
+    const int cost = ((ctas + sms - 1) / sms) * ((cps + ns - 1) / ns + 2);
     if (cost < best_cost) { best_cost = cost; best = ns; }
   }
-  return best;
+  pl.nsub = best;
+  return pl;
 }
 
+int layer_tc_segments(const lawcat_params& p) { return layer_tc_plan(p).nseg; }
+
 size_t layer_tc_workspace_bytes(const lawcat_params& p) {
-  const int nseg = layer_tc_segments(p);
-  if (nseg == 1) return 0;
-  const size_t pieces = (size_t)nseg * layer_tc_pieces(p, nseg);
-  return sizeof(float) * (size_t)p.B * p.H * ((pieces + nseg) * ((size_t)p.d_k * p.d_k + p.d_k) + pieces * p.d_k);
+  const TcPlan pl = layer_tc_plan(p);
+  if (pl.nseg == 1) return 0;
+  const size_t pieces = (size_t)pl.nseg * pl.nsub;
+  return sizeof(float) * (size_t)p.B * p.H * ((pieces + pl.nseg) * ((size_t)p.d_k * p.d_k + p.d_k) + pieces * p.d_k);
 }
 
 bool layer_tc_supported(const lawcat_params& p) {
+  // One decay per head under the plain sigmoid gate (tau < 2) concentrates the state on the last one or two tokens; the
+  // 2^-11 rounding of the kernel's fp16 operands then exceeds the accuracy bound on the largest state entries, so that
+  // combination goes to the exact path.
+  const bool sharp_scalar_gate = p.gate_dim == 1 && p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 2.f;
   return p.dtype == LAWCAT_BF16 && (p.d_k == tc::D || p.d_k == 64) && p.d_v == p.d_k &&
-         (p.gate_dim == p.d_k || p.gate_dim == 1) &&
+         (p.gate_dim == p.d_k || p.gate_dim == 1) && !sharp_scalar_gate &&
          p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
          (p.chunk == 0 || p.chunk == tc::C);
 }
@@ -126,15 +155,29 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   a.dev_status = c.dev_status;
   a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k;
   a.gate_mode = p.gate_mode; a.normalize = p.normalize; a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps;
-  const int nseg = layer_tc_segments(p);
+  const TcPlan pl = layer_tc_plan(p);
+  const int nseg = pl.nseg;
   a.nseg = nseg;
-  a.seg_len = ((p.T + nseg - 1) / nseg + C - 1) / C * C;
+  a.seg_len = pl.seg_len;
   const bool narrow = dh == 64;
   auto* const k_layer = narrow ? layer_tc_kernel<0, true> : layer_tc_kernel<0, false>;
   auto* const k_state = narrow ? layer_tc_kernel<1, true> : layer_tc_kernel<1, false>;
-  if (cudaFuncSetAttribute(k_layer, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
-      cudaFuncSetAttribute(k_state, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess)
-    return LAWCAT_ERR_CUDA;
+  {
+    // the kernels' shared-memory limit is raised once per device
+    static std::mutex mu;
+    static bool done[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LAWCAT_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!done[dev]) {
+      if (cudaFuncSetAttribute(layer_tc_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess)
+        return LAWCAT_ERR_CUDA;
+      done[dev] = true;
+    }
+  }
   const int BH = p.B * p.H;
   if (nseg == 1) {
     a.S0 = S0; a.z0 = z0; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
@@ -147,7 +190,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   // Several segments per sequence: (1) every segment but the last computes its end state from a zero state, and the
   // total decay of the segment; (2) a scan over the segments turns these into the state at each segment's start;
   // (3) the layer runs on all segments at once, each from its start state.
-  const int nsub = layer_tc_pieces(p, nseg);
+  const int nsub = pl.nsub;
   const size_t nS = (size_t)BH * nseg * dh * dh, nz = (size_t)BH * nseg * dh;
   float* loc_S = (float*)ws;              // [BH, nseg, nsub, D, D]
   float* loc_z = loc_S + nS * nsub;       // [BH, nseg, nsub, D]

@@ -1019,7 +1019,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_after_sync();
       const int c = r128;
       if (a.dtot != nullptr && ch == 0 && c < dh) a.dtot[seg_idx * dh + c] = dsum;
-      if (a.S_T != nullptr && (a.seg_out || seg == a.nseg - 1)) {
+      const bool last = a.seg_out || seg == a.nseg - 1;  // (each of the two outputs is optional on its own)
+      if (a.S_T != nullptr && last) {
         float s[32];
 #pragma unroll 1
         for (int b2 = 0; b2 < 2; ++b2) {
@@ -1032,11 +1033,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               *reinterpret_cast<float4*>(a.S_T + (out_idx * dh + c) * dh + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
           }
         }
-        if (ch == 1 && a.z_T) {
-          const float z = tmem_ld1(lane_base + COL_SZ);
-          tmem_wait_ld();
-          if (c < dh) a.z_T[out_idx * dh + c] = z;
-        }
+      }
+      if (a.z_T != nullptr && last && ch == 1) {
+        const float z = tmem_ld1(lane_base + COL_SZ);
+        tmem_wait_ld();
+        if (c < dh) a.z_T[out_idx * dh + c] = z;
       }
     }
   }

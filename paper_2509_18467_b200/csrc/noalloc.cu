@@ -46,6 +46,13 @@ int lawcat_layer_fwd_noalloc(const lawcat_params* p, const void* q, const void* 
   const int bad = validate_params(p, true);  // invalid argument vs unsupported shape; nothing is enqueued
   if (bad) return bad;
   // the exact path's scratch: two fp32 tensors [B,T,H,d_k]
+  // (the limit is tested by division, factor by factor: the element count itself could wrap around in 64 bits)
+  const size_t max_elems = kScratchBytes / (2 * sizeof(float));
+  size_t room = max_elems;
+  for (const size_t f : {(size_t)p->H, (size_t)p->d_k, (size_t)p->B, (size_t)p->T}) {
+    if (f != 0 && room / f == 0) return LAWCAT_ERR_TOO_LARGE;
+    if (f != 0) room /= f;
+  }
   const size_t half = align_up(sizeof(float) * (size_t)p->B * (size_t)p->T * p->H * p->d_k, 256);
   if (2 * half > kScratchBytes) return LAWCAT_ERR_TOO_LARGE;
   const void* const req[] = {w_q, w_k, W};

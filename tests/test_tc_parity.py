@@ -37,7 +37,7 @@ def P(api, s, **kw):
                       gate_tau=s.gate_tau, **kw)
 
 
-def run_case(api, s, with_state, **pkw):
+def run_case(api, s, with_state, expect_tc=True, **pkw):
     import torch
     extra = (["S0", "z0"] + (["cache_q", "cache_k"] if s.conv_k > 1 else [])) if with_state else []
     x = I.make(s, NAMES + extra)
@@ -48,7 +48,7 @@ def run_case(api, s, with_state, **pkw):
     r = api.lawcat_layer_fwd(P(api, s, **pkw), *[d[n] for n in NAMES], d.get("cache_q"), d.get("cache_k"),
                              d.get("S0"), d.get("z0"), dev_status=status)
     kernels = api.trace_end()
-    assert any(k.startswith("layer_tc") for k in kernels), f"tensor-core kernel not used: {kernels}"
+    assert any(k.startswith("layer_tc") for k in kernels) == expect_tc, f"unexpected kernels: {kernels}"
     assert api.launch_count() > n0
     assert int(status.item()) == 0
     ref = O.layer_fwd(oracle_params(s), *[x[n] for n in NAMES], x.get("cache_q"), x.get("cache_k"), x.get("S0"),
@@ -97,7 +97,10 @@ def test_one_decay_per_head(api, T, with_state):
 
 
 def test_one_decay_per_head_sharp_gate(api):
-    run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=1.0), False)
+    """One plain-sigmoid decay per head (gate_dim = 1, tau = 1): the library serves it with the exact recurrence, because
+    the state then sits on the last one or two tokens; tau = 2 is back on the tensor-core kernel."""
+    run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=1.0), False, expect_tc=False)
+    run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=2.0), True)
 
 
 def shape64(B, T, H, Hkv, cid, **kw):
@@ -121,6 +124,24 @@ def test_long_sequence_many_segments(api):
     """Long enough for the sequence to be split into segments whose states are handed across thread blocks."""
     e, _, _ = run_case(api, shape(1, 8192 + 77, 2, 1, 46), True)
     print(f"T=8269 error {e:.3e}")
+
+
+@pytest.mark.parametrize("chunk", [0, 1])
+@pytest.mark.parametrize("which", ["S", "z"])
+def test_state_outputs_are_optional_one_by_one(api, chunk, which):
+    """S_T without z_T and z_T without S_T, on the tensor-core kernel (chunk = 0) and on the exact path (chunk = 1)."""
+    s = shape(1, 150, 2, 1, 56)
+    x = I.make(s, NAMES)
+    d = {n: api.to_device(v, s.dtype) for n, v in x.items()}
+    r = api.lawcat_layer_fwd(P(api, s, chunk=chunk), *[d[n] for n in NAMES], want_state=which)
+    ref = O.layer_fwd(oracle_params(s), *[x[n] for n in NAMES])
+    check(r["o"], ref["o"], "bf16", "o")
+    if which == "S":
+        assert r["z_T"] is None
+        check(r["S_T"], ref["S_T"], "bf16", "S_T", f32_store=True)
+    else:
+        assert r["S_T"] is None
+        check(r["z_T"], ref["z_T"], "bf16", "z_T", f32_store=True)
 
 
 def test_log_decay_gate_mode(api):

@@ -1,10 +1,9 @@
 """Randomized parity of the tensor-core layer forward: 36 seeded draws of (head width, batch, length, head grouping,
 conv width, gate sharpness, gate width, carried state, normalizer on/off, eps) against the fp64 oracle, through the C ABI.
 
-Tolerance: 1e-2 of the RMS on every tensor, with one documented exception: with the plain sigmoid gate (tau = 1) and one
-decay per head the state is concentrated on the last few tokens, max|S_T| / rms(S_T) reaches 15, and the 2^-11 relative
-rounding of the fp16 operands (conv output into the mix, decayed key features into the state update) shows as up to
-1.5e-2 of the RMS in the strict max / RMS metric; the bound there is 2e-2. The outputs o meet 1e-2 everywhere."""
+Tolerance: 1e-2 of the RMS on every tensor (outputs and the final state). One decay per head under the plain sigmoid gate
+(gate_dim = 1, tau < 2) is served by the exact recurrence (see the header of lawcat_layer_fwd); every other draw must run on
+the tensor-core kernel."""
 import random
 
 import numpy as np
@@ -47,7 +46,8 @@ def test_random_configuration(case):
     r = api.lawcat_layer_fwd(p, *[dv[n] for n in NAMES], dv.get("cache_q"), dv.get("cache_k"), dv.get("S0"), dv.get("z0"),
                              dev_status=status)
     kernels = api.trace_end()
-    assert any(k.startswith("layer_tc") for k in kernels), kernels
+    exact = s.gate_dim == 1 and tau < 2.0
+    assert any(k.startswith("layer_tc") for k in kernels) != exact, kernels
     assert int(status.item()) == 0
     ref = O.layer_fwd(O.OracleParams(B, T, H, Hkv, d, d, conv_k=K, gate_tau=tau, gate_dim=s.gate_dim, normalize=norm,
                                      eps=eps),
@@ -58,5 +58,7 @@ def test_random_configuration(case):
     assert e_o <= 1e-2, f"o: {e_o:.3e}"
     rms = max(float(np.sqrt((ref["S_T"] ** 2).mean())), 1e-30)
     e_S = float(np.abs(r["S_T"].cpu().numpy() - ref["S_T"]).max()) / rms
-    tol_S = 2e-2 if (tau == 1.0 and s.gate_dim == 1) else 1e-2
-    assert e_S <= tol_S, f"S_T: {e_S:.3e} > {tol_S}"
+    assert e_S <= 1e-2, f"S_T: {e_S:.3e}"
+    rz = max(float(np.sqrt((ref["z_T"] ** 2).mean())), 1e-30)
+    e_z = float(np.abs(r["z_T"].cpu().numpy() - ref["z_T"]).max()) / rz
+    assert e_z <= 1e-2, f"z_T: {e_z:.3e}"
