@@ -157,11 +157,12 @@ int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, c
  * The *_out buffers must not alias the *_in buffers.
  * bf16 storage with d_k = d_v in {64, 128}, the softmax feature map, conv_k <= 4 and chunk in {0, 64} run on the
  * chunkwise tensor-core kernel (chunks of 64 tokens, 16-bit operands, fp32 accumulation: results within the bf16
- * tolerance of the exact recurrence); chunk = 1 selects the exact fp32 recurrence for any supported shape. One
- * combination inside that set also takes the exact recurrence: gate_dim = 1 with LAWCAT_GATE_LOGITS and gate_tau < 2
- * (one plain-sigmoid decay per head leaves the state on the last one or two tokens, where 16-bit operands miss the
- * tolerance on the largest entries of S_T). With LAWCAT_GATE_LOGDECAY the caller chooses the decays: when they are
- * that sharp (a state that halves or more at every token) and S_T is carried on, pass chunk = 1.
+ * tolerance of the exact recurrence); chunk = 1 selects the exact fp32 recurrence for any supported shape. Two
+ * combinations inside that set also take the exact recurrence, both under the plain sigmoid gate (LAWCAT_GATE_LOGITS
+ * with gate_tau < 2, where a token's decay is about one half and the chunk's factors need 8-bit-mantissa operands):
+ * gate_dim = 1 (the state sits on the last one or two tokens and its largest entries miss the tolerance) and
+ * normalize = 0 (no denominator to cancel the rounding of the weights). With LAWCAT_GATE_LOGDECAY the caller chooses
+ * the decays: when they are that sharp (a state that halves or more at every token), pass chunk = 1 for these two forms.
  * Asynchronous conditions arrive through dev_status (largest code wins): LAWCAT_ERR_NUMERIC, a decay exponent within
  * half a chunk left the range +-120 and was clamped; LAWCAT_ERR_TIMEOUT, a bounded device-side wait ran out (the kernel
  * has released its resources and returned; the outputs are undefined).

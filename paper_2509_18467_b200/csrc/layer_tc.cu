@@ -125,12 +125,15 @@ size_t layer_tc_workspace_bytes(const lawcat_params& p) {
 }
 
 bool layer_tc_supported(const lawcat_params& p) {
-  // One decay per head under the plain sigmoid gate (tau < 2) concentrates the state on the last one or two tokens; the
-  // 2^-11 rounding of the kernel's fp16 operands then exceeds the accuracy bound on the largest state entries, so that
-  // combination goes to the exact path.
-  const bool sharp_scalar_gate = p.gate_dim == 1 && p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 2.f;
+  // Under the plain sigmoid gate (tau < 2) a token's decay is about one half, so the exponents of the in-chunk
+  // factorization leave the fp16 range and the operands fall back to bf16 (8 significant bits). The normalized form with
+  // one decay per key channel stays within the accuracy bound there (numerator and denominator carry the same weights);
+  // one decay per head (the state sits on the last one or two tokens) and the numerator-only form do not, so those two
+  // go to the exact path.
+  const bool sharp = p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 2.f;
+  const bool sharp_unsupported = sharp && (p.gate_dim == 1 || !p.normalize);
   return p.dtype == LAWCAT_BF16 && (p.d_k == tc::D || p.d_k == 64) && p.d_v == p.d_k &&
-         (p.gate_dim == p.d_k || p.gate_dim == 1) && !sharp_scalar_gate &&
+         (p.gate_dim == p.d_k || p.gate_dim == 1) && !sharp_unsupported &&
          p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
          (p.chunk == 0 || p.chunk == tc::C);
 }

@@ -49,17 +49,19 @@ constexpr int THREADS = 18 * 32;
 
 // shared memory map (byte offsets from a 1024-byte aligned base)
 constexpr uint32_t OFF_W = 0;                     // W_h^T fp16, K-major, 2 slabs x [128 x 128 B]
-constexpr uint32_t OFF_SBF = OFF_W + 32768;       // 2^b_mid * S, 16 bit, MN-major, 2 slabs x [128 x 128 B]
-constexpr uint32_t OFF_AU = OFF_SBF + 32768;      // raw q|k tile, then conv output in place: A of MMA 1, 2 slabs
+constexpr uint32_t OFF_SBF = OFF_W + 32768;       // 2^b_mid * [S | z], 16 bit, MN-major B operand of the read-out product,
+                                                  // unswizzled 8x8 core matrices: block of 8 columns nb at nb * 2048,
+                                                  // key channel c at (c / 8) * 128 + (c % 8) * 16 inside a block; the
+                                                  // blocks of S are followed by two blocks whose first column is z
+constexpr uint32_t OFF_AU = OFF_SBF + 36864;      // raw q|k tile, then conv output in place: A of MMA 1, 2 slabs
 constexpr uint32_t OFF_QK = OFF_AU + 32768;       // qs (rows 0-63) | ks (rows 64-127), 16 bit, K-major, 2 slabs
 constexpr uint32_t OFF_X = OFF_QK + 32768;        // exponents x fp32 [64 x 128], XOR-swizzled 16-byte chunks
 constexpr uint32_t OFF_KH = OFF_X + 32768;        // kh fp16, MN-major A of the state update, 2 slabs x [64 tokens x 128 B]
 constexpr uint32_t OFF_G = OFF_KH + 16384;        // gate logits bf16, 2 slabs x [64 x 128 B]
-constexpr uint32_t OFF_V = OFF_G + 16384;         // v bf16, then fp16 in place, MN-major B, 2 slabs x [64 x 128 B]
-constexpr uint32_t OFF_PH = OFF_V + 16384;        // masked scores fp16, K-major, [64 x 128 B]; an M=128 MMA also reads
-                                                  // (and ignores) the 8 KB that follow
-constexpr uint32_t OFF_SZ = OFF_PH + 8192;        // 2^b_mid * z as a [128 x 16] operand (column 0 is z)
-constexpr uint32_t OFF_ONES = OFF_SZ + 4096;      // [64 x 16] fp16 operand whose column 0 is 1 (the "1" of [v|1])
+constexpr uint32_t OFF_PH = OFF_G + 16384;        // masked scores fp16, K-major, [64 x 128 B]; an M=128 MMA also reads
+                                                  // (and ignores) the 8 KB that follow (the first half of the v tile)
+constexpr uint32_t OFF_V = OFF_PH + 8192;         // v bf16, then fp16 in place, MN-major B, 2 slabs x [64 x 128 B]
+constexpr uint32_t OFF_ONES = OFF_V + 16384;      // [64 x 16] fp16 operand whose column 0 is 1 (the "1" of [v|1])
 constexpr uint32_t OFF_HALO = OFF_ONES + 2048;    // [2 streams][3 rows][16 x 16 B]: raw rows in front of the next chunk
 constexpr uint32_t OFF_VEC = OFF_HALO + 1536;     // per parity: bm[128], ft[128], e63[128] fp32 (2 x 1536 B)
 constexpr uint32_t OFF_BAR = OFF_VEC + 3072;      // mbarriers (8 B each) and scalars
@@ -73,13 +75,15 @@ constexpr float RMAX_F16 = 8.f;     // largest |x| for which the operands are ke
 // tensor memory map (32-bit columns)
 constexpr uint32_t COL_Y = 0;      // [128 x 128] mix output
 constexpr uint32_t COL_S = 128;    // [128 x 128] state S
-constexpr uint32_t COL_O = 256;    // [128 x 128] numerator (lanes 0-63 meaningful)
-constexpr uint32_t COL_P = 384;    // [128 x 64] scores (lanes 0-63 meaningful)
-constexpr uint32_t COL_SZ = 448;   // [128 x 16] column 0: normalizer state z
-constexpr uint32_t COL_OZ = 464;   // [128 x 16] column 0: denominator
+constexpr uint32_t COL_O = 256;    // [128 x (128 + 16)] numerator, directly followed by the state's part of the denominator
+                                   // (column COL_O + head width); lanes 0-63 meaningful
+constexpr uint32_t COL_P = 400;    // [128 x 64] scores (lanes 0-63 meaningful)
+constexpr uint32_t COL_SZ = 464;   // [128 x 16] column 0: normalizer state z
 constexpr uint32_t COL_MAIL = 480; // spare columns used as per-row mailboxes between threads of one TMEM lane:
                                    // +2, +3: row max / softmax sum of the two column halves; +4 p + half (p = chunk
-                                   // parity): the dropped query normalizer (softmax sum) of that half, row warps -> output pass
+                                   // parity): the dropped query normalizer (softmax sum) of that half, row warps -> output
+                                   // pass; +8 + 2 p + half: the chunk's own part of the denominator (row sum of the masked
+                                   // scores of that half), mask pass -> output pass
 constexpr uint32_t TMEM_COLS = 512;
 
 // mbarrier indices. "full": producer -> consumer, "free": consumer -> producer. Each completes once per chunk, so the
@@ -97,7 +101,8 @@ enum {
   B_X_FREE,        // row warps: exponents consumed                  -> prep (gate of the next chunk)
   B_QK_FULL,       // row warps: qs, ks, kh written                  -> MMA 2
   B_SBF_FULL,      // row warps: state operand written, S decayed    -> MMA 2
-  B_MMA2,          // MMA 2 complete: P ready, state updated, qs/ks/kh/state operand free
+  B_P,             // score product complete: P ready                -> row warps (mask)
+  B_MMA2,          // MMA 2 complete: state updated, read-out started O', qs/ks/kh/state operand free
   B_PH_FULL,       // row warps: masked scores written               -> MMA 3
   B_MMA3,          // MMA 3 complete: O' ready -> row warps; v tile free -> TMA
   B_O_FREE,        // row warps: O' consumed                         -> MMA 2 of the next chunk
@@ -295,6 +300,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     mbar_init(bar(B_X_FREE), 256);  // every row thread: it reads bm, ft and (phi threads) the exponents
     mbar_init(bar(B_QK_FULL), nphi);
     mbar_init(bar(B_SBF_FULL), 256);
+    mbar_init(bar(B_P), 1);
     mbar_init(bar(B_MMA2), 1);
     mbar_init(bar(B_PH_FULL), 128);
     mbar_init(bar(B_MMA3), 1);
@@ -329,8 +335,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // channels: its second slab is zeroed here and never written
   if (narrow)
     for (int i = tid; i < 8192 / 16; i += THREADS) reinterpret_cast<uint4*>(sg + OFF_KH + 8192)[i] = make_uint4(0u, 0u, 0u, 0u);
-  // constant "ones" operand and a zeroed z operand (unswizzled 8x8 core matrices)
-  for (int i = tid; i < (4096 + 2048) / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_SZ)[i] = 0u;
+  // constant "ones" operand and the zeroed column blocks of the state operand that carry z (unswizzled 8x8 core matrices)
+  for (int i = tid; i < 2048 / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_ONES)[i] = 0u;
+  for (int i = tid; i < 4096 / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_SBF + (dh >> 3) * 2048)[i] = 0u;
   // raw rows in front of the segment: earlier tokens, or the conv cache, or zeros (Section 4.1)
   if (tid < 96) {
     const int st = tid / 48, r = (tid % 48) / 16, oc = tid % 16;
@@ -448,8 +455,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint64_t dsc_w = smem_desc(sb + OFF_W, 16, 1024, LAYOUT_SW128);
       const uint64_t dsc_qk = smem_desc(sb + OFF_QK, 16, 1024, LAYOUT_SW128);
       const uint64_t dsc_ks = smem_desc(sb + OFF_QK + 8192, 16, 1024, LAYOUT_SW128);  // rows 64-127
-      const uint64_t dsc_s = smem_desc(sb + OFF_SBF, 16384, 1024, LAYOUT_SW128);
-      const uint64_t dsc_sz = smem_desc(sb + OFF_SZ, 128, 2048, LAYOUT_NONE);
+      const uint64_t dsc_s = smem_desc(sb + OFF_SBF, 128, 2048, LAYOUT_NONE);  // [S | z]: one operand
       const uint64_t dsc_kh = smem_desc(sb + OFF_KH, 8192, 1024, LAYOUT_SW128);
       const uint64_t dsc_v = smem_desc(sb + OFF_V, 8192, 1024, LAYOUT_SW128);
       const uint64_t dsc_one = smem_desc(sb + OFF_ONES, 128, 1024, LAYOUT_NONE);
@@ -476,35 +482,36 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       for (int n = 0; ok && n < nchunks; ++n) {
         const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
+        WAITSET(BIT(B_QK_FULL) | BIT(B_SBF_FULL) | BIT(B_VH_FULL) | (MODE == 0 && n > 0 ? BIT(B_O_FREE) : 0u),
+                PAR(B_QK_FULL, p) | PAR(B_SBF_FULL, p) | PAR(B_VH_FULL, p) | PAR(B_O_FREE, pp));
+        const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
+        const int fmt = f16 ? FMT_F16 : FMT_BF16;
+        if (MODE == 0 && lane == 0) {
+          // the scores first: their mask pass is the longest chain behind this hand-over
+          tc_fence_after_sync();
+          const uint32_t ID_P = instr_desc(128, 64, fmt, MAJOR_K, MAJOR_K);
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            if (k < ksteps) mma_f16(tmem + COL_P, adv(dsc_qk, kstep(k)), adv(dsc_ks, kstep(k)), ID_P, k > 0);
+          mma_commit(bar(B_P));
+        }
         if (n + 1 < nchunks) {
-          // the mix of the next chunk goes first: its phi pass starts reading Y while this chunk's MMA 2 executes
+          // then the mix of the next chunk: its phi pass reads Y while this chunk's read-out and state update execute
           WAITSET(BIT(B_U_FULL) | BIT(B_Y_FREE), PAR(B_U_FULL, pp) | PAR(B_Y_FREE, p));
           if (lane == 0) {
             tc_fence_after_sync();
             issue_mma1();
           }
         }
-        WAITSET(BIT(B_QK_FULL) | BIT(B_SBF_FULL) | BIT(B_VH_FULL) | (MODE == 0 && n > 0 ? BIT(B_O_FREE) : 0u),
-                PAR(B_QK_FULL, p) | PAR(B_SBF_FULL, p) | PAR(B_VH_FULL, p) | PAR(B_O_FREE, pp));
         if (lane == 0) {
-        tc_fence_after_sync();
-        if (MODE == 0) {
-          const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
-          const int fmt = f16 ? FMT_F16 : FMT_BF16;
-          const uint32_t ID_P = instr_desc(128, 64, fmt, MAJOR_K, MAJOR_K);
-          const uint32_t ID_O = instr_desc(128, NW, fmt, MAJOR_K, MAJOR_MN);
-          const uint32_t ID_OZ = instr_desc(128, 16, fmt, MAJOR_K, MAJOR_MN);
+          tc_fence_after_sync();
+          if (MODE == 0) {
+            // read-out O' | denominator = qs [2^b_mid S | 2^b_mid z] in one product per K step
+            const uint32_t ID_O = instr_desc(128, NW + 16, fmt, MAJOR_K, MAJOR_MN);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            if (k < ksteps) {
-              const uint64_t ad = adv(dsc_qk, kstep(k));
-              mma_f16(tmem + COL_P, ad, adv(dsc_ks, kstep(k)), ID_P, k > 0);
-              mma_f16(tmem + COL_O, ad, adv(dsc_s, k * (2048 >> 4)), ID_O, k > 0);
-              mma_f16(tmem + COL_OZ, ad, adv(dsc_sz, k * (256 >> 4)), ID_OZ, k > 0);
-            }
+            for (int k = 0; k < 8; ++k)
+              if (k < ksteps) mma_f16(tmem + COL_O, adv(dsc_qk, kstep(k)), adv(dsc_s, k * (256 >> 4)), ID_O, k > 0);
           }
-        }
-        {
           const uint32_t ID_S = instr_desc(128, NW, FMT_F16, MAJOR_MN, MAJOR_MN);
           constexpr uint32_t ID_SZ = instr_desc(128, 16, FMT_F16, MAJOR_MN, MAJOR_MN);
 #pragma unroll
@@ -515,20 +522,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           mma_commit(bar(B_MMA2));
         }
-        }
         if (MODE == 0) {
           WAITSET(BIT(B_PH_FULL), PAR(B_PH_FULL, p));
           if (lane == 0) {
-          tc_fence_after_sync();
-          const uint32_t ID_O = instr_desc(128, NW, FMT_F16, MAJOR_K, MAJOR_MN);
-          constexpr uint32_t ID_OZ = instr_desc(128, 16, FMT_F16, MAJOR_K, MAJOR_MN);
+            // O' += P v  (the scores' part of the denominator is summed by the mask pass)
+            tc_fence_after_sync();
+            const uint32_t ID_O = instr_desc(128, NW, FMT_F16, MAJOR_K, MAJOR_MN);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint64_t ad = adv(dsc_p, k * 2);
-            mma_f16(tmem + COL_O, ad, adv(dsc_v, k * (2048 >> 4)), ID_O, 1);
-            mma_f16(tmem + COL_OZ, ad, adv(dsc_one, k * (256 >> 4)), ID_OZ, 1);
-          }
-          mma_commit(bar(B_MMA3));
+            for (int k = 0; k < 4; ++k)
+              mma_f16(tmem + COL_O, adv(dsc_p, k * 2), adv(dsc_v, k * (2048 >> 4)), ID_O, 1);
+            mma_commit(bar(B_MMA3));
           }
         }
       }
@@ -570,7 +573,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int ot0 = t_begin + m * C;
       const int onvalid = min(C, t_end - ot0);
       tc_fence_after_sync();
-      float den = tmem_ld1(lane_base + COL_OZ);
+      float den = tmem_ld1(lane_base + COL_O + dh);
+      const float den_p0 = tmem_ld1(lane_base + COL_MAIL + 8 + 2 * (m & 1));
+      const float den_p1 = tmem_ld1(lane_base + COL_MAIL + 8 + 2 * (m & 1) + 1);
       // The query features went in as exp(y - max), without their softmax normalizer: it cancels in Eq. 8 except next to
       // eps, which therefore gets scaled by it; without normalization the numerator is divided by it.
       float qs = 0.f;
@@ -579,6 +584,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!narrow) qs += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
       }
       tmem_wait_ld();
+      den += den_p0 + den_p1;
       const float inv = 1.f / (a.normalize ? fmaf(a.eps, qs, den) : qs);
       bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * dh + och * 64;
       float y[32];
@@ -780,19 +786,30 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // reading sweeps of chunk m + 1, which do not have to wait for MMA 2 of chunk m.
     auto mask_chunk = [&](int m) {
       // (MMA 3 of the chunk before: the score tile was its operand)
-      WAITSETF(BIT(B_MMA2) | (m > 0 ? BIT(B_MMA3) : 0u), PAR(B_MMA2, m & 1) | PAR(B_MMA3, (m - 1) & 1));
+      WAITSETF(BIT(B_P) | (m > 0 ? BIT(B_MMA3) : 0u), PAR(B_P, m & 1) | PAR(B_MMA3, (m - 1) & 1));
       if (fail) return;
       tc_fence_after_sync();
       float s[32];
       tmem_ld32(lane_base + COL_P + ch * 32, s);
       tmem_wait_ld();
+      // The chunk's own part of the denominator is the row sum of the masked scores AS ROUNDED to fp16: numerator and
+      // denominator then carry the same weights (the first tokens of a sequence do not average a mismatch out).
+      float rs = 0.f;
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
-        float v[8];
+        uint32_t w[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = (ch * 32 + q4 * 8 + i <= row) ? s[q4 * 8 + i] : 0.f;
-        sts128(sb + OFF_PH + sw128(row, ch * 4 + q4), pack8(v, true));
+        for (int i = 0; i < 4; ++i) {
+          const int col = ch * 32 + q4 * 8 + 2 * i;
+          const __half2 h2 = __floats2half2_rn(col <= row ? s[q4 * 8 + 2 * i] : 0.f, col + 1 <= row ? s[q4 * 8 + 2 * i + 1] : 0.f);
+          const float2 f2 = __half22float2(h2);
+          rs += f2.x + f2.y;
+          w[i] = *reinterpret_cast<const uint32_t*>(&h2);
+        }
+        sts128(sb + OFF_PH + sw128(row, ch * 4 + q4), make_uint4(w[0], w[1], w[2], w[3]));
       }
+      tmem_st1(lane_base + COL_MAIL + 8 + 2 * (m & 1) + ch, rs);
+      tmem_wait_st();
       fence_proxy_async();
       tc_fence_before_sync();
       mbar_arrive(bar(B_PH_FULL));
@@ -802,6 +819,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int nvalid = min(C, t_end - (t_begin + n * C));
       float y[32], ya[16], yb[16];
       float mb = 0.f, sum = 0.f;
+      // ---- mask of the previous chunk: its scores are the first product issued after the hand-over, ahead of this
+      // chunk's mix ---------------------------------------------------------------------------------------------------
+      if (MODE == 0 && is_q && n > 0) mask_chunk(n - 1);
       // ---- phi, reading sweeps ----------------------------------------------------------------------------------------
       if (phi_on) {
         WAITF(B_MMA1, p);
@@ -873,7 +893,6 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       // ---- the previous chunk's MMA 2 has completed: the state is updated; qs / ks / kh / state operand are free ---------
-      if (MODE == 0 && is_q && n > 0) mask_chunk(n - 1);
       WAITSETF(BIT(B_X_FULL) | (n > 0 ? BIT(B_MMA2) : 0u), PAR(B_X_FULL, p) | PAR(B_MMA2, pp));
       tc_fence_after_sync();
       const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
@@ -901,7 +920,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               uint64_t w[4];
 #pragma unroll
               for (int i = 0; i < 4; ++i) w[i] = f2_mul(dm2, f2_pack(y[8 * q4 + 2 * i], y[8 * q4 + 2 * i + 1]));
-              sts128(sb + OFF_SBF + ch * 16384 + sw128(c, b2 * 4 + q4), pack8p(w, f16));
+              // columns [8 nb, 8 nb + 8) of row c: block nb of the unswizzled operand (a warp's 32 rows: 512 contiguous bytes)
+              sts128(sb + OFF_SBF + (uint32_t)(ch * 8 + b2 * 4 + q4) * 2048u + (uint32_t)c * 16u, pack8p(w, f16));
             }
           }
           {
@@ -915,7 +935,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           const float z = tmem_ld1(lane_base + COL_SZ);
           tmem_wait_ld();
           if (MODE == 0) {
-            *reinterpret_cast<uint16_t*>(sg + OFF_SZ + (c >> 3) * 128 + (c & 7) * 16) = to16(dm * z, f16);
+            *reinterpret_cast<uint16_t*>(sg + OFF_SBF + (dh >> 3) * 2048 + c * 16) = to16(dm * z, f16);
             mx = fmaxf(mx, fabsf(z));
           }
           tmem_st1(lane_base + COL_SZ, dC * z);

@@ -67,9 +67,11 @@ def test_c4_distillation_step_forward_and_backward(api):
     torch.cuda.synchronize()
     op = oracle_params(s)
     ref_f = O.layer_fwd(op, *[x[n] for n in NAMES])
-    check(f["o"], ref_f["o"], "bf16", "o")
-    # the oracle's backward takes the stored (bf16-rounded) intermediate features, as the GPU chain does
+    check(qd, ref_f["qdot"], "bf16", "qdot")
+    check(kd, ref_f["kdot"], "bf16", "kdot")
+    # each call against the oracle on the inputs that call was given: the stored (bf16-rounded) features for the attention
     qd_h, kd_h = qd.float().cpu().numpy(), kd.float().cpu().numpy()
+    check(f["o"], O.gla_fwd(op, qd_h, kd_h, x["v"], x["gate"])["o"], "bf16", "o")
     ref_g = O.gla_bwd(op, qd_h, kd_h, x["v"], x["gate"], x["dO"], None, None)
     for name in ("d_qdot", "d_kdot", "dv", "dgate"):
         check(g[name], ref_g[name], "bf16", name)

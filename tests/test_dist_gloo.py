@@ -60,3 +60,26 @@ def test_reference_arm_prints_on_rank_zero_only():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
     assert outs[1].strip() == ""
+
+
+def test_gpus_flag_against_the_launcher_environment():
+    """--gpus N either matches the launcher's world size, or (no launcher) makes bench.py start the N ranks itself; a
+    contradiction between the two is an error, never a silent single-replica run."""
+    import bench
+    assert bench.replica_launch_plan(1, {}) == "run"
+    assert bench.replica_launch_plan(8, {}) == "spawn"
+    assert bench.replica_launch_plan(2, {"WORLD_SIZE": "2"}) == "run"
+    assert "contradicts" in bench.replica_launch_plan(8, {"WORLD_SIZE": "2"})
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--impl", "reference"], cwd=ROOT,
+                       env=dict(os.environ, WORLD_SIZE="2", RANK="0"), capture_output=True, text=True)
+    assert r.returncode != 0 and "contradicts" in r.stderr
+
+
+def test_reference_arm_covers_training_and_decode_workloads():
+    for wl, extra in (("c4", ["--ref-tokens", "1024"]), ("c5-decode", [])):
+        r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
+                            "--warmup", "0", "--workload", wl] + extra, cwd=ROOT, capture_output=True, text=True,
+                           env={k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK")})
+        assert r.returncode == 0, r.stderr[-2000:]
+        line = json.loads(r.stdout.strip().splitlines()[-1])
+        assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["cores"] >= 1
