@@ -245,3 +245,12 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
 }
 
 }  // namespace lawcat
+
+#ifdef LAWCAT_TIMELINE
+// (profiling builds only) copies the clock stamps of the last layer-kernel launch to the host
+extern "C" int lawcat_timeline_read(long long* host, size_t n) {
+  const size_t have = sizeof(lawcat::tc::g_timeline) / sizeof(long long);
+  return cudaMemcpyFromSymbol(host, lawcat::tc::g_timeline, sizeof(long long) * (n < have ? n : have)) == cudaSuccess
+             ? LAWCAT_OK : LAWCAT_ERR_CUDA;
+}
+#endif

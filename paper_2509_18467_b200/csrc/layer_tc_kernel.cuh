@@ -37,6 +37,20 @@
 namespace lawcat {
 namespace tc {
 
+// Optional time line (profiling builds only, -DLAWCAT_TIMELINE): one lane per role of thread block 0 stamps the clock at
+// fixed points of four consecutive chunks into a device array that lawcat_timeline_read copies out.
+#ifdef LAWCAT_TIMELINE
+constexpr int TL_ROLES = 6, TL_IDS = 16, TL_N0 = 40, TL_NCH = 4;
+__device__ long long g_timeline[TL_ROLES * TL_IDS * TL_NCH];
+#define TL(role, id, n, who)                                                                        \
+  do {                                                                                              \
+    if (MODE == 0 && blockIdx.x == 0 && (who) && (n) >= TL_N0 && (n) < TL_N0 + TL_NCH)              \
+      g_timeline[((role) * TL_IDS + (id)) * TL_NCH + ((n) - TL_N0)] = clock64();                    \
+  } while (0)
+#else
+#define TL(role, id, n, who) do { } while (0)
+#endif
+
 constexpr int D = 128;       // d_k = d_v
 constexpr int C = 64;        // tokens per chunk
 constexpr int MID = 31;      // reference token of the in-chunk decay factorization
@@ -484,6 +498,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t p = (uint32_t)(n & 1), pp = p ^ 1u;
         WAITSET(BIT(B_QK_FULL) | BIT(B_SBF_FULL) | BIT(B_VH_FULL) | (MODE == 0 && n > 0 ? BIT(B_O_FREE) : 0u),
                 PAR(B_QK_FULL, p) | PAR(B_SBF_FULL, p) | PAR(B_VH_FULL, p) | PAR(B_O_FREE, pp));
+        TL(0, 0, n, lane == 0);
         const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
         const int fmt = f16 ? FMT_F16 : FMT_BF16;
         if (MODE == 0 && lane == 0) {
@@ -495,14 +510,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (k < ksteps) mma_f16(tmem + COL_P, adv(dsc_qk, kstep(k)), adv(dsc_ks, kstep(k)), ID_P, k > 0);
           mma_commit(bar(B_P));
         }
+        TL(0, 1, n, lane == 0);
         if (n + 1 < nchunks) {
-          // then the mix of the next chunk: its phi pass reads Y while this chunk's read-out and state update execute
+          // then the mix of the next chunk: its phi sweeps read Y while this chunk's read-out and state update execute
           WAITSET(BIT(B_U_FULL) | BIT(B_Y_FREE), PAR(B_U_FULL, pp) | PAR(B_Y_FREE, p));
           if (lane == 0) {
             tc_fence_after_sync();
             issue_mma1();
           }
         }
+        TL(0, 2, n, lane == 0);
         if (lane == 0) {
           tc_fence_after_sync();
           if (MODE == 0) {
@@ -522,8 +539,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           mma_commit(bar(B_MMA2));
         }
+        TL(0, 3, n, lane == 0);
         if (MODE == 0) {
           WAITSET(BIT(B_PH_FULL), PAR(B_PH_FULL, p));
+          TL(0, 4, n, lane == 0);
           if (lane == 0) {
             // O' += P v  (the scores' part of the denominator is summed by the mask pass)
             tc_fence_after_sync();
@@ -533,6 +552,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               mma_f16(tmem + COL_O, adv(dsc_p, k * 2), adv(dsc_v, k * (2048 >> 4)), ID_O, 1);
             mma_commit(bar(B_MMA3));
           }
+          TL(0, 5, n, lane == 0);
         }
       }
     }
@@ -620,6 +640,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // ---- conv, in place: the three rows in front of this thread's rows belong to another thread (or to the previous
       // chunk), so they are read before the barrier and every row is overwritten only after it ------------------------
       WAITF(B_RAW_FULL, p);
+      TL(warp == 0 ? 3 : 4, 0, n, (warp == 0 || warp == 2) && lane == 0);
       uint64_t x1[4], x2[4], x3[4], x0[4];  // sliding window of raw rows, packed pairs of fp32
       if (cv_on && !fail) {
         if (cv_rg == 0) {
@@ -655,9 +676,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       fence_proxy_async();
       named_bar_sync(1, PREP_THREADS);
       mbar_arrive(bar(B_U_FULL));
+      TL(warp == 0 ? 3 : 4, 1, n, (warp == 0 || warp == 2) && lane == 0);
 
       // ---- gate: exponents x_t = b_t - b_mid, scanned outwards from MID ------------------------------------------------
       if (a.gate_dim != 1) WAITF(B_G_FULL, p);
+      TL(warp == 0 ? 3 : 4, 2, n, (warp == 0 || warp == 2) && lane == 0);
       {
         const uint8_t* gcol = sg + OFF_G + (gc >> 6) * 8192 + (gc & 7) * 2;
         // x[t][c] fp32, 512-byte rows whose 16-byte chunks are XOR-swizzled with t & 7 (conflict-free for this
@@ -701,7 +724,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
         // the exponent tile is free once the previous chunk's phi pass has read it; the log-decays above did not need it
         mbar_arrive(bar(B_G_FREE));
+        TL(warp == 0 ? 3 : 4, 3, n, (warp == 0 || warp == 2) && lane == 0);
         if (n > 0) WAITF(B_X_FREE, pp);
+        TL(warp == 0 ? 3 : 4, 4, n, (warp == 0 || warp == 2) && lane == 0);
         float acc = 0.f;
         if (!g_on) {
           // nothing: nobody reads these channels' exponents or sums
@@ -728,15 +753,19 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (lane == 0) atomicMax(&s_rmax[p], __float_as_int(am));  // g <= 0: the largest exponent magnitude
       }
       mbar_arrive(bar(B_X_FULL));
+      TL(warp == 0 ? 3 : 4, 5, n, (warp == 0 || warp == 2) && lane == 0);
 
       // ---- output of the previous chunk (its last product completes about now; the v tile is loaded after it) -----------
       if (MODE == 0 && n > 0) {
         WAITF(B_MMA3, pp);
+        TL(warp == 0 ? 3 : 4, 6, n, (warp == 0 || warp == 2) && lane == 0);
         if (!fail) out_pass(n - 1);
+        TL(warp == 0 ? 3 : 4, 7, n, (warp == 0 || warp == 2) && lane == 0);
       }
 
       // ---- v: bf16 -> fp16 in place (exact for |v| in the fp16 normal range) ------------------------------------------
       WAITF(B_V_FULL, p);
+      TL(warp == 0 ? 3 : 4, 8, n, (warp == 0 || warp == 2) && lane == 0);
       // (layer mode: by the warps of TMEM quadrants 2-3 only; those of quadrants 0-1 carry the output pass)
       if (!fail && (MODE == 1 || (warp & 3) >= 2)) {
         const int vthreads = MODE == 1 ? PREP_THREADS : PREP_THREADS / 2;
@@ -756,6 +785,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       }
       fence_proxy_async();
       mbar_arrive(bar(B_VH_FULL));
+      TL(warp == 0 ? 3 : 4, 9, n, (warp == 0 || warp == 2) && lane == 0);
     }
     if (MODE == 0 && nchunks > 0 && !fail && !*s_abort &&
         wait_or_abort(bar(B_MMA3), (uint32_t)((nchunks - 1) & 1), s_abort))
@@ -819,12 +849,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int nvalid = min(C, t_end - (t_begin + n * C));
       float y[32], ya[16], yb[16];
       float mb = 0.f, sum = 0.f;
+      TL(warp == 8 ? 1 : 2, 0, n, (warp == 8 || warp == 10) && lane == 0);
       // ---- mask of the previous chunk: its scores are the first product issued after the hand-over, ahead of this
       // chunk's mix ---------------------------------------------------------------------------------------------------
       if (MODE == 0 && is_q && n > 0) mask_chunk(n - 1);
+      TL(warp == 8 ? 1 : 2, 1, n, (warp == 8 || warp == 10) && lane == 0);
       // ---- phi, reading sweeps ----------------------------------------------------------------------------------------
       if (phi_on) {
         WAITF(B_MMA1, p);
+        TL(warp == 8 ? 1 : 2, 2, n, (warp == 8 || warp == 10) && lane == 0);
         tc_fence_after_sync();
         float m = -INFINITY;
         // (64-wide head: the threads of the upper 64 columns have no outputs: they skip every sweep, and the two threads
@@ -855,6 +888,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
         }
         mb = m * L2E;
+        TL(warp == 8 ? 1 : 2, 3, n, (warp == 8 || warp == 10) && lane == 0);
         if (!is_q) {
           // key rows: e = exp(y - max) and its sum; e is parked in Y's own columns for the writing sweep
           if (!fail && !padded) {
@@ -893,12 +927,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       // ---- the previous chunk's MMA 2 has completed: the state is updated; qs / ks / kh / state operand are free ---------
+      TL(warp == 8 ? 1 : 2, 4, n, (warp == 8 || warp == 10) && lane == 0);
       WAITSETF(BIT(B_X_FULL) | (n > 0 ? BIT(B_MMA2) : 0u), PAR(B_X_FULL, p) | PAR(B_MMA2, pp));
+      TL(warp == 8 ? 1 : 2, 5, n, (warp == 8 || warp == 10) && lane == 0);
       tc_fence_after_sync();
       const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
       // ---- state pass: 16-bit operand 2^b_mid [S|z], accumulator [S|z] *= 2^b_C (this thread: 64 columns of row r128)
       // (64-wide head: only the rows and columns that exist)
       const bool s_on = !narrow || (!padded && r128 < dh);
+      // The largest state entry (which decides between fp16 and bf16 operands) is measured every 8th chunk; in between
+      // its bound grows by 64 max|v| per chunk (kh <= 1), a few thousand at most against the threshold of 3e4.
+      const bool track = (n & 7) == 0;
       if (!fail && !s_on && !phi_on) mbar_arrive(bar(B_X_FREE));  // (see the end of the pass)
       if (!fail && s_on) {
         const int c = r128;
@@ -912,8 +951,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tmem_ld32(lane_base + COL_S + blk * 32, y);
           tmem_wait_ld();
           if (MODE == 0) {
+            if (track) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(y[i]));
+              for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fabsf(y[i]));
+            }
             const uint64_t dm2 = f2_pack(dm, dm);
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
@@ -936,17 +977,18 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tmem_wait_ld();
           if (MODE == 0) {
             *reinterpret_cast<uint16_t*>(sg + OFF_SBF + (dh >> 3) * 2048 + c * 16) = to16(dm * z, f16);
-            mx = fmaxf(mx, fabsf(z));
+            if (track) mx = fmaxf(mx, fabsf(z));
           }
           tmem_st1(lane_base + COL_SZ, dC * z);
         }
-        if (MODE == 0) {
+        if (MODE == 0 && track) {
           mx = warp_max(mx);
           if (lane == 0) atomicMax(s_smax, __float_as_int(mx < 3.0e38f ? mx : 3.0e38f));
         }
         tmem_wait_st();
         if (!phi_on) mbar_arrive(bar(B_X_FREE));  // (state-only pass) this thread has read bm, ft and reads no exponents
       }
+      TL(warp == 8 ? 1 : 2, 6, n, (warp == 8 || warp == 10) && lane == 0);
       // ---- phi, writing sweep -------------------------------------------------------------------------------------------
       if (phi_on && !fail && !padded) {
         if (is_q) {
@@ -1015,14 +1057,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       // ---- hand-over to MMA 2: state operand, qs / ks / kh, and the bound on the state for the next chunk ------------
+      TL(warp == 8 ? 1 : 2, 7, n, (warp == 8 || warp == 10) && lane == 0);
       WAITF(B_VH_FULL, p);  // the chunk's max|v| is known
+      TL(warp == 8 ? 1 : 2, 8, n, (warp == 8 || warp == 10) && lane == 0);
       fence_proxy_async();
       tc_fence_before_sync();
       fail = named_bar_or(2, 256, fail);
+      TL(warp == 8 ? 1 : 2, 9, n, (warp == 8 || warp == 10) && lane == 0);
       if (fail) break;
       if (MODE == 0 && tw == 0) {
         // |S_new| <= |S_old| + 64 max|v|: the next chunk's choice of operand type
-        s_sbound[pp] = __float_as_int(__int_as_float(*s_smax) + 64.f * fmaxf(__int_as_float(s_vmax[p]), 1.f));
+        s_sbound[pp] = __float_as_int(__int_as_float(track ? *s_smax : s_sbound[p]) + 64.f * fmaxf(__int_as_float(s_vmax[p]), 1.f));
         *s_smax = 0;
         __threadfence_block();
       }
