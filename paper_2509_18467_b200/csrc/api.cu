@@ -69,6 +69,7 @@ size_t lawcat_workspace_bytes(const lawcat_params* p, int op) {
     case LAWCAT_OP_CONV_BWD:
       return align_up(sizeof(float) * elems(p, p->H, p->d_k), 256) + align_up(sizeof(float) * elems(p, p->H_kv, p->d_k), 256);
     case LAWCAT_OP_GLA_BWD:
+      if (gla_tc_bwd_supported(*p)) return gla_tc_bwd_workspace_bytes(*p);
       return align_up(sizeof(float) * elems(p, p->H, p->d_v), 256) + 2 * align_up(sizeof(float) * elems(p, p->H, 1), 256) +
              align_up(sizeof(float) * elems(p, p->H, p->d_k), 256);
     case LAWCAT_OP_LAYER_FWD:
@@ -124,6 +125,8 @@ int lawcat_gla_fwd(const lawcat_params* p, const void* qdot, const void* kdot, c
   const void* const opt[] = {S0, z0, den, S_T, z_T};
   if ((r = check_ptrs(req, opt, (size_t)p->B * p->T == 0))) return r;
   Ctx c{p, (cudaStream_t)stream, dev_status};
+  if ((size_t)p->B * p->T != 0 && gla_tc_supported(*p))  // chunkwise tensor-core kernel
+    return launch_gla_fwd_tc(c, qdot, kdot, v, gate, S0, z0, o, den, S_T, z_T);
   return launch_gla_fwd_rec(c, qdot, kdot, false, v, gate, S0, z0, o, den, S_T, z_T);
 }
 
@@ -139,6 +142,8 @@ int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, c
   const size_t need = lawcat_workspace_bytes(p, LAWCAT_OP_GLA_BWD);
   if (need && (!ws || ws_bytes < need)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
   Ctx c{p, (cudaStream_t)stream, dev_status};
+  if ((size_t)p->B * p->T != 0 && gla_tc_bwd_supported(*p))  // chunkwise tensor-core kernel
+    return launch_gla_bwd_tc(c, qdot, kdot, v, gate, S0, z0, dO, d_qdot, d_kdot, dv, dgate, ws);
   return launch_gla_bwd_rec(c, qdot, kdot, v, gate, S0, z0, o, den, dO, d_qdot, d_kdot, dv, dgate, ws);
 }
 

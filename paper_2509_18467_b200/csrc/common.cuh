@@ -79,6 +79,15 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
                     const void* w_k, const void* W, const void* cache_q_in, const void* cache_k_in, const float* S0,
                     const float* z0, void* o, float* S_T, float* z_T, void* ws);
 
+// Chunkwise tensor-core GLA on given features and its backward (gla_tc.cu).
+bool gla_tc_supported(const lawcat_params& p);
+bool gla_tc_bwd_supported(const lawcat_params& p);
+size_t gla_tc_bwd_workspace_bytes(const lawcat_params& p);
+int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
+                      const float* z0, void* o, float* den, float* S_T, float* z_T);
+int launch_gla_bwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
+                      const float* z0, const void* dO, void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws);
+
 // Counts one kernel launch; while tracing is on it also brackets the launch with CUDA events on its stream.
 struct LaunchScope {
   LaunchScope(const char* name, cudaStream_t s);
