@@ -92,7 +92,7 @@ int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const 
   const void* const opt[] = {W, cache_q, cache_k};
   if ((r = check_ptrs(req, opt, (size_t)p->B * p->T == 0))) return r;
   Ctx c{p, (cudaStream_t)stream, dev_status};
-  if (W) return launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot, false);
+  if (W) return launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot, false, p->chunk == 1);
   if ((r = launch_conv_plain(c, q, w_q, cache_q, qdot, p->H))) return r;
   return launch_conv_plain(c, k, w_k, cache_k, kdot, p->H_kv);
 }
@@ -169,7 +169,7 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
   // exact path: conv + mix + phi into fp32 scratch, then the recurrent GLA
   float* qdot = (float*)ws;
   float* kdot = (float*)((char*)ws + align_up(sizeof(float) * elems(p, p->H, p->d_k), 256));
-  if ((r = launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true))) return r;
+  if ((r = launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true, true))) return r;
   if ((r = launch_gla_fwd_rec(c, qdot, kdot, true, v, gate, S0, z0, o, nullptr, S_T, z_T))) return r;
   return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
 }

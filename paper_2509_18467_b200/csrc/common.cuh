@@ -50,8 +50,9 @@ struct Ctx {
 };
 
 int launch_conv_plain(const Ctx& c, const void* x, const void* w, const void* cache, void* out, int NH);
+// (exact: the fp32 CUDA-core kernel even where the tensor-core one applies)
 int launch_convmix_fwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
-                       const void* cache_q, const void* cache_k, void* qdot, void* kdot, bool out_f32);
+                       const void* cache_q, const void* cache_k, void* qdot, void* kdot, bool out_f32, bool exact);
 int launch_conv_bwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
                     const void* cache_q, const void* cache_k, const void* d_qdot, const void* d_kdot, void* dq,
                     void* dk, float* dw_q, float* dw_k, float* dW, void* ws);
@@ -87,6 +88,15 @@ int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const vo
                       const float* z0, void* o, float* den, float* S_T, float* z_T);
 int launch_gla_bwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
                       const float* z0, const void* dO, void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws);
+
+// Tensor-core conv -> mix -> softmax and the chain rule back through mix and softmax (convmix_tc.cu).
+bool convmix_tc_fwd_supported(const lawcat_params& p);
+bool convmix_tc_bwd_supported(const lawcat_params& p);
+int launch_convmix_tc_fwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
+                          const void* cache_q, const void* cache_k, void* qdot, void* kdot, bool out_f32);
+int launch_convmix_tc_bwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
+                          const void* cache_q, const void* cache_k, const void* d_qdot, const void* d_kdot, bool grads_f32,
+                          float* du_q, float* du_k, float* dW);
 
 // Counts one kernel launch; while tracing is on it also brackets the launch with CUDA events on its stream.
 struct LaunchScope {

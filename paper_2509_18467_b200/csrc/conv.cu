@@ -1,5 +1,7 @@
 // Causal depthwise Conv1D across tokens, the shared per-head linear layer and the feature map phi (Section 4.1),
 // forward and backward, CUDA-core (fp32 FMA) kernels. Storage type T is float or bfloat16; arithmetic is fp32.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace lawcat {
@@ -161,9 +163,11 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_fwd_kernel(ConvMixArgs a) 
 }
 
 int launch_convmix_fwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
-                       const void* cache_q, const void* cache_k, void* qdot, void* kdot, bool out_f32) {
+                       const void* cache_q, const void* cache_k, void* qdot, void* kdot, bool out_f32, bool exact) {
   const lawcat_params& p = *c.p;
   if (p.B * p.T == 0) return LAWCAT_OK;
+  if (convmix_tc_fwd_supported(p) && !exact)  // tensor-core kernel
+    return launch_convmix_tc_fwd(c, q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot, out_f32);
   ConvMixArgs a{q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot, p.B, p.T, p.H, p.H_kv, p.d_k, p.conv_k, p.phi};
   const size_t smem = sizeof(float) * ((size_t)p.d_k * p.d_k + (size_t)CM_TT * p.d_k);
   dim3 grid(p.B * ((p.T + CM_TT - 1) / CM_TT), p.H, 2);
@@ -443,6 +447,14 @@ static int conv_bwd_typed(const Ctx& c, const void* q, const void* k, const void
     return LAWCAT_ERR_CUDA;
   ConvMixBwdArgs a{q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, du_q, du_k, dW,
                    p.B, p.T, p.H, p.H_kv, p.conv_k, p.phi};
+  if (std::is_same<TI, bf16>::value && convmix_tc_bwd_supported(p) && p.chunk != 1) {
+    // tensor-core kernel for the mix and the softmax Jacobian; the conv's own backward follows on du as below
+    int r0 = launch_convmix_tc_bwd(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, false, du_q, du_k, dW);
+    if (r0) return r0;
+    r0 = conv_bwd_stream<TI, float>(c, du_q, (const TI*)q, (const TI*)w_q, (const TI*)cache_q, (TI*)dq, dw_q, p.H);
+    if (r0) return r0;
+    return conv_bwd_stream<TI, float>(c, du_k, (const TI*)k, (const TI*)w_k, (const TI*)cache_k, (TI*)dk, dw_k, p.H_kv);
+  }
   dim3 grid(p.B * ((p.T + CB_SPAN - 1) / CB_SPAN), p.H_kv);
 #define LAUNCH_CB(D)                                                                                             \
   do {                                                                                                           \

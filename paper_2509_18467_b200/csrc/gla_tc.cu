@@ -604,6 +604,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
     for (int n = nchunks - 1; n >= 0; --n) {
       const int t0 = n * C, nvalid = min(C, a.T - t0);
       prefetch_chunk(n - 1);
+      GTL(8);
       // ---- what crosses the end of this chunk: all pairs (key at or before the chunk, query behind it) feel every decay of
       // the chunk; their sum per key channel is the row-wise product of the state after the chunk with its adjoint,
       // sum_e S'_n[c,e] R_n[c,e]. S'_n is taken from the next chunk's state operand 2^bm S'_n (two-term, still in shared
@@ -626,7 +627,9 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         __syncthreads();
         if (tid < D) carry = (s_row[tid] + s_row[C + tid]) * ex2f(fminf(-s_bm[tid], 126.f)) * isc;
       }
+      GTL(9);
       gate_pass(t0, nvalid);
+      GTL(10);
       const uint8_t* src = a.ws_s16 + ((size_t)bh * nchunks + n) * (2 * TILE_CV + 16);
       const int fmt = *reinterpret_cast<const int*>(src + 2 * TILE_CV);
       const bool f16 = fmt == FMT_F16;
@@ -636,6 +639,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       __syncthreads();
       float vmax_unused = 0.f;
       operand_pass(t0, nvalid, f16, true, sc, vmax_unused);
+      GTL(11);
       // ---- adjoint-state pass: two-term operand 2^ft R, accumulator R *= 2^bC --------------------------------------------
       if (row_thr) {
         const float e63 = s_e63[row], dC = s_dC[row];
@@ -655,6 +659,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         tmem_wait_st();
       }
       publish();
+      GTL(12);
       if (tid == 0) {
         mma_split(COL_P, KV(OFF_QS, SLAB_T), KV(OFF_QSL, SLAB_T), KST_T, KV(OFF_KS, SLAB_T), KV(OFF_KSL, SLAB_T), KST_T,
                   D / 16, instr_desc(128, C, fmt, MAJOR_K, MAJOR_K), false);
@@ -664,6 +669,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         mma_commit(bar);
       }
       wait_mma();
+      GTL(13);
       if (row_thr) {
         const float dl = s_row[row], inv = s_row[C + row];  // dO_t . o_t and (scaled) 1 / den_t of this row
         float s[8], w[8];
@@ -682,6 +688,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         }
       }
       publish();
+      GTL(14);
       if (tid == 0) {
         const uint32_t ID_KM = instr_desc(128, D, fmt, MAJOR_K, MAJOR_MN), ID_MM = instr_desc(128, D, fmt, MAJOR_MN, MAJOR_MN),
                        ID_KK = instr_desc(128, D, fmt, MAJOR_K, MAJOR_K);
@@ -707,6 +714,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         mma_commit(bar);
       }
       wait_mma();
+      GTL(15);
       // ---- gradients of this chunk's rows ----------------------------------------------------------------------------------
       if (row_thr) {
         const size_t th = ((size_t)b * a.T + t0 + row) * a.H + h;
@@ -754,6 +762,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       tc_fence_before_sync();
       __syncthreads();
       tc_fence_after_sync();
+      GTL(16);
       // ---- gate gradient: reverse running sum over the chunk's tokens on top of what crosses its end, then the derivative
       // of the log-decay ----------------------------------------------------------------------------------------------------
       if (tid < D) {
@@ -792,6 +801,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         }
       }
       __syncthreads();
+      GTL(17);
     }
   }
 

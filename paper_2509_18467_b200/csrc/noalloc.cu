@@ -72,7 +72,7 @@ int lawcat_layer_fwd_noalloc(const lawcat_params* p, const void* q, const void* 
   Ctx c{p, (cudaStream_t)stream, dev_status};
   float* qdot = (float*)scratch;
   float* kdot = (float*)((char*)scratch + half);
-  if ((r = launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true))) return r;
+  if ((r = launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true, true))) return r;
   if ((r = launch_gla_fwd_rec(c, qdot, kdot, true, v, gate, S0, z0, o, nullptr, S_T, z_T))) return r;
   return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
 }
