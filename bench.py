@@ -7,7 +7,8 @@ Workloads (seeded synthetic inputs of `paper_2509_18467_b200.inputs`, through th
   c1, c2, c3, c5-T<N>   prefill: one step = one `lawcat_layer_fwd` (conv -> mix -> phi -> normalized GLA) over one batch,
                         returning the state and the conv caches a caller needs to continue; c3 is the headline
                         (Mistral-7B layer shape, T = 32768); c5-T<N> is the same shape at T = N
-  c4                    distillation step: conv_fwd -> gla_fwd -> gla_bwd -> conv_bwd (forward + backward) at B = 8, T = 1024
+  c4                    distillation step: `lawcat_layer_fwd` (the output the loss needs) + `lawcat_layer_bwd` (every gradient of
+                        the layer for a seeded upstream gradient) at B = 8, T = 1024
   c5-decode             one recurrent `lawcat_decode_step` for B = 64 sequences
 Prints ONE JSON line (rank 0). N > 1 runs N independent replicas (the layer has no inter-GPU exchange), one process per
 GPU; the time is the max over ranks. Started without a launcher, `--gpus N` starts the N ranks itself.
@@ -313,8 +314,9 @@ class Runner:
             self.o = torch.empty(s.B, s.T, s.H, s.d_v, dtype=self.tdt, device=dev)
             self.ws = torch.empty(max(api.workspace_bytes(p, api.OP_LAYER_FWD), 16), dtype=torch.uint8, device=dev)
         elif kind == "train":
-            self.ws_g = torch.empty(max(api.workspace_bytes(p, api.OP_GLA_BWD), 16), dtype=torch.uint8, device=dev)
-            self.ws_c = torch.empty(max(api.workspace_bytes(p, api.OP_CONV_BWD), 16), dtype=torch.uint8, device=dev)
+            self.o = torch.empty(s.B, s.T, s.H, s.d_v, dtype=self.tdt, device=dev)
+            self.ws = torch.empty(max(api.workspace_bytes(p, api.OP_LAYER_FWD), 16), dtype=torch.uint8, device=dev)
+            self.ws_b = torch.empty(max(api.workspace_bytes(p, api.OP_LAYER_BWD), 16), dtype=torch.uint8, device=dev)
         else:
             self.ws = torch.empty(max(api.workspace_bytes(p, api.OP_DECODE_STEP), 16), dtype=torch.uint8, device=dev)
             self.o = torch.empty(s.B, s.H, s.d_v, dtype=self.tdt, device=dev)
@@ -326,11 +328,9 @@ class Runner:
         if self.kind == "prefill":   # the state and the caches are part of what a prefill hands back
             self.res = api.lawcat_layer_fwd(p, *[d[n] for n in LAYER_NAMES], o=self.o, ws=self.ws)
         elif self.kind == "train":
-            qd, kd = api.lawcat_conv_fwd(p, d["q"], d["k"], d["w_q"], d["w_k"], d["W"])
-            f = api.lawcat_gla_fwd(p, qd, kd, d["v"], d["gate"], want_state=False)
-            g = api.lawcat_gla_bwd(p, qd, kd, d["v"], d["gate"], f["o"], f["den"], d["dO"], ws=self.ws_g)
-            c = api.lawcat_conv_bwd(p, d["q"], d["k"], d["w_q"], d["w_k"], d["W"], g["d_qdot"], g["d_kdot"], ws=self.ws_c)
-            self.res = dict(o=f["o"], dv=g["dv"], dgate=g["dgate"], **c)
+            api.lawcat_layer_fwd(p, *[d[n] for n in LAYER_NAMES], o=self.o, want_state=False, want_cache=False, ws=self.ws)
+            g = api.lawcat_layer_bwd(p, *[d[n] for n in LAYER_NAMES], d["dO"], ws=self.ws_b)
+            self.res = dict(o=self.o, **g)
         else:
             api.lawcat_decode_step(p, d["q"], d["k"], d["v"], d["gate"], d["w_q"], d["w_k"], d["W"], d["S"], d["z"],
                                    d["cache_q"], d["cache_k"], o_t=self.o, ws=self.ws)
@@ -505,7 +505,7 @@ def run_ours(args):
         if kind == "prefill":
             errs = {"o": err(R.o, ref["o"])}
         elif kind == "train":
-            # the chain stores its intermediate features in the storage type; the oracle differentiates the whole layer
+            # the oracle differentiates the whole layer from the raw inputs
             errs = {n: err(R.res[n], ref[n], n in ("dw_q", "dw_k", "dW")) for n in ("o", "dq", "dk", "dv", "dgate",
                                                                                   "dw_q", "dw_k", "dW")
                     if n not in ("dw_q", "dw_k", "dW") or n_units == units}

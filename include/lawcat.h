@@ -64,7 +64,8 @@ enum {
   LAWCAT_OP_GLA_FWD = 2,
   LAWCAT_OP_GLA_BWD = 3,
   LAWCAT_OP_LAYER_FWD = 4,
-  LAWCAT_OP_DECODE_STEP = 5
+  LAWCAT_OP_DECODE_STEP = 5,
+  LAWCAT_OP_LAYER_BWD = 6
 };
 
 typedef struct {
@@ -172,6 +173,24 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
                      const void* cache_k_in, const float* S0, const float* z0, void* o, void* cache_q_out,
                      void* cache_k_out, float* S_T, float* z_T, void* ws, size_t ws_bytes, void* stream,
                      int* dev_status);
+
+/*
+ * Backward of the whole layer (Fig. 1) for an upstream gradient dO [B,T,H,d_v]: the layer-wise distillation step of
+ * Section 5.1 in one call (chain rule on conv -> mix -> phi -> Eq. 4, Eq. 8; the paper prints no formulas). The features
+ * qdot, kdot are recomputed from q, k and never stored in the storage type: on the tensor-core path (bf16, d_k = d_v =
+ * 64, softmax feature map, conv_k <= 4, at most 4 query heads per key head, gate_tau >= 8 in LOGITS mode, chunk != 1) they
+ * and their gradients pass between the stages in fp32 scratch; every other shape runs the exact kernels as the chain
+ * conv -> attention -> attention backward -> conv backward entirely in fp32 (bf16 tensors are widened into scratch
+ * first and the four activation gradients narrowed at the end).
+ *   in:  the inputs of lawcat_layer_fwd (caches and initial state nullable) and dO
+ *   out: dq [B,T,H,d_k], dk [B,T,H_kv,d_k], dv [B,T,H_kv,d_v], dgate [B,T,H,gate_dim] in p->dtype;
+ *        dw_q, dw_k, dW in fp32, shaped like w_q, w_k, W, overwritten. All outputs are required.
+ * No gradient flows into the conv caches or the initial state.
+ */
+int lawcat_layer_bwd(const lawcat_params* p, const void* q, const void* k, const void* v, const void* gate,
+                     const void* w_q, const void* w_k, const void* W, const void* cache_q, const void* cache_k,
+                     const float* S0, const float* z0, const void* dO, void* dq, void* dk, void* dv, void* dgate,
+                     float* dw_q, float* dw_k, float* dW, void* ws, size_t ws_bytes, void* stream, int* dev_status);
 
 /*
  * One recurrent decode step for B sequences (p->T is ignored): the layer at a single token, using the conv cache

@@ -18,11 +18,11 @@ LIB_PATH = os.path.join(_PKG, "liblawcat.so")
 F32, BF16 = 0, 1
 PHI_SOFTMAX, PHI_ELU1, PHI_IDENTITY = 0, 1, 2
 GATE_LOGITS, GATE_LOGDECAY = 0, 1
-OP_CONV_FWD, OP_CONV_BWD, OP_GLA_FWD, OP_GLA_BWD, OP_LAYER_FWD, OP_DECODE_STEP = range(6)
+OP_CONV_FWD, OP_CONV_BWD, OP_GLA_FWD, OP_GLA_BWD, OP_LAYER_FWD, OP_DECODE_STEP, OP_LAYER_BWD = range(7)
 
 EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "lawcat_launch_count",
            "lawcat_trace_begin", "lawcat_trace_end", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
-           "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
+           "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_layer_bwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
            "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc"]
 
 
@@ -76,7 +76,8 @@ def lib() -> ctypes.CDLL:
                                            [ctypes.c_size_t, ctypes.c_void_p]
         L.lawcat_trace_end.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
         for name, nptr in (("lawcat_conv_fwd", 9), ("lawcat_conv_bwd", 14), ("lawcat_gla_fwd", 10),
-                           ("lawcat_gla_bwd", 13), ("lawcat_layer_fwd", 16), ("lawcat_decode_step", 12)):
+                           ("lawcat_gla_bwd", 13), ("lawcat_layer_fwd", 16), ("lawcat_layer_bwd", 19),
+                           ("lawcat_decode_step", 12)):
             f = getattr(L, name)
             f.restype = ctypes.c_int
             f.argtypes = [ctypes.POINTER(Params)] + [ctypes.c_void_p] * nptr + \
@@ -206,6 +207,20 @@ def lawcat_layer_fwd(p: Params, q, k, v, gate, w_q, w_k, W, cache_q=None, cache_
     _call("lawcat_layer_fwd", p, [q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0, o, cq, ck, S_T, z_T], ws, nb,
           stream, dev_status)
     return dict(o=o, cache_q=cq, cache_k=ck, S_T=S_T, z_T=z_T)
+
+
+def lawcat_layer_bwd(p: Params, q, k, v, gate, w_q, w_k, W, dO, cache_q=None, cache_k=None, S0=None, z0=None, ws=None,
+                     stream=None, dev_status=None):
+    """Gradients of the whole layer for the upstream gradient dO: dict(dq, dk, dv, dgate, dw_q, dw_k, dW)."""
+    dev = q.device
+    dq, dk, dv, dgate = (torch.empty_like(x) for x in (q, k, v, gate))
+    dw_q = torch.empty(w_q.shape, dtype=torch.float32, device=dev)
+    dw_k = torch.empty(w_k.shape, dtype=torch.float32, device=dev)
+    dW = torch.empty(W.shape, dtype=torch.float32, device=dev)
+    ws, nb = _ws(p, OP_LAYER_BWD, ws, dev)
+    _call("lawcat_layer_bwd", p, [q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0, dO, dq, dk, dv, dgate, dw_q, dw_k,
+                                  dW], ws, nb, stream, dev_status)
+    return dict(dq=dq, dk=dk, dv=dv, dgate=dgate, dw_q=dw_q, dw_k=dw_k, dW=dW)
 
 
 def lawcat_decode_step(p: Params, q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cache_q, cache_k, o_t=None, ws=None,

@@ -45,6 +45,62 @@ namespace lawcat {
 int validate_params(const lawcat_params* p, bool need_T) { return check_params(p, need_T); }
 }  // namespace lawcat
 
+extern "C" size_t lawcat_workspace_bytes(const lawcat_params* p, int op);
+
+namespace {
+// whether the fused layer backward runs on the tensor-core kernels (fp32 features between its stages)
+bool layer_bwd_tc(const lawcat_params& p) {
+  return p.chunk != 1 && gla_tc_bwd_supported(p) && convmix_tc_fwd_supported(p) && convmix_tc_bwd_supported(p);
+}
+
+__global__ void widen_kernel(const bf16* __restrict__ x, float* __restrict__ y, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) y[i] = __bfloat162float(x[i]);
+}
+__global__ void narrow_kernel(const float* __restrict__ x, bf16* __restrict__ y, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) y[i] = __float2bfloat16_rn(x[i]);
+}
+
+// Scratch of the exact layer backward: the chain conv_fwd -> gla_fwd -> gla_bwd -> conv_bwd in fp32. bf16 tensors are
+// widened to fp32 copies first and the four activation gradients narrowed at the end, so that no feature and no feature
+// gradient is rounded to bf16 between the stages.
+struct ExactBwdLayout {
+  size_t in[10];    // q k v gate w_q w_k W dO cache_q cache_k  (fp32 copies; only for bf16 storage)
+  size_t out[4];    // dq dk dv dgate (fp32; only for bf16 storage)
+  size_t qd, kd, dqd, dkd, o, den, ws_g, ws_c, total;
+};
+ExactBwdLayout exact_bwd_layout(const lawcat_params* p) {
+  ExactBwdLayout L{};
+  lawcat_params p32 = *p;
+  p32.dtype = LAWCAT_F32;
+  const size_t n_in[10] = {elems(p, p->H, p->d_k), elems(p, p->H_kv, p->d_k), elems(p, p->H_kv, p->d_v),
+                           elems(p, p->H, p->gate_dim), (size_t)p->H * p->d_k * p->conv_k,
+                           (size_t)p->H_kv * p->d_k * p->conv_k, (size_t)p->H * p->d_k * p->d_k, elems(p, p->H, p->d_v),
+                           (size_t)p->B * (p->conv_k - 1) * p->H * p->d_k, (size_t)p->B * (p->conv_k - 1) * p->H_kv * p->d_k};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes, 256); return o; };
+  const bool widen = p->dtype == LAWCAT_BF16;
+  for (int i = 0; i < 10; ++i) L.in[i] = take(widen ? 4 * n_in[i] : 0);
+  for (int i = 0; i < 4; ++i) L.out[i] = take(widen ? 4 * n_in[i] : 0);
+  L.qd = take(4 * n_in[0]); L.kd = take(4 * n_in[0]); L.dqd = take(4 * n_in[0]); L.dkd = take(4 * n_in[0]);
+  L.o = take(4 * n_in[7]); L.den = take(4 * elems(p, p->H, 1));
+  L.ws_g = take(lawcat_workspace_bytes(&p32, LAWCAT_OP_GLA_BWD));
+  L.ws_c = take(lawcat_workspace_bytes(&p32, LAWCAT_OP_CONV_BWD));
+  L.total = off;
+  return L;
+}
+
+size_t layer_bwd_workspace(const lawcat_params* p) {
+  if (layer_bwd_tc(*p)) {
+    // fp32 features and their gradients between the stages, then the scratch of the attention and the conv backward
+    return 4 * align_up(4 * elems(p, p->H, p->d_k), 256) + lawcat_workspace_bytes(p, LAWCAT_OP_GLA_BWD) +
+           lawcat_workspace_bytes(p, LAWCAT_OP_CONV_BWD);
+  }
+  return exact_bwd_layout(p).total;
+}
+}  // namespace
+
 extern "C" {
 
 int lawcat_version(void) { return 100; }
@@ -77,6 +133,8 @@ size_t lawcat_workspace_bytes(const lawcat_params* p, int op) {
       return 2 * align_up(sizeof(float) * elems(p, p->H, p->d_k), 256);
     case LAWCAT_OP_DECODE_STEP:
       return align_up(decode_workspace_bytes(*p), 256);
+    case LAWCAT_OP_LAYER_BWD:
+      return layer_bwd_workspace(p);
     default:
       return 0;
   }
@@ -143,7 +201,7 @@ int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, c
   if (need && (!ws || ws_bytes < need)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
   Ctx c{p, (cudaStream_t)stream, dev_status};
   if ((size_t)p->B * p->T != 0 && gla_tc_bwd_supported(*p))  // chunkwise tensor-core kernel
-    return launch_gla_bwd_tc(c, qdot, kdot, v, gate, S0, z0, dO, d_qdot, d_kdot, dv, dgate, ws);
+    return launch_gla_bwd_tc(c, qdot, kdot, v, gate, S0, z0, dO, d_qdot, d_kdot, dv, dgate, ws, false);
   return launch_gla_bwd_rec(c, qdot, kdot, v, gate, S0, z0, o, den, dO, d_qdot, d_kdot, dv, dgate, ws);
 }
 
@@ -172,6 +230,75 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
   if ((r = launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true, true))) return r;
   if ((r = launch_gla_fwd_rec(c, qdot, kdot, true, v, gate, S0, z0, o, nullptr, S_T, z_T))) return r;
   return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
+}
+
+int lawcat_layer_bwd(const lawcat_params* p, const void* q, const void* k, const void* v, const void* gate,
+                     const void* w_q, const void* w_k, const void* W, const void* cache_q, const void* cache_k,
+                     const float* S0, const float* z0, const void* dO, void* dq, void* dk, void* dv, void* dgate,
+                     float* dw_q, float* dw_k, float* dW, void* ws, size_t ws_bytes, void* stream, int* dev_status) {
+  int r = check_params(p, true);
+  if (r) return r;
+  const void* const req[] = {q, k, v, gate, w_q, w_k, W, dO, dq, dk, dv, dgate, dw_q, dw_k, dW};
+  const void* const opt[] = {cache_q, cache_k, S0, z0, ws};
+  if ((r = check_ptrs(req, opt))) return r;
+  const size_t need = lawcat_workspace_bytes(p, LAWCAT_OP_LAYER_BWD);
+  if (need && (!ws || ws_bytes < need)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
+  Ctx c{p, (cudaStream_t)stream, dev_status};
+  if ((size_t)p->B * p->T != 0 && layer_bwd_tc(*p)) {
+    char* w = (char*)ws;
+    const size_t nf = align_up(4 * elems(p, p->H, p->d_k), 256);
+    void* qd = w; void* kd = w + nf; void* dqd = w + 2 * nf; void* dkd = w + 3 * nf;
+    void* ws_g = w + 4 * nf;
+    void* ws_c = (char*)ws_g + lawcat_workspace_bytes(p, LAWCAT_OP_GLA_BWD);
+    // features recomputed in fp32, attention backward on them (it runs its own forward sweep), mix / softmax / conv backward
+    if ((r = launch_convmix_tc_fwd(c, q, k, w_q, w_k, W, cache_q, cache_k, qd, kd, true))) return r;
+    if ((r = launch_gla_bwd_tc(c, qd, kd, v, gate, S0, z0, dO, dqd, dkd, dv, dgate, ws_g, true))) return r;
+    return launch_conv_bwd(c, q, k, w_q, w_k, W, cache_q, cache_k, dqd, dkd, dq, dk, dw_q, dw_k, dW, ws_c, true);
+  }
+  // exact kernels, the whole chain in fp32
+  const ExactBwdLayout L = exact_bwd_layout(p);
+  char* w = (char*)ws;
+  lawcat_params p32 = *p;
+  p32.dtype = LAWCAT_F32;
+  p32.chunk = 1;
+  Ctx c32{&p32, (cudaStream_t)stream, dev_status};
+  const void* in[10] = {q, k, v, gate, w_q, w_k, W, dO, cache_q, cache_k};
+  void* out[4] = {dq, dk, dv, dgate};
+  const size_t n_in[10] = {elems(p, p->H, p->d_k), elems(p, p->H_kv, p->d_k), elems(p, p->H_kv, p->d_v),
+                           elems(p, p->H, p->gate_dim), (size_t)p->H * p->d_k * p->conv_k,
+                           (size_t)p->H_kv * p->d_k * p->conv_k, (size_t)p->H * p->d_k * p->d_k, elems(p, p->H, p->d_v),
+                           (size_t)p->B * (p->conv_k - 1) * p->H * p->d_k, (size_t)p->B * (p->conv_k - 1) * p->H_kv * p->d_k};
+  const bool widen = p->dtype == LAWCAT_BF16;
+  if (widen) {
+    for (int i = 0; i < 10; ++i) {
+      if (!in[i] || !n_in[i]) continue;
+      LAWCAT_LAUNCH("widen", c.stream, widen_kernel<<<(unsigned)((n_in[i] + 255) / 256), 256, 0, c.stream>>>(
+                                           (const bf16*)in[i], (float*)(w + L.in[i]), n_in[i]));
+      LAWCAT_CHECK_LAUNCH();
+      in[i] = w + L.in[i];
+    }
+    for (int i = 0; i < 4; ++i) out[i] = w + L.out[i];
+  }
+  if ((size_t)p->B * p->T != 0) {
+    if ((r = launch_convmix_fwd(c32, in[0], in[1], in[4], in[5], in[6], in[8], in[9], w + L.qd, w + L.kd, false, true))) return r;
+    if ((r = launch_gla_fwd_rec(c32, w + L.qd, w + L.kd, false, in[2], in[3], S0, z0, w + L.o, (float*)(w + L.den), nullptr, nullptr))) return r;
+    if ((r = launch_gla_bwd_rec(c32, w + L.qd, w + L.kd, in[2], in[3], S0, z0, w + L.o, (const float*)(w + L.den), in[7],
+                                w + L.dqd, w + L.dkd, out[2], out[3], w + L.ws_g)))
+      return r;
+  }
+  if ((r = launch_conv_bwd(c32, in[0], in[1], in[4], in[5], in[6], in[8], in[9], w + L.dqd, w + L.dkd, out[0], out[1], dw_q,
+                           dw_k, dW, w + L.ws_c, false)))
+    return r;
+  if (widen) {
+    void* dst[4] = {dq, dk, dv, dgate};
+    for (int i = 0; i < 4; ++i) {
+      if (!n_in[i]) continue;
+      LAWCAT_LAUNCH("narrow", c.stream, narrow_kernel<<<(unsigned)((n_in[i] + 255) / 256), 256, 0, c.stream>>>(
+                                            (const float*)out[i], (bf16*)dst[i], n_in[i]));
+      LAWCAT_CHECK_LAUNCH();
+    }
+  }
+  return LAWCAT_OK;
 }
 
 int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t, const void* v_t,

@@ -53,9 +53,10 @@ int launch_conv_plain(const Ctx& c, const void* x, const void* w, const void* ca
 // (exact: the fp32 CUDA-core kernel even where the tensor-core one applies)
 int launch_convmix_fwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
                        const void* cache_q, const void* cache_k, void* qdot, void* kdot, bool out_f32, bool exact);
+// (grads_f32: d_qdot, d_kdot are fp32 scratch of the fused layer backward; only on the tensor-core path)
 int launch_conv_bwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
                     const void* cache_q, const void* cache_k, const void* d_qdot, const void* d_kdot, void* dq,
-                    void* dk, float* dw_q, float* dw_k, float* dW, void* ws);
+                    void* dk, float* dw_q, float* dw_k, float* dW, void* ws, bool grads_f32 = false);
 int launch_cache_out(const Ctx& c, const void* q, const void* k, const void* cache_q_in, const void* cache_k_in,
                      void* cache_q_out, void* cache_k_out);
 int launch_gla_fwd_rec(const Ctx& c, const void* qdot, const void* kdot, bool qk_f32, const void* v,
@@ -87,7 +88,8 @@ size_t gla_tc_bwd_workspace_bytes(const lawcat_params& p);
 int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
                       const float* z0, void* o, float* den, float* S_T, float* z_T);
 int launch_gla_bwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
-                      const float* z0, const void* dO, void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws);
+                      const float* z0, const void* dO, void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws,
+                      bool feat_f32);
 
 // Tensor-core conv -> mix -> softmax and the chain rule back through mix and softmax (convmix_tc.cu).
 bool convmix_tc_fwd_supported(const lawcat_params& p);

@@ -426,7 +426,8 @@ static int conv_bwd_stream(const Ctx& c, const TD* du, const TI* x, const TI* w,
 template <typename TI>
 static int conv_bwd_typed(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k,
                           const void* W, const void* cache_q, const void* cache_k, const void* d_qdot,
-                          const void* d_kdot, void* dq, void* dk, float* dw_q, float* dw_k, float* dW, void* ws) {
+                          const void* d_kdot, void* dq, void* dk, float* dw_q, float* dw_k, float* dW, void* ws,
+                          bool grads_f32) {
   const lawcat_params& p = *c.p;
   if (p.B * p.T == 0) {
     if (dw_q && cudaMemsetAsync(dw_q, 0, sizeof(float) * (size_t)p.H * p.d_k * p.conv_k, c.stream)) return LAWCAT_ERR_CUDA;
@@ -449,12 +450,13 @@ static int conv_bwd_typed(const Ctx& c, const void* q, const void* k, const void
                    p.B, p.T, p.H, p.H_kv, p.conv_k, p.phi};
   if (std::is_same<TI, bf16>::value && convmix_tc_bwd_supported(p) && p.chunk != 1) {
     // tensor-core kernel for the mix and the softmax Jacobian; the conv's own backward follows on du as below
-    int r0 = launch_convmix_tc_bwd(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, false, du_q, du_k, dW);
+    int r0 = launch_convmix_tc_bwd(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, grads_f32, du_q, du_k, dW);
     if (r0) return r0;
     r0 = conv_bwd_stream<TI, float>(c, du_q, (const TI*)q, (const TI*)w_q, (const TI*)cache_q, (TI*)dq, dw_q, p.H);
     if (r0) return r0;
     return conv_bwd_stream<TI, float>(c, du_k, (const TI*)k, (const TI*)w_k, (const TI*)cache_k, (TI*)dk, dw_k, p.H_kv);
   }
+  if (grads_f32) return LAWCAT_ERR_UNSUPPORTED;  // (fp32 gradients only reach the tensor-core kernel)
   dim3 grid(p.B * ((p.T + CB_SPAN - 1) / CB_SPAN), p.H_kv);
 #define LAUNCH_CB(D)                                                                                             \
   do {                                                                                                           \
@@ -482,10 +484,10 @@ static int conv_bwd_typed(const Ctx& c, const void* q, const void* k, const void
 
 int launch_conv_bwd(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
                     const void* cache_q, const void* cache_k, const void* d_qdot, const void* d_kdot, void* dq,
-                    void* dk, float* dw_q, float* dw_k, float* dW, void* ws) {
+                    void* dk, float* dw_q, float* dw_k, float* dW, void* ws, bool grads_f32) {
   if (c.p->dtype == LAWCAT_F32)
-    return conv_bwd_typed<float>(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, dq, dk, dw_q, dw_k, dW, ws);
-  return conv_bwd_typed<bf16>(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, dq, dk, dw_q, dw_k, dW, ws);
+    return conv_bwd_typed<float>(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, dq, dk, dw_q, dw_k, dW, ws, false);
+  return conv_bwd_typed<bf16>(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, dq, dk, dw_q, dw_k, dW, ws, grads_f32);
 }
 
 // ------------------------------------------------------------------------------------------------ conv cache out

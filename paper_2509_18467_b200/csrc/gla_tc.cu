@@ -94,11 +94,14 @@ constexpr uint32_t COL_P = 0, COL_A = 64 /* O' | dQ */, COL_ST = 144 /* S' or R 
                    COL_V = 384 /* dV */;
 
 struct GArgs {
-  const bf16 *qdot, *kdot, *v, *gate, *dO;
+  const void *qdot, *kdot;   // features: bf16, or fp32 when feat_f32 (scratch of the fused layer backward)
+  const bf16 *v, *gate, *dO;
   const float *S0, *z0;
   bf16* o;
   float *den, *S_T, *z_T;
-  bf16 *d_qdot, *d_kdot, *dgate;
+  void *d_qdot, *d_kdot;     // bf16, or fp32 when feat_f32
+  bf16* dgate;
+  int feat_f32;
   float* dvh;         // [B,T,H,D] per-head dv (fp32), reduced over the heads of a group afterwards
   uint8_t* ws_s16;    // [B*H][chunks][2 TILE_CV + 16] the (two-term) state operand of every chunk and its format
   float *ws_den, *ws_delta;  // [B,T,H]: 1 / den_t and dO_t . o_t
@@ -294,7 +297,8 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
     const int r = tid >> 2, which = tid & 3, t = m * C + r;
     if (t >= a.T) return;
     const size_t tq = ((size_t)b * a.T + t) * a.H + h, tv = ((size_t)b * a.T + t) * a.Hkv + j;
-    const void* ptr = which == 0 ? (const void*)(a.qdot + tq * D) : which == 1 ? (const void*)(a.kdot + tq * D)
+    const size_t fb = a.feat_f32 ? 4 : 2;
+    const void* ptr = which == 0 ? (const void*)((const char*)a.qdot + tq * D * fb) : which == 1 ? (const void*)((const char*)a.kdot + tq * D * fb)
                     : which == 2 ? (const void*)(a.v + tv * D)
                     : (a.gate_dim == 1 ? (const void*)(a.gate + tq) : (const void*)(a.gate + tq * D));
     asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
@@ -389,8 +393,17 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       float inv = 0.f, dl = 0.f;
       if (r < nvalid) {
         const size_t tq = ((size_t)b * a.T + t0 + r) * a.H + h, tv = ((size_t)b * a.T + t0 + r) * a.Hkv + j;
-        zq = *reinterpret_cast<const uint4*>(a.qdot + tq * D + o8 * 8);
-        zk = *reinterpret_cast<const uint4*>(a.kdot + tq * D + o8 * 8);
+        if (BWD && a.feat_f32) {
+          const float* fq = reinterpret_cast<const float*>(a.qdot) + tq * D + o8 * 8;
+          const float* fk = reinterpret_cast<const float*>(a.kdot) + tq * D + o8 * 8;
+          const float4 q0 = *reinterpret_cast<const float4*>(fq), q1 = *reinterpret_cast<const float4*>(fq + 4);
+          const float4 k0 = *reinterpret_cast<const float4*>(fk), k1 = *reinterpret_cast<const float4*>(fk + 4);
+          q[0] = q0.x; q[1] = q0.y; q[2] = q0.z; q[3] = q0.w; q[4] = q1.x; q[5] = q1.y; q[6] = q1.z; q[7] = q1.w;
+          k[0] = k0.x; k[1] = k0.y; k[2] = k0.z; k[3] = k0.w; k[4] = k1.x; k[5] = k1.y; k[6] = k1.z; k[7] = k1.w;
+        } else {
+          zq = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(a.qdot) + tq * D + o8 * 8);
+          zk = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(a.kdot) + tq * D + o8 * 8);
+        }
         zv = *reinterpret_cast<const uint4*>(a.v + tv * D + o8 * 8);
         if (BWD && reverse) {
           zg = *reinterpret_cast<const uint4*>(a.dO + tq * D + o8 * 8);
@@ -398,7 +411,8 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
           dl = a.ws_delta[tq];
         }
       }
-      unpack8b(zq, q); unpack8b(zk, k); unpack8b(zv, vv);
+      if (!(BWD && a.feat_f32) || r >= nvalid) { unpack8b(zq, q); unpack8b(zk, k); }
+      unpack8b(zv, vv);
       const float4 xa = *reinterpret_cast<const float4*>(s_x + r * D + o8 * 8), xb = *reinterpret_cast<const float4*>(s_x + r * D + o8 * 8 + 4);
       x[0] = xa.x; x[1] = xa.y; x[2] = xa.z; x[3] = xa.w; x[4] = xb.x; x[5] = xb.y; x[6] = xb.z; x[7] = xb.w;
 #pragma unroll
@@ -752,8 +766,17 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
           *reinterpret_cast<float4*>(s_dt + row * D + c0) = make_float4(dd[0], dd[1], dd[2], dd[3]);
           *reinterpret_cast<float4*>(s_dt + row * D + c0 + 4) = make_float4(dd[4], dd[5], dd[6], dd[7]);
           if (valid) {
-            *reinterpret_cast<uint4*>(a.d_qdot + th * D + c0) = pack8h(dq, false);
-            *reinterpret_cast<uint4*>(a.d_kdot + th * D + c0) = pack8h(dk, false);
+            if (a.feat_f32) {
+              float* gq = reinterpret_cast<float*>(a.d_qdot) + th * D + c0;
+              float* gk = reinterpret_cast<float*>(a.d_kdot) + th * D + c0;
+              *reinterpret_cast<float4*>(gq) = make_float4(dq[0], dq[1], dq[2], dq[3]);
+              *reinterpret_cast<float4*>(gq + 4) = make_float4(dq[4], dq[5], dq[6], dq[7]);
+              *reinterpret_cast<float4*>(gk) = make_float4(dk[0], dk[1], dk[2], dk[3]);
+              *reinterpret_cast<float4*>(gk + 4) = make_float4(dk[4], dk[5], dk[6], dk[7]);
+            } else {
+              *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.d_qdot) + th * D + c0) = pack8h(dq, false);
+              *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(a.d_kdot) + th * D + c0) = pack8h(dk, false);
+            }
             *reinterpret_cast<float4*>(a.dvh + th * D + c0) = make_float4(dvv[0], dvv[1], dvv[2], dvv[3]);
             *reinterpret_cast<float4*>(a.dvh + th * D + c0 + 4) = make_float4(dvv[4], dvv[5], dvv[6], dvv[7]);
           }
@@ -881,7 +904,7 @@ int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const vo
   int r = set_smem_once();
   if (r) return r;
   GArgs a = gla_tc_args(c);
-  a.qdot = (const bf16*)qdot; a.kdot = (const bf16*)kdot; a.v = (const bf16*)v; a.gate = (const bf16*)gate;
+  a.qdot = qdot; a.kdot = kdot; a.v = (const bf16*)v; a.gate = (const bf16*)gate;
   a.S0 = S0; a.z0 = z0; a.o = (bf16*)o; a.den = den; a.S_T = S_T; a.z_T = z_T;
   LaunchScope _ls("gla_tc_fwd", c.stream);
   gla_tc_kernel<false><<<p.B * p.H, THREADS, SMEM_FWD, c.stream>>>(a);
@@ -890,15 +913,16 @@ int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const vo
 }
 
 int launch_gla_bwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
-                      const float* z0, const void* dO, void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws) {
+                      const float* z0, const void* dO, void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws,
+                      bool feat_f32) {
   using namespace gtc;
   const lawcat_params& p = *c.p;
   int r = set_smem_once();
   if (r) return r;
   GArgs a = gla_tc_args(c);
-  a.qdot = (const bf16*)qdot; a.kdot = (const bf16*)kdot; a.v = (const bf16*)v; a.gate = (const bf16*)gate;
+  a.qdot = qdot; a.kdot = kdot; a.v = (const bf16*)v; a.gate = (const bf16*)gate;
   a.dO = (const bf16*)dO; a.S0 = S0; a.z0 = z0;
-  a.d_qdot = (bf16*)d_qdot; a.d_kdot = (bf16*)d_kdot; a.dgate = (bf16*)dgate;
+  a.d_qdot = d_qdot; a.d_kdot = d_kdot; a.dgate = (bf16*)dgate; a.feat_f32 = feat_f32 ? 1 : 0;
   const size_t bth = (size_t)p.B * p.T * p.H;
   char* w = (char*)ws;
   a.dvh = (float*)w; w += align_up(sizeof(float) * bth * D, 256);
