@@ -178,7 +178,7 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
  * Backward of the whole layer (Fig. 1) for an upstream gradient dO [B,T,H,d_v]: the layer-wise distillation step of
  * Section 5.1 in one call (chain rule on conv -> mix -> phi -> Eq. 4, Eq. 8; the paper prints no formulas). The features
  * qdot, kdot are recomputed from q, k and never stored in the storage type: on the tensor-core path (bf16, d_k = d_v =
- * 64, softmax feature map, conv_k <= 4, at most 4 query heads per key head, gate_tau >= 8 in LOGITS mode, chunk != 1) they
+ * 64, softmax feature map, conv_k <= 4, gate_tau >= 8 in LOGITS mode, chunk != 1) they
  * and their gradients pass between the stages in fp32 scratch; every other shape runs the exact kernels as the chain
  * conv -> attention -> attention backward -> conv backward entirely in fp32 (bf16 tensors are widened into scratch
  * first and the four activation gradients narrowed at the end).

@@ -5,10 +5,10 @@
 // W_h): raw rows (with the conv_k - 1 rows in front) into shared memory, depthwise causal conv in fp32 -> fp16 operand,
 // Y = u W_h as one tcgen05 product per 16 channels (fp32 accumulator in tensor memory), softmax over a row by the thread
 // that owns the row's TMEM lane, 16-bit or fp32 store.
-// Backward (head width 64, up to 4 query heads per key head): one block = one (batch, key head, tile); for each query head of
+// Backward (head width 64): one block = one (batch, key head, tile); for each query head of
 // the group and each stream it recomputes u and p = softmax(u W_h), applies the softmax Jacobian dy = p (dp - p . dp),
-// and forms du = dy W_h^T (the key stream summed over the group in registers) and dW_h += u^T dy (one accumulator per
-// head in tensor memory, flushed with atomic adds at the end of the block). The conv's own backward then runs on du.
+// and forms du = dy W_h^T (the key stream summed over the group in registers) and dW_h += u^T dy (accumulators of two
+// heads at a time in tensor memory, flushed with atomic adds). The conv's own backward then runs on du.
 // Tiles are unswizzled 8x8 core matrices with every 8-column slab contiguous (see gla_tc.cu): W_h serves as the
 // MN-major B of the forward mix and, without a second copy, as the K-major B of dy W_h^T.
 #include <cuda.h>
@@ -247,14 +247,14 @@ __global__ void __launch_bounds__(128) convmix_tc_fwd_kernel(const CArgs a) {
 // Backward through phi and the mix for head width 64: du_q [B,T,H,64], du_k [B,T,Hkv,64] (fp32), dW [H,64,64] (atomic adds
 // into a zeroed array). TG: type of the incoming gradients d_qdot, d_kdot.
 template <typename TG>
-__global__ void __launch_bounds__(128) convmix_tc_bwd_kernel(const CArgs a) {
+__global__ void __launch_bounds__(128, 2) convmix_tc_bwd_kernel(const CArgs a) {
   constexpr int D = 64;
   using L = Lay<D>;
   extern __shared__ __align__(128) uint8_t sg[];
   constexpr uint32_t OFF_WT = 0, OFF_U = OFF_WT + L::TILE_W, OFF_DY = OFF_U + L::TILE_U, OFF_DYL = OFF_DY + L::TILE_U;
   constexpr uint32_t OFF_RAW = OFF_DYL + L::TILE_U + 2048, OFF_TAPS = OFF_RAW + (L::RAW_BYTES + 15) / 16 * 16;
   constexpr uint32_t OFF_BAR = OFF_TAPS + D * 4 * 4;
-  constexpr uint32_t COL_Y = 0, COL_DW = 64, TMEM_COLS = 512;
+  constexpr uint32_t COL_Y = 0, COL_DW = 64, TMEM_COLS = 256;  // Y / du, and the dW accumulators of two heads at a time
   const uint32_t sb = smem_u32(sg);
   const int tid = threadIdx.x, warp = tid >> 5;
   volatile int* const s_flags = reinterpret_cast<volatile int*>(sg + OFF_BAR + 16);
@@ -361,7 +361,7 @@ __global__ void __launch_bounds__(128) convmix_tc_bwd_kernel(const CArgs a) {
         const uint32_t id_dw = instr_desc(128, D, FMT_F16, MAJOR_MN, MAJOR_MN);
         const uint64_t ua = mview(sb + OFF_U, L::SLAB_U), yb = mview(sb + OFF_DY, L::SLAB_U);
         for (int kk = 0; kk < TT / 16; ++kk)
-          mma_f16(tmem + COL_DW + 64 * g, dadv(ua, 256 * kk), dadv(yb, 256 * kk), id_dw, (stream > 0 || kk > 0) ? 1u : 0u);
+          mma_f16(tmem + COL_DW + 64 * (g & 1), dadv(ua, 256 * kk), dadv(yb, 256 * kk), id_dw, (stream > 0 || kk > 0) ? 1u : 0u);
         mma_commit(sb + OFF_BAR);
       }
       wt.wait();
@@ -385,26 +385,29 @@ __global__ void __launch_bounds__(128) convmix_tc_bwd_kernel(const CArgs a) {
       __syncthreads();
       tc_fence_after_sync();
     }
+    // dW of the last two heads (or the last one): row c of each accumulator is owned by thread c
+    if (((g & 1) || g == G - 1) && warp < 2 && a.dW) {
+#pragma unroll 1
+      for (int gg = g & ~1; gg <= g; ++gg) {
+        float r[32];
+#pragma unroll 1
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          tmem_ld32(lane_base + COL_DW + 64 * (gg & 1) + c0, r);
+          tmem_wait_ld();
+          float* dst = a.dW + ((size_t)(j * G + gg) * D + tid) * D + c0;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) atomicAdd(dst + i, r[i]);
+        }
+      }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
   }
   if (valid) {
     float* dst = a.du_k + (((size_t)b * a.T + t) * a.Hkv + j) * D;
 #pragma unroll
     for (int c0 = 0; c0 < D; c0 += 8) store_row8(dst + c0, duk + c0);
-  }
-  // dW of the group's heads: row c of each accumulator is owned by thread c
-  if (warp < 2 && a.dW) {
-#pragma unroll 1
-    for (int g = 0; g < G; ++g) {
-      float r[32];
-#pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
-        tmem_ld32(lane_base + COL_DW + 64 * g + c0, r);
-        tmem_wait_ld();
-        float* dst = a.dW + ((size_t)(j * G + g) * D + tid) * D + c0;
-#pragma unroll
-        for (int i = 0; i < 32; ++i) atomicAdd(dst + i, r[i]);
-      }
-    }
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -436,8 +439,8 @@ bool convmix_tc_fwd_supported(const lawcat_params& p) {
          p.conv_k <= ctc::HALO + 1 && p.B > 0 && p.T > 0;
 }
 bool convmix_tc_bwd_supported(const lawcat_params& p) {
-  return p.dtype == LAWCAT_BF16 && p.d_k == 64 && p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= ctc::HALO + 1 &&
-         p.H / p.H_kv <= 4 && p.B > 0 && p.T > 0;
+  return p.dtype == LAWCAT_BF16 && p.d_k == 64 && p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= ctc::HALO + 1 && p.B > 0 &&
+         p.T > 0;
 }
 
 static ctc::CArgs convmix_tc_args(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,

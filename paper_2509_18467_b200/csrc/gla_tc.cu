@@ -788,13 +788,26 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       GTL(16);
       // ---- gate gradient: reverse running sum over the chunk's tokens on top of what crosses its end, then the derivative
       // of the log-decay ----------------------------------------------------------------------------------------------------
-      if (tid < D) {
-        const int c = tid;
-        float acc = carry;
-        for (int t = C - 1; t >= 0; --t) {
-          acc += s_dt[t * D + c];   // (rows past the end hold zeros: their operands were zero)
-          s_dt[t * D + c] = acc;
+      {
+        // thread = (channel, quarter of the chunk): running sums inside the quarter, then the totals of the quarters behind
+        // it and what crosses the chunk's end on top (rows past the end hold zeros: their operands were zero)
+        const int c = tid & (D - 1), seg = tid >> 6;
+        float* const s_tot = s_ft;  // [4][D]: s_ft, s_dm, s_e63, s_dC are free until the next chunk's gate pass
+        if (tid < D) s_row[tid] = carry;
+        float v[16], acc = 0.f;
+#pragma unroll
+        for (int i = 15; i >= 0; --i) {
+          acc += s_dt[(seg * 16 + i) * D + c];
+          v[i] = acc;
         }
+        s_tot[seg * D + c] = acc;
+        __syncthreads();
+        float off = s_row[c];
+#pragma unroll
+        for (int s2 = 3; s2 >= 1; --s2)
+          if (s2 > seg) off += s_tot[s2 * D + c];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) s_dt[(seg * 16 + i) * D + c] = v[i] + off;
       }
       __syncthreads();
       if (a.gate_dim == 1) {
