@@ -103,6 +103,15 @@ int lawcat_trace_begin(void);
 int lawcat_trace_end(char* buf, size_t buf_bytes);
 
 /*
+ * Test hook (no counterpart in the paper). Every device-side wait of the tensor-core layer kernels is bounded: after
+ * `cycles` clock cycles (default about two seconds) a waiting role gives up, the block leaves its loops, lets its
+ * copies land, frees its tensor memory and returns, and dev_status receives LAWCAT_ERR_TIMEOUT. This call sets the bound
+ * for the launches that follow (0 restores the default), so that a test can make a wait run out without faulting or
+ * hanging anything. Host-side, process-wide, not meant for production code.
+ */
+void lawcat_test_set_wait_limit(long long cycles);
+
+/*
  * Causal depthwise conv on q and k (Section 4.1: qtilde_t = sum_delta w_delta q_{t-delta}), then, when W is not
  * NULL, the shared per-head linear layer and phi (Section 4.1; Section 4.2 defines qdot, kdot).
  *   q [B,T,H,d_k]  k [B,T,H_kv,d_k]  w_q [H*d_k,conv_k]  w_k [H_kv*d_k,conv_k]  W [H,d_k,d_k] or NULL

@@ -21,7 +21,7 @@ GATE_LOGITS, GATE_LOGDECAY = 0, 1
 OP_CONV_FWD, OP_CONV_BWD, OP_GLA_FWD, OP_GLA_BWD, OP_LAYER_FWD, OP_DECODE_STEP, OP_LAYER_BWD = range(7)
 
 EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "lawcat_launch_count",
-           "lawcat_trace_begin", "lawcat_trace_end", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
+           "lawcat_trace_begin", "lawcat_trace_end", "lawcat_test_set_wait_limit", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
            "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_layer_bwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
            "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc"]
 
@@ -109,6 +109,13 @@ def trace_end() -> dict:
         name, n, ms = line.split()
         out[name] = (int(n), float(ms))
     return out
+
+
+def test_set_wait_limit(cycles: int) -> None:
+    """Test hook: bound (clock cycles) of the device-side waits of the tensor-core layer kernels; 0 = default."""
+    f = lib().lawcat_test_set_wait_limit
+    f.argtypes, f.restype = [ctypes.c_longlong], None
+    f(cycles)
 
 
 def workspace_bytes(p: Params, op: int) -> int:

@@ -1,4 +1,5 @@
 // Host side of the chunkwise tensor-core layer forward: tensor maps, segment split, launches.
+#include <atomic>
 #include <mutex>
 
 #include "layer_tc_kernel.cuh"
@@ -117,6 +118,9 @@ static TcPlan layer_tc_plan(const lawcat_params& p) {
 
 int layer_tc_segments(const lawcat_params& p) { return layer_tc_plan(p).nseg; }
 
+// Limit of the kernels' device-side waits in clock cycles (about two seconds); a test hook may shorten it.
+static std::atomic<long long> g_wait_limit{4000000000LL};
+
 size_t layer_tc_workspace_bytes(const lawcat_params& p) {
   const TcPlan pl = layer_tc_plan(p);
   if (pl.nseg == 1) return 0;
@@ -158,6 +162,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   a.dev_status = c.dev_status;
   a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k;
   a.gate_mode = p.gate_mode; a.normalize = p.normalize; a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps;
+  a.wait_limit = g_wait_limit.load();
   const TcPlan pl = layer_tc_plan(p);
   const int nseg = pl.nseg;
   a.nseg = nseg;
@@ -245,6 +250,14 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
 }
 
 }  // namespace lawcat
+
+// Test hook: the limit (clock cycles) of every bounded device-side wait of the tensor-core layer kernels launched from
+// now on; 0 restores the default. A limit of a few cycles makes the first unsatisfied wait give up, which exercises the
+// path that reports LAWCAT_ERR_TIMEOUT (nothing faults or hangs: the block leaves its loops, lets its copies land, frees
+// its tensor memory and returns).
+extern "C" void lawcat_test_set_wait_limit(long long cycles) {
+  lawcat::g_wait_limit.store(cycles > 0 ? cycles : 4000000000LL);
+}
 
 #ifdef LAWCAT_TIMELINE
 // (profiling builds only) copies the clock stamps of the last layer-kernel launch to the host

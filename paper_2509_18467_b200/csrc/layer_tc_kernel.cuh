@@ -145,6 +145,7 @@ struct TcArgs {
   int gate_mode;
   int normalize;         // 1: Eq. 8; 0: the numerator alone (the query features then carry their softmax normalizer)
   float inv_tau, eps;
+  long long wait_limit;  // clock cycles a device-side wait may take before the block gives up (about 2 s by default)
 };
 
 __device__ __forceinline__ void unpack8(const uint4& v, float* f) {
@@ -207,15 +208,16 @@ __device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool flag) {
 }
 
 // Bounded wait that also gives up as soon as another role has raised the abort flag.
-__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
+  const int batch = limit < 1000000LL ? 1 : 256;  // polls between two looks at the clock (a short limit is looked at often)
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 256; ++i)
+    for (int i = 0; i < batch; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > 4000000000LL) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       return false;
     }
@@ -228,7 +230,7 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
 // parity barrier l is waited with. All 32 lanes must call it together. A lane stops polling once its barrier's phase has
 // completed: the barrier may run on into its next phase while the other lanes still wait.
 __device__ __forceinline__ bool wait_set_or_abort(uint32_t bar0, uint32_t mask, uint32_t parities, int lane,
-                                                  volatile int* abort_flag) {
+                                                  volatile int* abort_flag, long long limit) {
   const uint32_t b = bar0 + 8u * (uint32_t)lane, par = (parities >> lane) & 1u;
   bool ok = ((mask >> lane) & 1u) == 0u || mbar_try_wait(b, par);
   if (__all_sync(0xffffffffu, ok)) {
@@ -236,9 +238,10 @@ __device__ __forceinline__ bool wait_set_or_abort(uint32_t bar0, uint32_t mask, 
     return true;
   }
   const long long t0 = clock64();
+  const int batch = limit < 1000000LL ? 1 : 256;
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 256; ++i) {
+    for (int i = 0; i < batch; ++i) {
       if (!ok) ok = mbar_try_wait(b, par);
       if (__all_sync(0xffffffffu, ok)) {
         __syncwarp();
@@ -246,7 +249,7 @@ __device__ __forceinline__ bool wait_set_or_abort(uint32_t bar0, uint32_t mask, 
       }
     }
     bool stop = *abort_flag != 0;
-    if (!stop && clock64() - t0 > 4000000000LL) {
+    if (!stop && clock64() - t0 > limit) {
       *abort_flag = 1;
       stop = true;
     }
@@ -411,17 +414,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   tc_fence_after_sync();
 
 #define WAIT(b, par)                                     \
-  if (!wait_or_abort(bar(b), (uint32_t)(par), s_abort)) break
+  if (!wait_or_abort(bar(b), (uint32_t)(par), s_abort, a.wait_limit)) break
   // for roles with barriers of their own: remember the failure, skip the work, leave at the role's next OR-barrier
 #define WAITF(b, par)                                    \
-  if (!fail && !wait_or_abort(bar(b), (uint32_t)(par), s_abort)) fail = true
+  if (!fail && !wait_or_abort(bar(b), (uint32_t)(par), s_abort, a.wait_limit)) fail = true
   // several barriers at once (whole warp): BIT(barrier) selects, PAR(barrier, parity) gives its parity
 #define BIT(b) (1u << (b))
 #define PAR(b, par) ((uint32_t)(par) << (b))
 #define WAITSET(mask, pars)                              \
-  if (!wait_set_or_abort(bar(0), (mask), (pars), lane, s_abort)) break
+  if (!wait_set_or_abort(bar(0), (mask), (pars), lane, s_abort, a.wait_limit)) break
 #define WAITSETF(mask, pars)                             \
-  if (!fail && !wait_set_or_abort(bar(0), (mask), (pars), lane, s_abort)) fail = true
+  if (!fail && !wait_set_or_abort(bar(0), (mask), (pars), lane, s_abort, a.wait_limit)) fail = true
 
   if (warp == TMA_WARP) {
     // ================================================================================================ TMA producer
@@ -489,7 +492,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mma_commit(bar(B_MMA1));
       };
       bool ok = nchunks > 0;
-      if (ok) ok = wait_set_or_abort(bar(0), BIT(B_U_FULL), 0u, lane, s_abort);
+      if (ok) ok = wait_set_or_abort(bar(0), BIT(B_U_FULL), 0u, lane, s_abort, a.wait_limit);
       if (ok && lane == 0) {
         tc_fence_after_sync();
         issue_mma1();
@@ -788,7 +791,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       TL(warp == 0 ? 3 : 4, 9, n, (warp == 0 || warp == 2) && lane == 0);
     }
     if (MODE == 0 && nchunks > 0 && !fail && !*s_abort &&
-        wait_or_abort(bar(B_MMA3), (uint32_t)((nchunks - 1) & 1), s_abort))
+        wait_or_abort(bar(B_MMA3), (uint32_t)((nchunks - 1) & 1), s_abort, a.wait_limit))
       out_pass(nchunks - 1);
   } else {
     // ================================================================================================ row warps
@@ -857,6 +860,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // ---- phi, reading sweeps ----------------------------------------------------------------------------------------
       if (phi_on) {
         WAITF(B_MMA1, p);
+        fail = __any_sync(0xffffffffu, fail);  // (the collective waits below need the whole warp)
         TL(warp == 8 ? 1 : 2, 2, n, (warp == 8 || warp == 10) && lane == 0);
         tc_fence_after_sync();
         float m = -INFINITY;
@@ -1080,7 +1084,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
     if (MODE == 0 && is_q && nchunks > 0) mask_chunk(nchunks - 1);
     // ---- final state -------------------------------------------------------------------------------------------------
-    if (!fail && !*s_abort && (nchunks == 0 || wait_or_abort(bar(B_MMA2), (uint32_t)((nchunks - 1) & 1), s_abort))) {
+    if (!fail && !*s_abort && (nchunks == 0 || wait_or_abort(bar(B_MMA2), (uint32_t)((nchunks - 1) & 1), s_abort, a.wait_limit))) {
       tc_fence_after_sync();
       const int c = r128;
       if (a.dtot != nullptr && ch == 0 && c < dh) a.dtot[seg_idx * dh + c] = dsum;
