@@ -184,6 +184,27 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
                      int* dev_status);
 
 /*
+ * lawcat_layer_fwd over PACKED sequences of different lengths (batched and chunked prefill of a serving loop; the paper
+ * points to the streaming use of the constant-size state in Section 6). The tokens of nseq sequences lie back to back
+ * along T: p->B must be 1, p->T is the total, and sequence i covers tokens [cu_seqlens[i], cu_seqlens[i+1]).
+ *   cu_seqlens: HOST array of nseq + 1 non-decreasing ints, cu_seqlens[0] = 0, cu_seqlens[nseq] = p->T
+ *   q, k, v, gate, o: as in lawcat_layer_fwd with B = 1
+ *   S0 [nseq,H,d_k,d_v], z0 [nseq,H,d_k], cache_q_in [nseq,conv_k-1,H*d_k], cache_k_in [nseq,conv_k-1,H_kv*d_k]:
+ *     what each sequence starts from (nullable: every sequence starts from nothing, i.e. the state is reset at every
+ *     boundary; a chunk of a longer sequence passes the state and caches its previous chunk returned)
+ *   S_T, z_T, cache_q_out, cache_k_out: the same per sequence after its last token (nullable)
+ * No token of one sequence reaches another: neither through the conv (its first conv_k - 1 tokens see the sequence's own
+ * cache or zeros) nor through the state. An empty sequence hands its state and caches through. The sequences are
+ * enqueued one after the other on `stream`, sharing `ws` (lawcat_layer_fwd_varlen_workspace_bytes: the largest need).
+ */
+size_t lawcat_layer_fwd_varlen_workspace_bytes(const lawcat_params* p, const int32_t* cu_seqlens, int nseq);
+int lawcat_layer_fwd_varlen(const lawcat_params* p, const int32_t* cu_seqlens, int nseq, const void* q, const void* k,
+                            const void* v, const void* gate, const void* w_q, const void* w_k, const void* W,
+                            const void* cache_q_in, const void* cache_k_in, const float* S0, const float* z0, void* o,
+                            void* cache_q_out, void* cache_k_out, float* S_T, float* z_T, void* ws, size_t ws_bytes,
+                            void* stream, int* dev_status);
+
+/*
  * Backward of the whole layer (Fig. 1) for an upstream gradient dO [B,T,H,d_v]: the layer-wise distillation step of
  * Section 5.1 in one call (chain rule on conv -> mix -> phi -> Eq. 4, Eq. 8; the paper prints no formulas). The features
  * qdot, kdot are recomputed from q, k and never stored in the storage type: on the tensor-core path (bf16, d_k = d_v =

@@ -22,7 +22,8 @@ OP_CONV_FWD, OP_CONV_BWD, OP_GLA_FWD, OP_GLA_BWD, OP_LAYER_FWD, OP_DECODE_STEP, 
 
 EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "lawcat_launch_count",
            "lawcat_trace_begin", "lawcat_trace_end", "lawcat_test_set_wait_limit", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
-           "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_layer_bwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
+           "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_layer_fwd_varlen_workspace_bytes",
+           "lawcat_layer_fwd_varlen", "lawcat_layer_bwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
            "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc"]
 
 
@@ -213,6 +214,35 @@ def lawcat_layer_fwd(p: Params, q, k, v, gate, w_q, w_k, W, cache_q=None, cache_
     ws, nb = _ws(p, OP_LAYER_FWD, ws, dev)
     _call("lawcat_layer_fwd", p, [q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0, o, cq, ck, S_T, z_T], ws, nb,
           stream, dev_status)
+    return dict(o=o, cache_q=cq, cache_k=ck, S_T=S_T, z_T=z_T)
+
+
+def lawcat_layer_fwd_varlen(p: Params, cu_seqlens, q, k, v, gate, w_q, w_k, W, cache_q=None, cache_k=None, S0=None, z0=None,
+                            stream=None, dev_status=None):
+    """Packed sequences (B = 1): cu_seqlens is a host sequence of nseq + 1 token offsets. Returns dict(o, cache_q, cache_k,
+    S_T, z_T) with the state outputs per sequence."""
+    L = lib()
+    nseq = len(cu_seqlens) - 1
+    cu = (ctypes.c_int32 * (nseq + 1))(*[int(x) for x in cu_seqlens])
+    dt, dev = torch_dtype(p), q.device
+    o = torch.empty(1, p.T, p.H, p.d_v, dtype=dt, device=dev)
+    S_T = torch.empty(nseq, p.H, p.d_k, p.d_v, dtype=torch.float32, device=dev)
+    z_T = torch.empty(nseq, p.H, p.d_k, dtype=torch.float32, device=dev)
+    cq = torch.empty(nseq, p.conv_k - 1, p.H * p.d_k, dtype=dt, device=dev)
+    ck = torch.empty(nseq, p.conv_k - 1, p.H_kv * p.d_k, dtype=dt, device=dev)
+    L.lawcat_layer_fwd_varlen_workspace_bytes.restype = ctypes.c_size_t
+    L.lawcat_layer_fwd_varlen_workspace_bytes.argtypes = [ctypes.POINTER(Params), ctypes.c_void_p, ctypes.c_int]
+    need = int(L.lawcat_layer_fwd_varlen_workspace_bytes(ctypes.byref(p), cu, nseq))
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    f = L.lawcat_layer_fwd_varlen
+    f.restype = ctypes.c_int
+    f.argtypes = [ctypes.POINTER(Params), ctypes.c_void_p, ctypes.c_int] + [ctypes.c_void_p] * 17 + \
+                 [ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p]
+    st = f(ctypes.byref(p), cu, nseq, *[_ptr(t) for t in (q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0, o, cq, ck,
+                                                          S_T, z_T)], _ptr(ws), ws.numel(), _stream(stream),
+           _ptr(dev_status))
+    if st != 0:
+        raise LawcatError(st, "lawcat_layer_fwd_varlen")
     return dict(o=o, cache_q=cq, cache_k=ck, S_T=S_T, z_T=z_T)
 
 

@@ -224,12 +224,79 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
     if ((r = launch_layer_tc(c, q, k, v, gate, w_q, w_k, W, cache_q_in, cache_k_in, S0, z0, o, S_T, z_T, ws))) return r;
     return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
   }
-  // exact path: conv + mix + phi into fp32 scratch, then the recurrent GLA
   float* qdot = (float*)ws;
   float* kdot = (float*)((char*)ws + align_up(sizeof(float) * elems(p, p->H, p->d_k), 256));
+  // The feature maps of Section 2 other than the softmax (1 + ELU, identity) on head width 64: tensor-core conv + mix +
+  // phi into fp32 scratch, then the chunkwise tensor-core attention on those features.
+  if ((size_t)p->B * p->T != 0 && p->phi != LAWCAT_PHI_SOFTMAX && p->chunk != 1 && convmix_tc_fwd_supported(*p) &&
+      gla_tc_supported(*p)) {
+    if ((r = launch_convmix_tc_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true))) return r;
+    if ((r = launch_gla_fwd_tc(c, qdot, kdot, v, gate, S0, z0, o, nullptr, S_T, z_T, true))) return r;
+    return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
+  }
+  // exact path: conv + mix + phi into fp32 scratch, then the recurrent GLA
   if ((r = launch_convmix_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true, true))) return r;
   if ((r = launch_gla_fwd_rec(c, qdot, kdot, true, v, gate, S0, z0, o, nullptr, S_T, z_T))) return r;
   return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
+}
+
+size_t lawcat_layer_fwd_varlen_workspace_bytes(const lawcat_params* p, const int32_t* cu_seqlens, int nseq) {
+  if (check_params(p, true) != LAWCAT_OK || !cu_seqlens || nseq < 0) return 0;
+  size_t need = 0;
+  for (int i = 0; i < nseq; ++i) {
+    lawcat_params pi = *p;
+    pi.B = 1;
+    pi.T = cu_seqlens[i + 1] - cu_seqlens[i];
+    if (pi.T <= 0) continue;
+    const size_t n = lawcat_workspace_bytes(&pi, LAWCAT_OP_LAYER_FWD);
+    if (n > need) need = n;
+  }
+  return need;
+}
+
+int lawcat_layer_fwd_varlen(const lawcat_params* p, const int32_t* cu_seqlens, int nseq, const void* q, const void* k,
+                            const void* v, const void* gate, const void* w_q, const void* w_k, const void* W,
+                            const void* cache_q_in, const void* cache_k_in, const float* S0, const float* z0, void* o,
+                            void* cache_q_out, void* cache_k_out, float* S_T, float* z_T, void* ws, size_t ws_bytes,
+                            void* stream, int* dev_status) {
+  int r = check_params(p, true);
+  if (r) return r;
+  if (p->B != 1 || !cu_seqlens || nseq < 0) return LAWCAT_ERR_INVALID_ARG;
+  if (cu_seqlens[0] != 0 || cu_seqlens[nseq] != p->T) return LAWCAT_ERR_INVALID_ARG;
+  for (int i = 0; i < nseq; ++i)
+    if (cu_seqlens[i + 1] < cu_seqlens[i]) return LAWCAT_ERR_INVALID_ARG;
+  if (ws_bytes < lawcat_layer_fwd_varlen_workspace_bytes(p, cu_seqlens, nseq)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
+  const size_t es = p->dtype == LAWCAT_F32 ? 4 : 2;
+  const size_t nS = (size_t)p->H * p->d_k * p->d_v, nz = (size_t)p->H * p->d_k;
+  const size_t ncq = (size_t)(p->conv_k - 1) * p->H * p->d_k * es, nck = (size_t)(p->conv_k - 1) * p->H_kv * p->d_k * es;
+  auto at = [](const void* base, size_t bytes) -> const void* { return base ? (const char*)base + bytes : nullptr; };
+  auto atw = [](void* base, size_t bytes) -> void* { return base ? (char*)base + bytes : nullptr; };
+  cudaStream_t st = (cudaStream_t)stream;
+  for (int i = 0; i < nseq; ++i) {
+    const size_t t0 = (size_t)cu_seqlens[i];
+    lawcat_params pi = *p;
+    pi.T = cu_seqlens[i + 1] - cu_seqlens[i];
+    const float* S0i = S0 ? S0 + i * nS : nullptr;
+    const float* z0i = z0 ? z0 + i * nz : nullptr;
+    float* STi = S_T ? S_T + i * nS : nullptr;
+    float* zTi = z_T ? z_T + i * nz : nullptr;
+    if (pi.T == 0) {  // an empty sequence hands its state and caches through
+      auto pass = [&](void* dst, const void* src, size_t bytes) -> bool {
+        if (!dst || !bytes) return true;
+        return (src ? cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, st) : cudaMemsetAsync(dst, 0, bytes, st)) == cudaSuccess;
+      };
+      if (!pass(STi, S0i, nS * 4) || !pass(zTi, z0i, nz * 4) || !pass(atw(cache_q_out, i * ncq), at(cache_q_in, i * ncq), ncq) ||
+          !pass(atw(cache_k_out, i * nck), at(cache_k_in, i * nck), nck))
+        return LAWCAT_ERR_CUDA;
+      continue;
+    }
+    r = lawcat_layer_fwd(&pi, at(q, t0 * p->H * p->d_k * es), at(k, t0 * p->H_kv * p->d_k * es), at(v, t0 * p->H_kv * p->d_v * es),
+                         at(gate, t0 * p->H * p->gate_dim * es), w_q, w_k, W, at(cache_q_in, i * ncq), at(cache_k_in, i * nck),
+                         S0i, z0i, atw(o, t0 * p->H * p->d_v * es), atw(cache_q_out, i * ncq), atw(cache_k_out, i * nck), STi,
+                         zTi, ws, ws_bytes, stream, dev_status);
+    if (r) return r;
+  }
+  return LAWCAT_OK;
 }
 
 int lawcat_layer_bwd(const lawcat_params* p, const void* q, const void* k, const void* v, const void* gate,

@@ -86,7 +86,7 @@ bool gla_tc_supported(const lawcat_params& p);
 bool gla_tc_bwd_supported(const lawcat_params& p);
 size_t gla_tc_bwd_workspace_bytes(const lawcat_params& p);
 int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
-                      const float* z0, void* o, float* den, float* S_T, float* z_T);
+                      const float* z0, void* o, float* den, float* S_T, float* z_T, bool feat_f32 = false);
 int launch_gla_bwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
                       const float* z0, const void* dO, void* d_qdot, void* d_kdot, void* dv, void* dgate, void* ws,
                       bool feat_f32);

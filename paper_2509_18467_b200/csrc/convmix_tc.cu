@@ -3,8 +3,8 @@
 //
 // Forward: one thread block = one (batch, query head, tile of 128 tokens), both streams one after the other (they share
 // W_h): raw rows (with the conv_k - 1 rows in front) into shared memory, depthwise causal conv in fp32 -> fp16 operand,
-// Y = u W_h as one tcgen05 product per 16 channels (fp32 accumulator in tensor memory), softmax over a row by the thread
-// that owns the row's TMEM lane, 16-bit or fp32 store.
+// Y = u W_h as one tcgen05 product per 16 channels (fp32 accumulator in tensor memory), phi (softmax over the row, or the
+// elementwise 1 + ELU / identity of Section 2) by the thread that owns the row's TMEM lane, 16-bit or fp32 store.
 // Backward (head width 64): one block = one (batch, key head, tile); for each query head of
 // the group and each stream it recomputes u and p = softmax(u W_h), applies the softmax Jacobian dy = p (dp - p . dp),
 // and forms du = dy W_h^T (the key stream summed over the group in registers) and dW_h += u^T dy (accumulators of two
@@ -70,7 +70,7 @@ struct CArgs {
   const void *d_qdot, *d_kdot;       // backward inputs (bf16 or fp32)
   float *du_q, *du_k, *dW;           // backward outputs: d(conv out) per stream (fp32), dW (fp32, atomic adds)
   int* dev_status;
-  int B, T, H, Hkv, K;
+  int B, T, H, Hkv, K, phi;
 };
 
 // one mbarrier, bounded wait (a product batch completes within microseconds; 2e8 cycles is about a tenth of a second)
@@ -204,8 +204,25 @@ __global__ void __launch_bounds__(128) convmix_tc_fwd_kernel(const CArgs a) {
       mma_commit(sb + OFF_BAR);
     }
     wt.wait();
-    // softmax over the row this thread owns (row = token t0 + tid)
-    {
+    // phi over the row this thread owns (row = token t0 + tid): softmax, or elementwise 1 + ELU / identity
+    if (a.phi != LAWCAT_PHI_SOFTMAX) {
+      const int t = t0 + tid;
+      float y[32];
+      TO* out = reinterpret_cast<TO*>(stream ? a.kdot : a.qdot) + (((size_t)b * a.T + t) * a.H + h) * D;
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        tmem_ld32(lane_base + c0, y);
+        tmem_wait_ld();
+        if (a.phi == LAWCAT_PHI_ELU1) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) y[i] = y[i] > 0.f ? y[i] + 1.f : __expf(y[i]);
+        }
+        if (t < a.T) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) store_row8(out + c0 + i, y + i);
+        }
+      }
+    } else {
       const int t = t0 + tid;
       float y[32], m = -INFINITY, sum = 0.f;
 #pragma unroll 1
@@ -435,8 +452,7 @@ static int raise_smem(K kernel, uint32_t bytes) {
 }  // namespace ctc
 
 bool convmix_tc_fwd_supported(const lawcat_params& p) {
-  return p.dtype == LAWCAT_BF16 && (p.d_k == 64 || p.d_k == 128) && p.phi == LAWCAT_PHI_SOFTMAX &&
-         p.conv_k <= ctc::HALO + 1 && p.B > 0 && p.T > 0;
+  return p.dtype == LAWCAT_BF16 && (p.d_k == 64 || p.d_k == 128) && p.conv_k <= ctc::HALO + 1 && p.B > 0 && p.T > 0;
 }
 bool convmix_tc_bwd_supported(const lawcat_params& p) {
   return p.dtype == LAWCAT_BF16 && p.d_k == 64 && p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= ctc::HALO + 1 && p.B > 0 &&
@@ -450,7 +466,7 @@ static ctc::CArgs convmix_tc_args(const Ctx& c, const void* q, const void* k, co
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.w_q = (const bf16*)w_q; a.w_k = (const bf16*)w_k; a.W = (const bf16*)W;
   a.cache_q = (const bf16*)cache_q; a.cache_k = (const bf16*)cache_k;
   a.dev_status = c.dev_status;
-  a.B = p.B; a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k;
+  a.B = p.B; a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k; a.phi = p.phi;
   return a;
 }
 

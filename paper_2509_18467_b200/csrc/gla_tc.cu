@@ -393,7 +393,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       float inv = 0.f, dl = 0.f;
       if (r < nvalid) {
         const size_t tq = ((size_t)b * a.T + t0 + r) * a.H + h, tv = ((size_t)b * a.T + t0 + r) * a.Hkv + j;
-        if (BWD && a.feat_f32) {
+        if (a.feat_f32) {
           const float* fq = reinterpret_cast<const float*>(a.qdot) + tq * D + o8 * 8;
           const float* fk = reinterpret_cast<const float*>(a.kdot) + tq * D + o8 * 8;
           const float4 q0 = *reinterpret_cast<const float4*>(fq), q1 = *reinterpret_cast<const float4*>(fq + 4);
@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
           dl = a.ws_delta[tq];
         }
       }
-      if (!(BWD && a.feat_f32) || r >= nvalid) { unpack8b(zq, q); unpack8b(zk, k); }
+      if (!a.feat_f32 || r >= nvalid) { unpack8b(zq, q); unpack8b(zk, k); }
       unpack8b(zv, vv);
       const float4 xa = *reinterpret_cast<const float4*>(s_x + r * D + o8 * 8), xb = *reinterpret_cast<const float4*>(s_x + r * D + o8 * 8 + 4);
       x[0] = xa.x; x[1] = xa.y; x[2] = xa.z; x[3] = xa.w; x[4] = xb.x; x[5] = xb.y; x[6] = xb.z; x[7] = xb.w;
@@ -911,14 +911,14 @@ static gtc::GArgs gla_tc_args(const Ctx& c) {
 }
 
 int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const void* v, const void* gate, const float* S0,
-                      const float* z0, void* o, float* den, float* S_T, float* z_T) {
+                      const float* z0, void* o, float* den, float* S_T, float* z_T, bool feat_f32) {
   using namespace gtc;
   const lawcat_params& p = *c.p;
   int r = set_smem_once();
   if (r) return r;
   GArgs a = gla_tc_args(c);
   a.qdot = qdot; a.kdot = kdot; a.v = (const bf16*)v; a.gate = (const bf16*)gate;
-  a.S0 = S0; a.z0 = z0; a.o = (bf16*)o; a.den = den; a.S_T = S_T; a.z_T = z_T;
+  a.S0 = S0; a.z0 = z0; a.o = (bf16*)o; a.den = den; a.S_T = S_T; a.z_T = z_T; a.feat_f32 = feat_f32 ? 1 : 0;
   LaunchScope _ls("gla_tc_fwd", c.stream);
   gla_tc_kernel<false><<<p.B * p.H, THREADS, SMEM_FWD, c.stream>>>(a);
   LAWCAT_CHECK_LAUNCH();

@@ -97,3 +97,28 @@ def test_log_decay_gate_mode(api):
 def test_eps_and_numerator_only(api):
     run(api, shape(1, 150, 2, 1, 67), False, eps=0.5)
     run(api, shape(1, 150, 2, 1, 68), True, normalize=0)
+
+
+@pytest.mark.parametrize("phi,T,with_state", [(1, 65, False), (1, 300, True), (1, 1223, True), (2, 200, False)])
+def test_layer_forward_with_the_elementwise_feature_maps(api, phi, T, with_state):
+    """The feature maps of Section 2 other than the softmax, phi = 1 + ELU (and the identity, with a positive mix so that
+    the features stay positive), through lawcat_layer_fwd on head width 64: tensor-core conv + mix + phi, then the
+    chunkwise tensor-core attention on fp32 features."""
+    names = ["q", "k", "v", "gate", "w_q", "w_k", "W"]
+    s = shape(2, T, 4, 2, 69)
+    extra = ["S0", "z0", "cache_q", "cache_k"] if with_state else []
+    x = I.make(s, names + extra)
+    if phi == 2:  # identity: keep the features (hence the denominators) positive
+        for n in ("q", "k", "w_q", "w_k", "W") + (("cache_q", "cache_k") if with_state else ()):
+            x[n] = I.round_to_bf16(np.abs(x[n]))
+    d = {n: api.to_device(v, "f32" if n in ("S0", "z0") else "bf16") for n, v in x.items()}
+    api.trace_begin()
+    r = api.lawcat_layer_fwd(P(api, s, phi=phi), *[d[n] for n in names], d.get("cache_q"), d.get("cache_k"), d.get("S0"),
+                             d.get("z0"))
+    kernels = api.trace_end()
+    assert "convmix_tc_fwd" in kernels and "gla_tc_fwd" in kernels, kernels
+    ref = O.layer_fwd(oracle_params(s, phi=phi), *[x[n] for n in names], x.get("cache_q"), x.get("cache_k"), x.get("S0"),
+                      x.get("z0"))
+    check(r["o"], ref["o"], "bf16", "o")
+    check(r["S_T"], ref["S_T"], "bf16", "S_T", f32_store=True)
+    check(r["z_T"], ref["z_T"], "bf16", "z_T", f32_store=True)
