@@ -100,19 +100,28 @@ def alg_flops_per_step(kind: str, s: I.LayerShape) -> float:
 
 
 def kernel_bytes_per_step(name: str, kind: str, s: I.LayerShape) -> float:
-    """Algorithmic bytes of ONE launch of kernel `name` (what that kernel alone has to move)."""
+    """Algorithmic bytes of ONE launch of kernel `name`: what that kernel's own interface has to move."""
     b, tok = io_bytes_per_token(s), s.B * s.T
-    f32_feat = 4 * 2 * s.H * s.d_k
+    f32_feat = 4 * 2 * s.H * s.d_k            # qdot and kdot in fp32
+    f32_dv = 4 * s.H * s.d_v                  # dv per query head in fp32 (before the group reduce)
     table = {
         "gla_fwd_rec": (f32_feat if kind == "prefill" else 2 * b["q"]) + b["v"] + b["gate"] + b["o"],
         "convmix_fwd": b["q"] + b["k"] + (f32_feat if kind == "prefill" else 2 * b["q"]),
-        "decode_state": None, "decode_features": None,
+        "convmix_tc_fwd": b["q"] + b["k"] + f32_feat,
+        # chunkwise backward inside layer_bwd: fp32 features in, fp32 feature gradients out, v, gate, dO in, dgate out,
+        # dv per query head out
+        "gla_tc_bwd": 2 * f32_feat + b["v"] + b["gate"] + b["o"] + b["gate"] + f32_dv,
+        "gla_tc_fwd": f32_feat + b["v"] + b["gate"] + b["o"],
+        "dv_reduce": f32_dv + b["v"],
+        # raw q, k and the fp32 feature gradients in, fp32 du out (dW is negligible)
+        "convmix_tc_bwd": b["q"] + b["k"] + f32_feat + 4 * (s.H + s.H_kv) * s.d_k,
+        "conv_bwd": 4 * (s.H + s.H_kv) * s.d_k + 2 * (b["q"] + b["k"]),
     }
     if name in ("decode_state", "decode_features"):
         return alg_bytes_per_step("decode", s)
     if name in table:
         return table[name] * tok
-    if name.startswith("gla_bwd") or name in ("convmix_bwd", "conv_bwd_dx", "conv_bwd_dw", "dv_group_reduce"):
+    if name.startswith("gla_bwd") or name in ("convmix_bwd", "dv_group_reduce"):
         return alg_bytes_per_step("train", s) / 2  # the backward half of the step
     return alg_bytes_per_step(kind, s)              # fused kernels: the whole step's traffic
 

@@ -118,6 +118,9 @@ void lawcat_test_set_wait_limit(long long cycles);
  *   cache_q [B,conv_k-1,H*d_k], cache_k [B,conv_k-1,H_kv*d_k]  (nullable)
  *   out, W != NULL: qdot [B,T,H,d_k], kdot [B,T,H,d_k]   (kdot per query head: phi uses W[h])
  *   out, W == NULL: qdot = conv(q) [B,T,H,d_k], kdot = conv(k) [B,T,H_kv,d_k]
+ * Kernels: bf16 storage with W, d_k = 64 or 128 and conv_k <= 4 runs the mix on the tensor cores (fp16 operands, fp32
+ * accumulation, results within the bf16 tolerance of 1e-2 of the RMS); every other case, and chunk = 1, runs exact
+ * fp32 kernels.
  */
 int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const void* w_q, const void* w_k,
                     const void* W, const void* cache_q, const void* cache_k, void* qdot, void* kdot, void* ws,
@@ -128,6 +131,8 @@ int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const 
  * this is the chain rule on conv -> mix -> phi). d_qdot, d_kdot have the shapes of the forward outputs.
  *   out: dq [B,T,H,d_k], dk [B,T,H_kv,d_k] in p->dtype; dw_q, dw_k, dW in fp32, shaped like w_q, w_k, W.
  * Weight gradients are overwritten, not accumulated. dW must be NULL when W is NULL. Any output may be NULL.
+ * Kernels: bf16 storage with W, d_k = 64 and the softmax feature map runs the mix, the softmax Jacobian and dW on the
+ * tensor cores (two-term fp16 operands); every other case, and chunk = 1, runs exact fp32 kernels.
  */
 int lawcat_conv_bwd(const lawcat_params* p, const void* q, const void* k, const void* w_q, const void* w_k,
                     const void* W, const void* cache_q, const void* cache_k, const void* d_qdot,
@@ -140,6 +145,8 @@ int lawcat_conv_bwd(const lawcat_params* p, const void* q, const void* k, const 
  *   S0 [B,H,d_k,d_v] fp32, z0 [B,H,d_k] fp32: state before token 0 (nullable = zero, Eq. 5)
  *   out: o [B,T,H,d_v]; den [B,T,H] fp32 = qdot_t . z_t + eps (nullable; gla_bwd needs it);
  *        S_T, z_T = state after the last token (nullable)
+ * Kernels: bf16 storage with d_k = d_v = 64 runs chunkwise (64 tokens) on the tensor cores; every other case, and
+ * chunk = 1, runs the exact recurrence. ws: lawcat_workspace_bytes(p, LAWCAT_OP_GLA_FWD).
  */
 int lawcat_gla_fwd(const lawcat_params* p, const void* qdot, const void* kdot, const void* v, const void* gate,
                    const float* S0, const float* z0, void* o, float* den, float* S_T, float* z_T, void* ws,
@@ -152,6 +159,9 @@ int lawcat_gla_fwd(const lawcat_params* p, const void* qdot, const void* kdot, c
  *   out: d_qdot, d_kdot [B,T,H,d_k]; dv [B,T,H_kv,d_v] (summed over the G query heads of a group);
  *        dgate [B,T,H,gate_dim] -- the gradient with respect to the `gate` input (logits or log-decays).
  * No gradient flows into S0, z0 and none is taken from S_T, z_T.
+ * Kernels: bf16 storage with d_k = d_v = 64, and log-decay gates or sigmoid gates with gate_tau >= 8, runs the
+ * chunkwise tensor-core backward (two-term fp16 operands: gradients within 1e-2 of their RMS); sharper gates, other
+ * shapes and chunk = 1 run the exact three-sweep backward. ws: lawcat_workspace_bytes(p, LAWCAT_OP_GLA_BWD).
  */
 int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, const void* v, const void* gate,
                    const float* S0, const float* z0, const void* o, const float* den, const void* dO,

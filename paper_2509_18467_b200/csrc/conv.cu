@@ -360,45 +360,68 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_bwd_kernel(ConvMixBwdArgs 
   }
 }
 
-// dx[b,t,ch] = sum_delta w[ch,delta] du[b,t+delta,ch]   (transpose of the causal conv)
-template <typename TD, typename TW, typename TO>
-__global__ void conv_bwd_dx_kernel(const TD* __restrict__ du, const TW* __restrict__ w, TO* __restrict__ dx, int B,
-                                   int Tn, int C, int K) {
-  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (size_t)B * Tn * C) return;
-  const int ch = (int)(idx % C);
-  const int t = (int)((idx / C) % Tn);
-  const int b = (int)(idx / ((size_t)C * Tn));
-  float acc = 0.f;
-  for (int dl = 0; dl < K && t + dl < Tn; ++dl)
-    acc = fmaf(ldf(w + (size_t)ch * K + dl), ldf(du + ((size_t)b * Tn + t + dl) * C + ch), acc);
-  stf(dx + idx, acc);
-}
-
-// dw[ch,delta] = sum_{b,t} du[b,t,ch] x[b,t-delta,ch]; one thread = one channel over a span of tokens, then atomics.
-constexpr int DW_SPAN = 128;
-template <typename TD, typename TX>
-__global__ void conv_bwd_dw_kernel(const TD* __restrict__ du, const TX* __restrict__ x, const TX* __restrict__ cache,
-                                   float* __restrict__ dw, int B, int Tn, int C, int K) {
+// The conv's own backward for one stream, both results in one sweep:
+//   dx[b,t,ch] = sum_delta w[ch,delta] du[b,t+delta,ch]   (transpose of the causal conv)
+//   dw[ch,delta] = sum_{b,t} du[b,t,ch] x[b,t-delta,ch]
+// One thread = one channel over a span of tokens, neighbouring threads neighbouring channels: it slides one register
+// window over du (the tokens ahead) and one over x (the tokens behind), so every input is read once; the span's part of
+// dw goes out with atomic adds. Either result may be absent.
+constexpr int CBW_SPAN = 64;
+template <typename TD, typename TX, int KM>
+__global__ void __launch_bounds__(128) conv_bwd_kernel(const TD* __restrict__ du, const TX* __restrict__ x,
+                                                      const TX* __restrict__ w, const TX* __restrict__ cache,
+                                                      TX* __restrict__ dx, float* __restrict__ dw, int B, int Tn, int C,
+                                                      int K) {
   const int ch = blockIdx.y * blockDim.x + threadIdx.x;
   if (ch >= C) return;
-  const int spans = (Tn + DW_SPAN - 1) / DW_SPAN;
-  const int b = blockIdx.x / spans, t0 = (blockIdx.x % spans) * DW_SPAN;
-  const int t1 = min(Tn, t0 + DW_SPAN);
-  float acc[8], win[8];
+  const int spans = (Tn + CBW_SPAN - 1) / CBW_SPAN;
+  const int b = blockIdx.x / spans, t0 = (blockIdx.x % spans) * CBW_SPAN;
+  const int t1 = min(Tn, t0 + CBW_SPAN);
+  float tap[KM], acc[KM], xw[KM], dwin[KM];
 #pragma unroll
-  for (int d = 0; d < 8; ++d) acc[d] = 0.f;
-#pragma unroll
-  for (int d = 1; d < 8; ++d) win[d] = d < K ? raw_token(x, cache, b, t0 - d, Tn, C, K, ch) : 0.f;
-  for (int t = t0; t < t1; ++t) {
-    win[0] = ldf(x + ((size_t)b * Tn + t) * C + ch);
-    const float g = ldf(du + ((size_t)b * Tn + t) * C + ch);
-#pragma unroll
-    for (int d = 0; d < 8; ++d) acc[d] = fmaf(g, win[d], acc[d]);
-#pragma unroll
-    for (int d = 7; d > 0; --d) win[d] = win[d - 1];
+  for (int d = 0; d < KM; ++d) {
+    tap[d] = d < K ? ldf(w + (size_t)ch * K + d) : 0.f;
+    acc[d] = 0.f;
+    xw[d] = (d >= 1 && d < K) ? raw_token(x, cache, b, t0 - d, Tn, C, K, ch) : 0.f;   // xw[d] = x[t - d]
+    dwin[d] = (d + 1 < K && t0 + d < Tn) ? ldf(du + ((size_t)b * Tn + t0 + d) * C + ch) : 0.f;  // shifted below
   }
-  for (int d = 0; d < K; ++d) atomicAdd(dw + (size_t)ch * K + d, acc[d]);
+  // entering token t the window holds du[t .. t+K-2] in dwin[0 .. K-2]; the newest entry du[t+K-1] comes from the batch
+  // of loads that opens every group of 8 tokens (all of a group's loads are in flight together)
+  for (int tg = t0; tg < t1; tg += 8) {
+    float ahead[8], xin[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int ta = tg + j + K - 1;
+      ahead[j] = (tg + j < t1 && ta < Tn) ? ldf(du + ((size_t)b * Tn + ta) * C + ch) : 0.f;
+      xin[j] = tg + j < t1 ? ldf(x + ((size_t)b * Tn + tg + j) * C + ch) : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int t = tg + j;
+      if (t < t1) {
+#pragma unroll
+        for (int d = 0; d < KM; ++d)
+          if (d == K - 1) dwin[d] = ahead[j];
+        xw[0] = xin[j];
+        float o = 0.f;
+        const float g = dwin[0];
+#pragma unroll
+        for (int d = 0; d < KM; ++d) {
+          o = fmaf(tap[d], dwin[d], o);
+          acc[d] = fmaf(g, xw[d], acc[d]);
+        }
+        if (dx) stf(dx + ((size_t)b * Tn + t) * C + ch, o);
+#pragma unroll
+        for (int d = 0; d < KM - 1; ++d) dwin[d] = dwin[d + 1];
+        dwin[KM - 1] = 0.f;
+#pragma unroll
+        for (int d = KM - 1; d > 0; --d) xw[d] = xw[d - 1];
+      }
+    }
+  }
+  if (dw) {
+    for (int d = 0; d < K; ++d) atomicAdd(dw + (size_t)ch * K + d, acc[d]);
+  }
 }
 
 template <typename TI, typename TD>
@@ -406,20 +429,15 @@ static int conv_bwd_stream(const Ctx& c, const TD* du, const TI* x, const TI* w,
                            int NH) {
   const lawcat_params& p = *c.p;
   const int C = NH * p.d_k;
-  const size_t total = (size_t)p.B * p.T * C;
-  if (dx) {
-    LaunchScope _ls("conv_bwd_dx", c.stream);
-    conv_bwd_dx_kernel<TD, TI, TI><<<(unsigned)((total + 255) / 256), 256, 0, c.stream>>>(du, w, dx, p.B, p.T, C,
-                                                                                           p.conv_k);
-    LAWCAT_CHECK_LAUNCH();
-  }
-  if (dw) {
-    if (cudaMemsetAsync(dw, 0, sizeof(float) * (size_t)C * p.conv_k, c.stream) != cudaSuccess) return LAWCAT_ERR_CUDA;
-    dim3 grid(p.B * ((p.T + DW_SPAN - 1) / DW_SPAN), (C + 127) / 128);
-    LaunchScope _ls("conv_bwd_dw", c.stream);
-    conv_bwd_dw_kernel<TD, TI><<<grid, 128, 0, c.stream>>>(du, x, cache, dw, p.B, p.T, C, p.conv_k);
-    LAWCAT_CHECK_LAUNCH();
-  }
+  if (!dx && !dw) return LAWCAT_OK;
+  if (dw && cudaMemsetAsync(dw, 0, sizeof(float) * (size_t)C * p.conv_k, c.stream) != cudaSuccess) return LAWCAT_ERR_CUDA;
+  dim3 grid(p.B * ((p.T + CBW_SPAN - 1) / CBW_SPAN), (C + 127) / 128);
+  LaunchScope _ls("conv_bwd", c.stream);
+  if (p.conv_k <= 4)
+    conv_bwd_kernel<TD, TI, 4><<<grid, 128, 0, c.stream>>>(du, x, w, cache, dx, dw, p.B, p.T, C, p.conv_k);
+  else
+    conv_bwd_kernel<TD, TI, 8><<<grid, 128, 0, c.stream>>>(du, x, w, cache, dx, dw, p.B, p.T, C, p.conv_k);
+  LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }
 
