@@ -251,8 +251,13 @@ int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t,
  * The layer forward of Fig. 1 for callers whose tensors live in HOST memory (pinned memory makes the copies
  * asynchronous). h_* are host pointers laid out like the device tensors of lawcat_layer_fwd (no caches, zero initial
  * state); `arena` is caller-owned DEVICE scratch of at least lawcat_layer_fwd_host_arena_bytes(p) bytes that receives
- * the inputs, the output and the workspace. Enqueues on `stream`: host-to-device copies, the layer, the copy of o back
- * to h_o. Returns without synchronizing; h_o is valid once the stream has drained.
+ * the inputs, the output, the workspace and the state handed from slice to slice. The sequence is processed in slices
+ * of 2048 tokens (the state of Eq. 4 and the conv cache of Section 4.1 carry over, as in chunked prefill): the
+ * host-to-device copies of the next slice, the layer on the current slice and the copy of the previous slice's output
+ * back to h_o run on three streams. The two copy streams belong to the library (one pair per device, created on the
+ * first call); they start behind everything already enqueued on `stream`, and `stream` ends behind the last copy, so
+ * that the caller orders and synchronizes on `stream` alone. Returns without synchronizing; h_o is valid once
+ * `stream` has drained. Calls that share an arena must be enqueued on the same stream.
  */
 size_t lawcat_layer_fwd_host_arena_bytes(const lawcat_params* p);
 int lawcat_layer_fwd_host(const lawcat_params* p, const void* h_q, const void* h_k, const void* h_v,

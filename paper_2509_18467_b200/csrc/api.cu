@@ -1,4 +1,8 @@
-// The C ABI: argument validation on the host, then dispatch to the kernels. Nothing here allocates or synchronizes.
+// The C ABI: argument validation on the host, then dispatch to the kernels. Nothing here allocates device memory or
+// synchronizes (the host-buffer variant creates its two copy streams and its events on first use and keeps them).
+#include <mutex>
+#include <vector>
+
 #include "common.cuh"
 
 using namespace lawcat;
@@ -385,28 +389,83 @@ int lawcat_decode_step(const lawcat_params* p, const void* q_t, const void* k_t,
 }
 
 // ---- host-buffer variant of the layer forward ---------------------------------------------------------------------
-static size_t host_arena_layout(const lawcat_params* p, size_t off[10]) {
+// The sequence is cut into slices along T (per batch element); the copies of slice i+1 to the device, the layer on
+// slice i (which starts from the state and conv caches slice i-1 left) and the copy of slice i-1's output back run
+// on three streams, so that the step costs about its host-to-device copies alone.
+constexpr int HOST_SLICE = 2048;  // tokens per slice (a multiple of the chunk)
+
+struct HostStateSet { size_t S, z, cq, ck, bytes; };
+static HostStateSet host_state_set(const lawcat_params* p) {
   const size_t es = p->dtype == LAWCAT_F32 ? 4 : 2;
-  const size_t n[9] = {elems(p, p->H, p->d_k) * es,      // q
-                       elems(p, p->H_kv, p->d_k) * es,   // k
-                       elems(p, p->H_kv, p->d_v) * es,   // v
-                       elems(p, p->H, p->gate_dim) * es, // gate
-                       (size_t)p->H * p->d_k * p->conv_k * es, (size_t)p->H_kv * p->d_k * p->conv_k * es,
-                       (size_t)p->H * p->d_k * p->d_k * es,  // w_q, w_k, W
-                       elems(p, p->H, p->d_v) * es,      // o
-                       lawcat_workspace_bytes(p, LAWCAT_OP_LAYER_FWD)};
+  HostStateSet h;
   size_t o = 0;
-  for (int i = 0; i < 9; ++i) {
+  h.S = o; o += align_up(sizeof(float) * (size_t)p->H * p->d_k * p->d_v, 256);
+  h.z = o; o += align_up(sizeof(float) * (size_t)p->H * p->d_k, 256);
+  h.cq = o; o += align_up(es * (size_t)(p->conv_k - 1) * p->H * p->d_k, 256);
+  h.ck = o; o += align_up(es * (size_t)(p->conv_k - 1) * p->H_kv * p->d_k, 256);
+  h.bytes = o;
+  return h;
+}
+static lawcat_params host_slice_params(const lawcat_params* p, int len) {
+  lawcat_params ps = *p;
+  ps.B = 1;
+  ps.T = len;
+  return ps;
+}
+// off[0..8]: q, k, v, gate, w_q, w_k, W, o, workspace; off[9]: two state sets (ping-pong between slices); off[10]: end
+static size_t host_arena_layout(const lawcat_params* p, size_t off[11]) {
+  const size_t es = p->dtype == LAWCAT_F32 ? 4 : 2;
+  const lawcat_params ps = host_slice_params(p, p->T < HOST_SLICE ? p->T : HOST_SLICE);
+  size_t ws = lawcat_workspace_bytes(p, LAWCAT_OP_LAYER_FWD);
+  const size_t ws_slice = lawcat_workspace_bytes(&ps, LAWCAT_OP_LAYER_FWD);
+  if (ws_slice > ws) ws = ws_slice;
+  const size_t n[10] = {elems(p, p->H, p->d_k) * es,      // q
+                        elems(p, p->H_kv, p->d_k) * es,   // k
+                        elems(p, p->H_kv, p->d_v) * es,   // v
+                        elems(p, p->H, p->gate_dim) * es, // gate
+                        (size_t)p->H * p->d_k * p->conv_k * es, (size_t)p->H_kv * p->d_k * p->conv_k * es,
+                        (size_t)p->H * p->d_k * p->d_k * es,  // w_q, w_k, W
+                        elems(p, p->H, p->d_v) * es,      // o
+                        ws, 2 * host_state_set(p).bytes};
+  size_t o = 0;
+  for (int i = 0; i < 10; ++i) {
     off[i] = o;
     o += align_up(n[i], 256);
   }
-  off[9] = o;
+  off[10] = o;
   return o;
+}
+
+// copy streams and events of the host path, one set per device, created on first use and kept
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  std::vector<cudaEvent_t> ev;
+  cudaEvent_t event(size_t i) {
+    while (ev.size() <= i) {
+      cudaEvent_t e;
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      ev.push_back(e);
+    }
+    return ev[i];
+  }
+};
+static HostPipe* host_pipe() {
+  static std::mutex mu;
+  static HostPipe pipes[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  HostPipe& hp = pipes[dev];
+  if (!hp.in) {
+    if (cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+  }
+  return &hp;
 }
 
 size_t lawcat_layer_fwd_host_arena_bytes(const lawcat_params* p) {
   if (check_params(p, true) != LAWCAT_OK) return 0;
-  size_t off[10];
+  size_t off[11];
   return host_arena_layout(p, off);
 }
 
@@ -417,24 +476,70 @@ int lawcat_layer_fwd_host(const lawcat_params* p, const void* h_q, const void* h
   if (r) return r;
   if (!h_q || !h_k || !h_v || !h_gate || !h_w_q || !h_w_k || !h_W || !h_o || !arena || !aligned16(arena))
     return LAWCAT_ERR_INVALID_ARG;
-  size_t off[10];
+  size_t off[11];
   if (arena_bytes < host_arena_layout(p, off)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
+  if (p->B * p->T == 0) return LAWCAT_OK;
+  HostPipe* hp = host_pipe();
+  if (!hp) return LAWCAT_ERR_CUDA;
   char* a = (char*)arena;
   cudaStream_t st = (cudaStream_t)stream;
-  const void* src[7] = {h_q, h_k, h_v, h_gate, h_w_q, h_w_k, h_W};
   const size_t es = p->dtype == LAWCAT_F32 ? 4 : 2;
-  const size_t nb[7] = {elems(p, p->H, p->d_k) * es, elems(p, p->H_kv, p->d_k) * es, elems(p, p->H_kv, p->d_v) * es,
-                        elems(p, p->H, p->gate_dim) * es, (size_t)p->H * p->d_k * p->conv_k * es,
-                        (size_t)p->H_kv * p->d_k * p->conv_k * es, (size_t)p->H * p->d_k * p->d_k * es};
-  for (int i = 0; i < 7; ++i)
-    if (nb[i] && cudaMemcpyAsync(a + off[i], src[i], nb[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
-      return LAWCAT_ERR_CUDA;
-  r = lawcat_layer_fwd(p, a + off[0], a + off[1], a + off[2], a + off[3], a + off[4], a + off[5], a + off[6], nullptr,
-                       nullptr, nullptr, nullptr, a + off[7], nullptr, nullptr, nullptr, nullptr, a + off[8],
-                       off[9] - off[8], stream, nullptr);
-  if (r) return r;
-  const size_t no = elems(p, p->H, p->d_v) * es;
-  if (no && cudaMemcpyAsync(h_o, a + off[7], no, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LAWCAT_ERR_CUDA;
+#define LAWCAT_HOST_TRY(x) do { if ((x) != cudaSuccess) return LAWCAT_ERR_CUDA; } while (0)
+  size_t ne = 0;
+  // both copy streams start behind whatever the caller's stream holds (an earlier call may still use the arena)
+  cudaEvent_t e0 = hp->event(ne++);
+  if (!e0) return LAWCAT_ERR_CUDA;
+  LAWCAT_HOST_TRY(cudaEventRecord(e0, st));
+  LAWCAT_HOST_TRY(cudaStreamWaitEvent(hp->in, e0, 0));
+  LAWCAT_HOST_TRY(cudaStreamWaitEvent(hp->out, e0, 0));
+  const void* wsrc[3] = {h_w_q, h_w_k, h_W};
+  const size_t wnb[3] = {(size_t)p->H * p->d_k * p->conv_k * es, (size_t)p->H_kv * p->d_k * p->conv_k * es,
+                         (size_t)p->H * p->d_k * p->d_k * es};
+  for (int i = 0; i < 3; ++i)
+    LAWCAT_HOST_TRY(cudaMemcpyAsync(a + off[4 + i], wsrc[i], wnb[i], cudaMemcpyHostToDevice, hp->in));
+  const HostStateSet hs = host_state_set(p);
+  // bytes per token of the four streams and of the output
+  const size_t row[4] = {(size_t)p->H * p->d_k * es, (size_t)p->H_kv * p->d_k * es, (size_t)p->H_kv * p->d_v * es,
+                         (size_t)p->H * p->gate_dim * es};
+  const size_t orow = (size_t)p->H * p->d_v * es;
+  const void* src[4] = {h_q, h_k, h_v, h_gate};
+  for (int b = 0; b < p->B; ++b) {
+    int set = 0;
+    for (int t0 = 0; t0 < p->T; t0 += HOST_SLICE) {
+      const int len = p->T - t0 < HOST_SLICE ? p->T - t0 : HOST_SLICE;
+      const size_t tok = (size_t)b * p->T + t0;
+      for (int i = 0; i < 4; ++i)
+        LAWCAT_HOST_TRY(cudaMemcpyAsync(a + off[i] + tok * row[i], (const char*)src[i] + tok * row[i], (size_t)len * row[i],
+                                        cudaMemcpyHostToDevice, hp->in));
+      cudaEvent_t e_in = hp->event(ne++), e_done = hp->event(ne++);
+      if (!e_in || !e_done) return LAWCAT_ERR_CUDA;
+      LAWCAT_HOST_TRY(cudaEventRecord(e_in, hp->in));
+      LAWCAT_HOST_TRY(cudaStreamWaitEvent(st, e_in, 0));
+      const lawcat_params ps = host_slice_params(p, len);
+      char* prev = a + off[9] + (size_t)(set ^ 1) * hs.bytes;
+      char* next = a + off[9] + (size_t)set * hs.bytes;
+      const bool first = t0 == 0, last = t0 + len >= p->T, cache = p->conv_k > 1;
+      r = lawcat_layer_fwd(&ps, a + off[0] + tok * row[0], a + off[1] + tok * row[1], a + off[2] + tok * row[2],
+                           a + off[3] + tok * row[3], a + off[4], a + off[5], a + off[6],
+                           (first || !cache) ? nullptr : prev + hs.cq, (first || !cache) ? nullptr : prev + hs.ck,
+                           first ? nullptr : (const float*)(prev + hs.S), first ? nullptr : (const float*)(prev + hs.z),
+                           a + off[7] + tok * orow, (last || !cache) ? nullptr : next + hs.cq,
+                           (last || !cache) ? nullptr : next + hs.ck, last ? nullptr : (float*)(next + hs.S),
+                           last ? nullptr : (float*)(next + hs.z), a + off[8], off[9] - off[8], stream, nullptr);
+      if (r) return r;
+      LAWCAT_HOST_TRY(cudaEventRecord(e_done, st));
+      LAWCAT_HOST_TRY(cudaStreamWaitEvent(hp->out, e_done, 0));
+      LAWCAT_HOST_TRY(cudaMemcpyAsync((char*)h_o + tok * orow, a + off[7] + tok * orow, (size_t)len * orow,
+                                      cudaMemcpyDeviceToHost, hp->out));
+      set ^= 1;
+    }
+  }
+  // the caller's stream ends behind the last copy back
+  cudaEvent_t e_end = hp->event(ne++);
+  if (!e_end) return LAWCAT_ERR_CUDA;
+  LAWCAT_HOST_TRY(cudaEventRecord(e_end, hp->out));
+  LAWCAT_HOST_TRY(cudaStreamWaitEvent(st, e_end, 0));
+#undef LAWCAT_HOST_TRY
   return LAWCAT_OK;
 }
 
