@@ -1,12 +1,19 @@
 // Recurrent single-token decode (streaming inference, Section 6): the layer at one token with the conv cache of
 // Section 4.1 and the constant-size state of Eq. 4. Two launches:
-//   decode_features  (one block per head and group of 8 sequences, which share the head's W) conv -> shared linear layer
-//                    -> feature map for the token's query and key, decay alpha = exp(g), the normalizer state z (Eq. 8's
-//                    denominator) advanced in place; writes qdot, kdot, alpha and the denominator to the workspace
+//   decode_features  conv -> shared linear layer -> feature map for the token's query and key, decay alpha = exp(g), the
+//                    normalizer state z (Eq. 8's denominator) advanced in place; writes qdot, kdot, alpha and the
+//                    denominator to the workspace. Two kernels: decode_features_tc_kernel (bf16, d_k = 64 or 128: one
+//                    block per head and group of 16 or 32 sequences, the mix of all their vectors as one tensor-core
+//                    product) and decode_features_kernel (any shape and type: one block per head and group of 8
+//                    sequences, which share the head's W, fp32 FMA)
 //   decode_state     (one block per sequence and head) S <- diag(alpha) S + kdot^T v (Eq. 4), o = qdot S / denominator (Eq. 8): the fp32 state is streamed
 //                    through HBM once (read + write), which is the whole cost of the step; the same blocks then shift
 //                    the conv caches (every reader of the caches belongs to the first launch, which has completed)
+#include <mutex>
+#include <type_traits>
+
 #include "common.cuh"
+#include "octet_tile.cuh"
 
 namespace lawcat {
 
@@ -20,6 +27,7 @@ struct DecodeArgs {
   int B, H, Hkv, dk, dv, K, gd, phi, gate_mode, normalize;
   int w_smem;  // 1: W of the head is staged in shared memory
   float inv_tau, eps;
+  int* dev_status;
 };
 
 constexpr int DEC_THREADS = 256;
@@ -199,6 +207,281 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_features_kernel(DecodeArgs
   }
 }
 
+// ---- decode_features on the tensor cores (bf16 storage, d_k = 64 or 128, conv width up to 4) -----------------------------
+// One block per (query head, group of NSEQ sequences): the query vectors and the key vectors of the group share W_h
+// (Section 4.1), so their mix is ONE product Y = U W_h on the tensor cores (fp32 accumulator in tensor memory). U, the conv
+// outputs, goes in as a two-term fp16 pair hi + lo (two accumulating passes), which keeps about 21 bits of it; W_h is
+// exact in fp16. The 2 NSEQ vectors of a group (query stream first) are written to the M = 128 operand several times
+// over, once per group of 2 NSEQ rows: a warp reads only its own 32 lanes of tensor memory, and with the copies every warp
+// of the block finds every vector in its lanes. Thread = (vector, 16 of its channels): conv from global memory in fp32,
+// then, straight from tensor memory, phi, the decay, the normalizer state z advanced in place, and the denominator of
+// Eq. 8; same workspace layout as decode_features_kernel. Small groups (16 sequences at d_k = 128) give enough blocks to
+// fill the GPU at batch 64: the step is a chain of dependent memory round trips, not arithmetic.
+constexpr int DFT_THREADS = 256;
+
+template <int D>
+struct DftLay {
+  using L = ctc::Lay<D>;
+  static constexpr int NSEQ = 2048 / D;        // sequences per block: 16 (d_k = 128), 32 (d_k = 64)
+  static constexpr int LR = 2 * NSEQ;          // vectors per block
+  static constexpr int NP = 2 * (128 / LR);    // threads per vector
+  static constexpr int HC = D / NP;            // channels per thread
+  static_assert(HC == 16, "one 16-column tensor-memory load per thread");
+  static constexpr uint32_t OFF_WT = 0, OFF_U = OFF_WT + L::TILE_W, OFF_UL = OFF_U + L::TILE_U;
+  static constexpr uint32_t OFF_Z = OFF_UL + L::TILE_U;                    // fp32 [NSEQ][D + 1]: z after the update
+  static constexpr uint32_t OFF_TAPS = OFF_Z + NSEQ * (D + 1) * 4;         // fp32 [2][D][4]
+  static constexpr uint32_t OFF_RED = OFF_TAPS + 2 * D * 4 * 4;            // fp32 [NP][LR]: exchange between a vector's threads
+  static constexpr uint32_t OFF_BAR = (OFF_RED + 256 * 4 + 15) / 16 * 16;
+  static constexpr uint32_t BYTES = OFF_BAR + 64;
+};
+
+template <int D>
+__global__ void __launch_bounds__(DFT_THREADS) decode_features_tc_kernel(DecodeArgs a) {
+  using namespace ctc;
+  using L = Lay<D>;
+  using M = DftLay<D>;
+  constexpr int NSEQ = M::NSEQ, LR = M::LR, NP = M::NP, HC = M::HC;
+  extern __shared__ __align__(128) uint8_t sg[];
+  const uint32_t sb = smem_u32(sg);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int r = tid & 127, lr = r % LR, part = (r / LR) * 2 + (tid >> 7);
+  const int stream = lr / NSEQ, seq = lr % NSEQ, c0 = part * HC;
+  const int h = blockIdx.x, G = a.H / a.Hkv, j = h / G, K = a.K;
+  const int b = blockIdx.y * NSEQ + seq;
+  const bool valid = b < a.B;
+  volatile int* const s_flags = reinterpret_cast<volatile int*>(sg + M::OFF_BAR + 16);  // [0] tmem base, [1] abort
+  float* const s_taps = reinterpret_cast<float*>(sg + M::OFF_TAPS);
+  float* const s_red = reinterpret_cast<float*>(sg + M::OFF_RED);
+  float* const s_z = reinterpret_cast<float*>(sg + M::OFF_Z);
+  const size_t bh = (size_t)(valid ? b : 0) * a.H + h;
+  // ---- every global read that does not depend on another goes out first: W_h, the taps, this thread's conv rows (the
+  // token, delta = 0, and the cache rows, delta >= 1: row K - 1 - delta), its gate values and its part of z
+  uint4 wreg[D * L::OPR / DFT_THREADS];
+  {
+    const bf16* Wh = (const bf16*)a.W + (size_t)h * D * D;
+#pragma unroll
+    for (int k = 0; k < D * L::OPR / DFT_THREADS; ++k) {
+      const int idx = tid + k * DFT_THREADS, c = idx / L::OPR, o = idx % L::OPR;
+      wreg[k] = __ldg(reinterpret_cast<const uint4*>(Wh + (size_t)c * D + o * 8));
+    }
+  }
+  uint4 xreg[4][HC / 8];
+  {
+    const int NH = stream ? a.Hkv : a.H, head = stream ? j : h;
+    const bf16* tok = (const bf16*)(stream ? a.k_t : a.q_t) + ((size_t)(valid ? b : 0) * NH + head) * D + c0;
+    const bf16* cache = (const bf16*)(stream ? a.cache_k : a.cache_q) + ((size_t)(valid ? b : 0) * (K - 1) * NH + head) * D + c0;
+#pragma unroll
+    for (int dl = 0; dl < 4; ++dl) {
+#pragma unroll
+      for (int o = 0; o < HC / 8; ++o) {
+        xreg[dl][o] = make_uint4(0u, 0u, 0u, 0u);
+        if (valid && dl < K)
+          xreg[dl][o] = __ldg(reinterpret_cast<const uint4*>(dl == 0 ? tok + o * 8 : cache + (size_t)(K - 1 - dl) * NH * D + o * 8));
+      }
+    }
+  }
+  float zold[HC], graw[HC];
+#pragma unroll
+  for (int i = 0; i < HC; ++i) zold[i] = graw[i] = 0.f;
+  if (stream == 1 && valid) {
+    const bf16* gt = (const bf16*)a.gate_t + bh * a.gd;
+    if (a.gd == 1) {
+      graw[0] = __bfloat162float(gt[0]);
+    } else {
+#pragma unroll
+      for (int o = 0; o < HC / 8; ++o) unpack8b(__ldg(reinterpret_cast<const uint4*>(gt + c0 + o * 8)), graw + o * 8);
+    }
+#pragma unroll
+    for (int i = 0; i < HC; i += 4) {
+      const float4 z4 = *reinterpret_cast<const float4*>(a.z + bh * D + c0 + i);
+      zold[i] = z4.x; zold[i + 1] = z4.y; zold[i + 2] = z4.z; zold[i + 3] = z4.w;
+    }
+  }
+  float treg[2 * D * 4 / DFT_THREADS];
+#pragma unroll
+  for (int k = 0; k < 2 * D * 4 / DFT_THREADS; ++k) {
+    const int idx = tid + k * DFT_THREADS, st = idx / (D * 4), c = (idx >> 2) % D, dl = idx & 3;
+    const bf16* w = st ? (const bf16*)a.w_k + ((size_t)j * D + c) * K : (const bf16*)a.w_q + ((size_t)h * D + c) * K;
+    treg[k] = dl < K ? __bfloat162float(w[dl]) : 0.f;
+  }
+  // the blocks of decode_state may be scheduled from here on: they start with loads of S, which this kernel never
+  // touches, and wait for the end of this grid before they read anything it writes
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#pragma unroll
+  for (int k = 0; k < 2 * D * 4 / DFT_THREADS; ++k) s_taps[tid + k * DFT_THREADS] = treg[k];
+  if (tid == 0) {
+    mbar_init(sb + M::OFF_BAR, 1);
+    mbar_fence_init();
+    s_flags[1] = 0;
+  }
+  if (warp == 0) {
+    tmem_alloc(sb + M::OFF_BAR + 16, D);
+    tmem_relinquish();
+  }
+#pragma unroll
+  for (int k = 0; k < D * L::OPR / DFT_THREADS; ++k) {  // W[h][c][e] (exact in fp16) as a tile with rows c, columns e
+    const int idx = tid + k * DFT_THREADS, c = idx / L::OPR, o = idx % L::OPR;
+    float f[8];
+    unpack8b(wreg[k], f);
+    *reinterpret_cast<uint4*>(sg + M::OFF_WT + toff(L::SLAB_W, c, o * 8)) = pack8f16(f);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = (uint32_t)s_flags[0];
+  const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)c0;
+  Waiter wt{sb + M::OFF_BAR, 0u, s_flags + 1, a.dev_status};
+
+  // ---- conv of this thread's channels, written to every copy of its vector's row -------------------------------------------
+  {
+    const float* tp = s_taps + (stream * D + c0) * 4;
+#pragma unroll
+    for (int o = 0; o < HC / 8; ++o) {
+      float u[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int dl = 0; dl < 4; ++dl) {
+        float x[8];
+        unpack8b(xreg[dl][o], x);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) u[i] = fmaf(tp[(o * 8 + i) * 4 + dl], x[i], u[i]);
+      }
+      const uint4 ph = pack8f16(u);
+      const __half2* h2 = reinterpret_cast<const __half2*>(&ph);
+      float lo[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h2[i]);
+        lo[2 * i] = u[2 * i] - f.x;
+        lo[2 * i + 1] = u[2 * i + 1] - f.y;
+      }
+      const uint4 pl = pack8f16(lo);
+#pragma unroll
+      for (int cp = 0; cp < 128 / LR; ++cp) {
+        *reinterpret_cast<uint4*>(sg + M::OFF_U + toff(L::SLAB_U, lr + cp * LR, c0 + o * 8)) = ph;
+        *reinterpret_cast<uint4*>(sg + M::OFF_UL + toff(L::SLAB_U, lr + cp * LR, c0 + o * 8)) = pl;
+      }
+    }
+  }
+  fence_proxy_async();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (tid == 0) {  // Y = (U_hi + U_lo) W_h
+    const uint32_t idesc = instr_desc(128, D, FMT_F16, MAJOR_K, MAJOR_MN);
+    const uint64_t dh = kview(sb + M::OFF_U, L::SLAB_U), dl = kview(sb + M::OFF_UL, L::SLAB_U);
+    const uint64_t db = mview(sb + M::OFF_WT, L::SLAB_W);
+    for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem, dadv(dh, 2 * L::SLAB_U * kk), dadv(db, 256 * kk), idesc, kk > 0);
+    for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem, dadv(dl, 2 * L::SLAB_U * kk), dadv(db, 256 * kk), idesc, 1);
+    mma_commit(sb + M::OFF_BAR);
+  }
+  wt.wait();
+
+  // ---- phi over this thread's channels of its vector ------------------------------------------------------------------------
+  float y[HC];
+  tmem_ld16(lane_base, y);
+  tmem_wait_ld();
+  if (a.phi == LAWCAT_PHI_SOFTMAX) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < HC; ++i) m = fmaxf(m, y[i]);
+    s_red[part * LR + lr] = m;
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < NP; ++q) m = fmaxf(m, s_red[q * LR + lr]);
+    const float mb = m * 1.4426950408889634f;
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < HC; ++i) {
+      y[i] = ex2f(fmaf(y[i], 1.4426950408889634f, -mb));
+      sum += y[i];
+    }
+    __syncthreads();  // (every thread of the vector has read the maxima)
+    s_red[part * LR + lr] = sum;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int q = 0; q < NP; ++q) tot += s_red[q * LR + lr];
+    const float inv = 1.f / tot;
+#pragma unroll
+    for (int i = 0; i < HC; ++i) y[i] *= inv;
+  } else if (a.phi == LAWCAT_PHI_ELU1) {
+#pragma unroll
+    for (int i = 0; i < HC; ++i) y[i] = y[i] > 0.f ? y[i] + 1.f : expf(y[i]);
+  }
+  __syncthreads();  // (the exchange buffer is used again below)
+
+  // ---- features and decays to the workspace, z advanced in place, denominator of Eq. 8 ----------------------------------------
+  float* out = a.vecs + bh * 3 * D + stream * D + c0;
+  if (valid) {
+#pragma unroll
+    for (int i = 0; i < HC; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(y[i], y[i + 1], y[i + 2], y[i + 3]);
+  }
+  if (stream == 1) {
+    float* al = a.vecs + bh * 3 * D + 2 * D + c0;
+    float* zg = a.z + bh * D + c0;
+    float alpha[HC], zn[HC];
+    const float a1 = (valid && a.gd == 1) ? expf(log_decay(graw[0], a.gate_mode, a.inv_tau)) : 0.f;
+#pragma unroll
+    for (int i = 0; i < HC; ++i) {
+      alpha[i] = a.gd == 1 ? a1 : (valid ? expf(log_decay(graw[i], a.gate_mode, a.inv_tau)) : 0.f);
+      zn[i] = fmaf(alpha[i], zold[i], y[i]);
+      s_z[seq * (D + 1) + c0 + i] = zn[i];
+    }
+    if (valid) {
+#pragma unroll
+      for (int i = 0; i < HC; i += 4) {
+        *reinterpret_cast<float4*>(al + i) = make_float4(alpha[i], alpha[i + 1], alpha[i + 2], alpha[i + 3]);
+        *reinterpret_cast<float4*>(zg + i) = make_float4(zn[i], zn[i + 1], zn[i + 2], zn[i + 3]);
+      }
+    }
+  }
+  __syncthreads();
+  if (stream == 0) {
+    float dot = 0.f;
+#pragma unroll
+    for (int i = 0; i < HC; ++i) dot = fmaf(y[i], s_z[seq * (D + 1) + c0 + i], dot);
+    s_red[part * LR + lr] = dot;
+  }
+  __syncthreads();
+  if (stream == 0 && part == 0 && valid) {
+    float den = a.eps;
+#pragma unroll
+    for (int q = 0; q < NP; ++q) den += s_red[q * LR + lr];
+    a.den[bh] = den;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, D);
+  }
+}
+
+bool decode_tc_supported(const lawcat_params& p) {
+  return p.dtype == LAWCAT_BF16 && (p.d_k == 64 || p.d_k == 128) && p.conv_k <= 4 && p.chunk != 1;
+}
+
+template <int D>
+static int launch_decode_features_tc(const Ctx& c, const DecodeArgs& a) {
+  static std::mutex mu;
+  static bool done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LAWCAT_ERR_CUDA;
+  {
+    std::lock_guard<std::mutex> lk(mu);
+    if (!done[dev]) {
+      if (cudaFuncSetAttribute(decode_features_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)DftLay<D>::BYTES) != cudaSuccess)
+        return LAWCAT_ERR_CUDA;
+      done[dev] = true;
+    }
+  }
+  const dim3 grid((unsigned)a.H, (unsigned)((a.B + DftLay<D>::NSEQ - 1) / DftLay<D>::NSEQ));
+  LAWCAT_LAUNCH("decode_features", c.stream,
+                decode_features_tc_kernel<D><<<grid, DFT_THREADS, DftLay<D>::BYTES, c.stream>>>(a));
+  return LAWCAT_OK;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(DEC_THREADS, 3) decode_state_kernel(DecodeArgs a) {
   extern __shared__ __align__(16) float smem[];
@@ -294,16 +577,22 @@ template <typename T>
 static int decode_typed(const Ctx& c, DecodeArgs& a) {
   const lawcat_params& p = *c.p;
   if (p.B * p.H == 0) return LAWCAT_OK;
-  size_t smem1 = sizeof(float) * (size_t)p.d_k * (2 * DEC_NV + DEC_SEQ) + sizeof(T) * (size_t)p.d_k * p.conv_k * (DEC_NV + 2);
-  if (p.d_k > 32 * DEC_ZR) return LAWCAT_ERR_UNSUPPORTED;  // (one warp holds a sequence's normalizer state)
-  const size_t wbytes = sizeof(T) * (size_t)p.d_k * p.d_k;
-  a.w_smem = smem1 + wbytes <= 100 * 1024 ? 1 : 0;
-  if (a.w_smem) smem1 += wbytes;
-  if (smem1 > 48 * 1024 &&
-      cudaFuncSetAttribute(decode_features_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess)
-    return LAWCAT_ERR_CUDA;
-  LAWCAT_LAUNCH("decode_features", c.stream, decode_features_kernel<T><<<p.H * ((p.B + DEC_SEQ - 1) / DEC_SEQ), DEC_THREADS, smem1, c.stream>>>(a));
-  LAWCAT_CHECK_LAUNCH();
+  if (std::is_same<T, bf16>::value && decode_tc_supported(p)) {
+    const int r = p.d_k == 64 ? launch_decode_features_tc<64>(c, a) : launch_decode_features_tc<128>(c, a);
+    if (r) return r;
+    LAWCAT_CHECK_LAUNCH();
+  } else {
+    size_t smem1 = sizeof(float) * (size_t)p.d_k * (2 * DEC_NV + DEC_SEQ) + sizeof(T) * (size_t)p.d_k * p.conv_k * (DEC_NV + 2);
+    if (p.d_k > 32 * DEC_ZR) return LAWCAT_ERR_UNSUPPORTED;  // (one warp holds a sequence's normalizer state)
+    const size_t wbytes = sizeof(T) * (size_t)p.d_k * p.d_k;
+    a.w_smem = smem1 + wbytes <= 100 * 1024 ? 1 : 0;
+    if (a.w_smem) smem1 += wbytes;
+    if (smem1 > 48 * 1024 &&
+        cudaFuncSetAttribute(decode_features_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess)
+      return LAWCAT_ERR_CUDA;
+    LAWCAT_LAUNCH("decode_features", c.stream, decode_features_kernel<T><<<p.H * ((p.B + DEC_SEQ - 1) / DEC_SEQ), DEC_THREADS, smem1, c.stream>>>(a));
+    LAWCAT_CHECK_LAUNCH();
+  }
   const size_t smem2 = sizeof(float) * ((size_t)3 * p.d_k + p.d_v + (size_t)(DEC_THREADS / 16) * p.d_v);
   if (smem2 > 48 * 1024 &&
       cudaFuncSetAttribute(decode_state_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
@@ -336,7 +625,7 @@ int launch_decode(const Ctx& c, const void* q_t, const void* k_t, const void* v_
   a.den = a.vecs + (size_t)p.B * p.H * 3 * p.d_k;
   a.B = p.B; a.H = p.H; a.Hkv = p.H_kv; a.dk = p.d_k; a.dv = p.d_v; a.K = p.conv_k; a.gd = p.gate_dim;
   a.phi = p.phi; a.gate_mode = p.gate_mode; a.normalize = p.normalize;
-  a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps;
+  a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps; a.dev_status = c.dev_status;
   if (p.dtype == LAWCAT_F32) return decode_typed<float>(c, a);
   return decode_typed<bf16>(c, a);
 }

@@ -257,3 +257,39 @@ def test_decode_steps_against_oracle(api, s):
     if s.conv_k > 1:
         assert np.array_equal(cq.float().cpu().numpy(), ref["cache_q"].astype(np.float32))
         assert np.array_equal(ck.float().cpu().numpy(), ref["cache_k"].astype(np.float32))
+
+
+@pytest.mark.parametrize("B,dk,dv,conv_k,gate_dim,kw", [
+    (70, 128, 128, 4, 0, {}),                       # two groups of sequences, the second ragged
+    (64, 64, 64, 2, 0, {"phi": 1}),                 # 1 + ELU, conv width 2
+    (3, 128, 64, 1, 1, {"phi": 2}),                 # identity feature map, no conv, one decay per head
+    (5, 64, 128, 3, 0, {"gate_mode": 1}),           # log-decay gates
+    (2, 128, 128, 4, 0, {"eps": 0.3, "normalize": 1}),
+    (2, 64, 64, 4, 0, {"normalize": 0}),
+], ids=["B70-d128", "elu1-K2", "identity-K1-g1", "logdecay", "eps", "no-normalizer"])
+def test_decode_steps_tensor_core_features(api, B, dk, dv, conv_k, gate_dim, kw):
+    """bf16 decode with d_k = 64 / 128 computes the mix of a step's query and key vectors on the tensor cores: the
+    variants of the feature map, gate and normalizer, and a batch that spans two groups of 64 sequences."""
+    import torch
+    s = shape(B, 4, 4, 2, dk, dv, "bf16", gate_dim=gate_dim, conv_k=conv_k, cid=12)
+    names = LAYER_NAMES + ["S0", "z0"] + (["cache_q", "cache_k"] if conv_k > 1 else [])
+    x = I.make(s, names)
+    if kw.get("gate_mode") == 1:
+        x["gate"] = I.round_to_bf16(-np.abs(x["gate"]) * 0.1)
+    if kw.get("phi") == 2:  # the identity map needs positive features for a positive denominator
+        for n in ("q", "k", "w_q", "w_k", "W"):
+            x[n] = np.abs(x[n])
+    d = dev(api, x, s)
+    p = P(api, s, **kw)
+    S, z = d["S0"].clone(), d["z0"].clone()
+    cq = d["cache_q"].clone() if conv_k > 1 else None
+    ck = d["cache_k"].clone() if conv_k > 1 else None
+    ref = O.layer_fwd(oracle_params(s, **kw), *[x[n] for n in LAYER_NAMES], x.get("cache_q"), x.get("cache_k"),
+                      x["S0"], x["z0"])
+    outs = []
+    for t in range(s.T):
+        tok = [d[n][:, t].contiguous() for n in LAYER_NAMES[:4]]
+        outs.append(api.lawcat_decode_step(p, *tok, d["w_q"], d["w_k"], d["W"], S, z, cq, ck))
+    check(torch.stack(outs, 1), ref["o"], "bf16", "decode o")
+    check(S, ref["S_T"], "bf16", "S", f32_store=True)
+    check(z, ref["z_T"], "bf16", "z", f32_store=True)
