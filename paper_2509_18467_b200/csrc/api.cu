@@ -225,8 +225,9 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
   if (need && (!ws || ws_bytes < need)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
   Ctx c{p, (cudaStream_t)stream, dev_status};
   if (layer_tc_supported(*p)) {  // chunkwise tensor-core kernel
-    if ((r = launch_layer_tc(c, q, k, v, gate, w_q, w_k, W, cache_q_in, cache_k_in, S0, z0, o, S_T, z_T, ws))) return r;
-    return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
+    // (the kernel also writes the conv caches after the last token)
+    return launch_layer_tc(c, q, k, v, gate, w_q, w_k, W, cache_q_in, cache_k_in, S0, z0, o, cache_q_out, cache_k_out, S_T,
+                           z_T, ws);
   }
   float* qdot = (float*)ws;
   float* kdot = (float*)((char*)ws + align_up(sizeof(float) * elems(p, p->H, p->d_k), 256));

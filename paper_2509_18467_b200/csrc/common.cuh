@@ -79,7 +79,7 @@ int layer_tc_segments(const lawcat_params& p);
 size_t layer_tc_workspace_bytes(const lawcat_params& p);
 int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, const void* gate, const void* w_q,
                     const void* w_k, const void* W, const void* cache_q_in, const void* cache_k_in, const float* S0,
-                    const float* z0, void* o, float* S_T, float* z_T, void* ws);
+                    const float* z0, void* o, void* cache_q_out, void* cache_k_out, float* S_T, float* z_T, void* ws);
 
 // Chunkwise tensor-core GLA on given features and its backward (gla_tc.cu).
 bool gla_tc_supported(const lawcat_params& p);

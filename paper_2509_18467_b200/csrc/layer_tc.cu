@@ -24,17 +24,40 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [B, T, heads, dh] bf16 tensor as a 4-D map (channel, head, token, batch) with boxes of 64 channels x rows tokens
+// [B, T, heads, dh] bf16 tensor as a 4-D map (channel, head, token, batch) with boxes of 64 channels x rows tokens.
+// A map depends only on the pointer and the shape, so the last few are kept per host thread: a serving loop that calls
+// with the same buffers encodes each map once.
 static bool make_map(CUtensorMap* m, const void* ptr, int heads, int T, int B, int rows, int dh) {
+  struct Slot {
+    const void* ptr;
+    int heads, T, B, rows, dh;
+    bool used;
+    CUtensorMap map;
+  };
+  constexpr int NSLOT = 16;
+  thread_local Slot cache[NSLOT] = {};
+  thread_local int next = 0;
+  for (int i = 0; i < NSLOT; ++i) {
+    const Slot& c = cache[i];
+    if (c.used && c.ptr == ptr && c.heads == heads && c.T == T && c.B == B && c.rows == rows && c.dh == dh) {
+      *m = c.map;
+      return true;
+    }
+  }
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[4] = {(cuuint64_t)dh, (cuuint64_t)heads, (cuuint64_t)T, (cuuint64_t)B};
   const cuuint64_t strides[3] = {(cuuint64_t)dh * 2, (cuuint64_t)heads * dh * 2, (cuuint64_t)T * heads * dh * 2};
   const cuuint32_t box[4] = {64, 1, (cuuint32_t)rows, 1};
   const cuuint32_t es[4] = {1, 1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, es,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  Slot& c = cache[next];
+  next = (next + 1) % NSLOT;
+  c.ptr = ptr; c.heads = heads; c.T = T; c.B = B; c.rows = rows; c.dh = dh; c.map = *m; c.used = true;
+  return true;
 }
 
 // State at the start of every segment from the end states of its pieces (each computed from a zero state) and their
@@ -144,7 +167,7 @@ bool layer_tc_supported(const lawcat_params& p) {
 
 int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, const void* gate, const void* w_q,
                     const void* w_k, const void* W, const void* cache_q_in, const void* cache_k_in, const float* S0,
-                    const float* z0, void* o, float* S_T, float* z_T, void* ws) {
+                    const float* z0, void* o, void* cache_q_out, void* cache_k_out, float* S_T, float* z_T, void* ws) {
   using namespace tc;
   const lawcat_params& p = *c.p;
   CUtensorMap tq, tk, tv, tg;
@@ -159,6 +182,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   a.gate = (const bf16*)gate; a.gate_dim = p.gate_dim; a.dh = dh;
   a.w_q = (const bf16*)w_q; a.w_k = (const bf16*)w_k; a.W = (const bf16*)W;
   a.cache_q = (const bf16*)cache_q_in; a.cache_k = (const bf16*)cache_k_in;
+  a.cache_q_out = (bf16*)cache_q_out; a.cache_k_out = (bf16*)cache_k_out;
   a.dev_status = c.dev_status;
   a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k;
   a.gate_mode = p.gate_mode; a.normalize = p.normalize; a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps;

@@ -135,6 +135,7 @@ struct TcArgs {
   float *S_T, *z_T;      // state after the last token of the CTA's segment
   float* dtot;           // [B,H,nseg,128]: log2 of the total decay of the segment per key channel (nullable)
   bf16* o;               // [B,T,H,128]
+  bf16 *cache_q_out, *cache_k_out;  // conv caches after the last token (nullable): [B,K-1,H*dh], [B,K-1,Hkv*dh]
   int* dev_status;
   int T, H, Hkv, K;
   int nseg, seg_len;     // segments per sequence and tokens per segment (a multiple of C)
@@ -373,6 +374,23 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     *reinterpret_cast<uint4*>(sg + OFF_HALO + ((st * 3 + r) * 16 + oc) * 16) = v;
   }
   __syncthreads();
+  // conv caches after the last token (Section 4.1: the last K - 1 raw rows of [cache_in, x]): they depend on the raw
+  // inputs alone, so the block of a head's last segment writes them here (the key stream by the first head of a group)
+  if (MODE == 0 && seg == a.nseg - 1 && sub == 0 && a.K > 1 && tid < PREP_THREADS) {
+    const int per = (a.K - 1) * (dh / 8);  // 16-byte units per stream
+    for (int idx = tid; idx < 2 * per; idx += PREP_THREADS) {
+      const int st = idx / per, r = (idx % per) / (dh / 8), oc = idx % (dh / 8);
+      bf16* dst = st ? a.cache_k_out : a.cache_q_out;
+      if (dst == nullptr || (st == 1 && h % G != 0)) continue;
+      const int NH = st ? a.Hkv : a.H, head = st ? j : h, tok = a.T - (a.K - 1) + r;
+      const bf16* x = st ? a.k : a.q;
+      const bf16* cin = st ? a.cache_k : a.cache_q;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (tok >= 0) v = *reinterpret_cast<const uint4*>(x + (((size_t)b * a.T + tok) * NH + head) * dh + oc * 8);
+      else if (cin != nullptr) v = *reinterpret_cast<const uint4*>(cin + (((size_t)b * (a.K - 1) + tok + a.K - 1) * NH + head) * dh + oc * 8);
+      *reinterpret_cast<uint4*>(dst + (((size_t)b * (a.K - 1) + r) * NH + head) * dh + oc * 8) = v;
+    }
+  }
   if (tid < C) *reinterpret_cast<__half*>(sg + OFF_ONES + (tid >> 3) * 128 + (tid & 7) * 16) = __float2half(1.f);
   fence_proxy_async();
   tc_fence_before_sync();
