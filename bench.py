@@ -112,6 +112,7 @@ def kernel_bytes_per_step(name: str, kind: str, s: I.LayerShape) -> float:
         # dv per query head out
         "gla_tc_bwd": 2 * f32_feat + b["v"] + b["gate"] + b["o"] + b["gate"] + f32_dv,
         "gla_tc_fwd": f32_feat + b["v"] + b["gate"] + b["o"],
+        "gla_tc_bwd_sweep": f32_feat + b["v"] + b["gate"] + b["o"],   # features, v, gate, dO in
         "dv_reduce": f32_dv + b["v"],
         # raw q, k and the fp32 feature gradients in, fp32 du out (dW is negligible)
         "convmix_tc_bwd": b["q"] + b["k"] + f32_feat + 4 * (s.H + s.H_kv) * s.d_k,

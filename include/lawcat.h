@@ -87,6 +87,13 @@ size_t lawcat_workspace_bytes(const lawcat_params* p, int op);
 /* Static, human-readable name of a status code. */
 const char* lawcat_status_string(int status);
 
+/*
+ * Detail of the last LAWCAT_ERR_CUDA this host thread got from a kernel launch: the CUDA runtime's message and the
+ * place in the library that saw it ("" when there was none). The string belongs to the library and is overwritten by
+ * the thread's next such error.
+ */
+const char* lawcat_last_cuda_error(void);
+
 /* Library version, major*10000 + minor*100 + patch. */
 int lawcat_version(void);
 

@@ -24,13 +24,18 @@ EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "
            "lawcat_trace_begin", "lawcat_trace_end", "lawcat_test_set_wait_limit", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
            "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_layer_fwd_varlen_workspace_bytes",
            "lawcat_layer_fwd_varlen", "lawcat_layer_bwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
-           "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc"]
+           "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc", "lawcat_last_cuda_error"]
 
 
 class LawcatError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {status_string(status)} (status {status})")
+        detail = ""
+        if status == 3:  # LAWCAT_ERR_CUDA: the runtime's own message, when a launch produced it
+            f = lib().lawcat_last_cuda_error
+            f.restype = ctypes.c_char_p
+            detail = (f() or b"").decode()
+        super().__init__(f"{where}: {status_string(status)} (status {status})" + (f": {detail}" if detail else ""))
 
 
 class Params(ctypes.Structure):

@@ -113,9 +113,16 @@ struct LaunchScope {
     __VA_ARGS__;                             \
   } while (0)
 
-#define LAWCAT_CHECK_LAUNCH()                                 \
-  do {                                                        \
-    if (cudaGetLastError() != cudaSuccess) return LAWCAT_ERR_CUDA; \
+// Keeps the text of a CUDA runtime error (with the place that saw it) for lawcat_last_cuda_error(); per host thread.
+void note_cuda_error(cudaError_t e, const char* file, int line);
+
+#define LAWCAT_CHECK_LAUNCH()                                   \
+  do {                                                          \
+    const cudaError_t _e = cudaGetLastError();                  \
+    if (_e != cudaSuccess) {                                    \
+      ::lawcat::note_cuda_error(_e, __FILE__, __LINE__);        \
+      return LAWCAT_ERR_CUDA;                                   \
+    }                                                           \
   } while (0)
 
 }  // namespace lawcat

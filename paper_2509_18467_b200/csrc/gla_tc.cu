@@ -86,7 +86,11 @@ constexpr uint32_t OFF_R16L = OFF_R16 + TILE_CV;
 constexpr uint32_t OFF_KQL = OFF_R16L + TILE_CV;     // low part of kh / qh
 constexpr uint32_t OFF_DT = (OFF_KQL + TILE_TD + 127) / 128 * 128;   // fp32 [64][D]: qdot dqdot - kdot dkdot and its running sum
 constexpr uint32_t SMEM_BWD = OFF_DT + C * D * 4;    // (the fp32 tile doubles as the pad behind the last operand)
-static_assert(SMEM_BWD <= 232448 && 2 * SMEM_FWD + 2048 <= 232448, "shared memory budget");
+// The forward sweep of the backward (its own launch, two thread blocks per SM) keeps the low parts of its two-term operands
+// right behind the state operand, in an order of its own (see the kernel): the tile that is read as an MN-major M = 128
+// operand -- sixteen slabs from its start -- must not be the last one.
+constexpr uint32_t SMEM_SWEEP = OFF_PML + TILE_TD + 2048;
+static_assert(SMEM_BWD <= 232448 && 2 * SMEM_SWEEP + 2048 <= 232448, "shared memory budget");
 static_assert(OFF_R16L + 16 * SLAB_C <= SMEM_BWD + 16 * SLAB_C, "");
 
 // tensor memory map (32-bit columns): the forward kernel allocates 256 columns, the backward 512
@@ -105,6 +109,7 @@ struct GArgs {
   float* dvh;         // [B,T,H,D] per-head dv (fp32), reduced over the heads of a group afterwards
   uint8_t* ws_s16;    // [B*H][chunks][2 TILE_CV + 16] the (two-term) state operand of every chunk and its format
   float *ws_den, *ws_delta;  // [B,T,H]: 1 / den_t and dO_t . o_t
+  float* ws_scale;           // [B*H]: largest |do'| of the head
   int* dev_status;
   int B, T, H, Hkv, gate_dim, gate_mode, normalize;
   float inv_tau, eps;
@@ -169,14 +174,21 @@ __device__ __forceinline__ void tmem_st8(uint32_t taddr, const float* v) {
                : "memory");
 }
 
-// BWD = false: the forward (o, den, S_T, z_T). BWD = true: forward sweep for the scratch quantities, then the reverse sweep;
-// there every product whose few, large terms decide the first tokens of a sequence (small denominators, gradients a
+// MODE 0: the forward (o, den, S_T, z_T). The backward is two launches: MODE 1, the forward sweep for the scratch quantities
+// (state operand of every chunk, 1 / den, dO . o, the scale of do'), two thread blocks per SM; MODE 2, the reverse sweep. In
+// the backward every product whose few, large terms decide the first tokens of a sequence (small denominators, gradients a
 // hundred times the typical size) runs on two-term operands x = hi + lo (hi hi + lo hi + hi lo, about 21 significant bits).
-template <bool BWD>
-__global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArgs a) {
+template <int MODE>
+__global__ void __launch_bounds__(THREADS, MODE == 2 ? 1 : 2) gla_tc_kernel(const GArgs a) {
   extern __shared__ __align__(128) uint8_t sg[];
-  constexpr bool SPLIT = BWD;
-  constexpr uint32_t TMEM_COLS = BWD ? 512 : 256;
+  constexpr bool BWD = MODE != 0, SPLIT = BWD;
+  constexpr uint32_t TMEM_COLS = MODE == 2 ? 512 : 256;
+  // Low-part tiles. The sweep kernel (MODE 1) packs them into the three tile slots behind the state operand: low part of
+  // kh first (it is read as an MN-major M = 128 operand, sixteen slabs from its start, so two tile slots must follow its
+  // start), then that of qs -- whose slot the low part of the masked scores takes over once the first batch of products
+  // has consumed it -- then that of ks (a B operand of 64 rows: nothing is read behind it).
+  constexpr uint32_t oKQL = MODE == 1 ? OFF_QSL : OFF_KQL, oQSL = MODE == 1 ? OFF_KSL : OFF_QSL;
+  constexpr uint32_t oKSL = MODE == 1 ? OFF_PML : OFF_KSL, oPML = MODE == 1 ? OFF_KSL : OFF_PML;
   const uint32_t sb = smem_u32(sg);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   float* const s_x = reinterpret_cast<float*>(sg + OFF_X);
@@ -207,7 +219,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
     const int r = i & (C - 1), sl = i >> 6;
     const uint4 w = make_uint4(0u, 0u, 0u, 0u);
     *reinterpret_cast<uint4*>(sg + OFF_VP + toff(SLAB_T, r, D + 8 * sl)) = w;
-    if (BWD) {
+    if (MODE == 2) {
       *reinterpret_cast<uint4*>(sg + OFF_DO + toff(SLAB_T, r, D + 8 * sl)) = w;
       *reinterpret_cast<uint4*>(sg + OFF_DOL + toff(SLAB_T, r, D + 8 * sl)) = w;
     }
@@ -278,8 +290,8 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       tmem_wait_st();
     }
   };
-  load_state(true);
-  if (row_thr && (a.S0 || a.z0)) {  // bound on the given state: decides the operand format of the first chunks
+  load_state(MODE != 2);  // (the reverse sweep starts from a zero adjoint state)
+  if (MODE != 2 && row_thr && (a.S0 || a.z0)) {  // bound on the given state: decides the operand format of the first chunks
     float mx = 0.f;
     for (int e = 0; e < D; ++e)
       if (a.S0) mx = fmaxf(mx, fabsf(a.S0[((size_t)bh * D + row) * D + e]));
@@ -422,9 +434,9 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         w[i] = reverse ? q[i] * s_dm[o8 * 8 + i] : k[i] * s_e63[o8 * 8 + i];
         vmax = fmaxf(vmax, fabsf(vv[i]));
       }
-      put8(OFF_QS, OFF_QSL, SLAB_T, r, o8 * 8, q, f16, SPLIT);
-      put8(OFF_KS, OFF_KSL, SLAB_T, r, o8 * 8, k, f16, SPLIT);
-      put8(OFF_KQ, OFF_KQL, SLAB_T, r, o8 * 8, w, f16, SPLIT);
+      put8(OFF_QS, oQSL, SLAB_T, r, o8 * 8, q, f16, SPLIT);
+      put8(OFF_KS, oKSL, SLAB_T, r, o8 * 8, k, f16, SPLIT);
+      put8(OFF_KQ, oKQL, SLAB_T, r, o8 * 8, w, f16, SPLIT);
       put8(OFF_VP, 0, SLAB_T, r, o8 * 8, vv, f16, false);
       const float one[8] = {1.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       if (o8 == 0) put8(OFF_VP, 0, SLAB_T, r, D, one, f16, false);
@@ -447,8 +459,8 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
 
   // ====================================================================================================== forward sweep
   float domax = 0.f;
-  prefetch_chunk(0);
-  for (int n = 0; n < nchunks; ++n) {
+  if (MODE != 2) prefetch_chunk(0);
+  for (int n = 0; MODE != 2 && n < nchunks; ++n) {
     const int t0 = n * C, nvalid = min(C, a.T - t0);
     GTL(0);
     prefetch_chunk(n + 1);
@@ -495,9 +507,9 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       if (tid == 0) *reinterpret_cast<int*>(dst + 2 * TILE_CV) = fmt;
     }
     if (tid == 0) {
-      mma_split(COL_P, KV(OFF_QS, SLAB_T), SPLIT ? KV(OFF_QSL, SLAB_T) : NONE, KST_T, KV(OFF_KS, SLAB_T),
-                SPLIT ? KV(OFF_KSL, SLAB_T) : NONE, KST_T, D / 16, instr_desc(128, C, fmt, MAJOR_K, MAJOR_K), false);
-      mma_split(COL_A, KV(OFF_QS, SLAB_T), SPLIT ? KV(OFF_QSL, SLAB_T) : NONE, KST_T, MV(OFF_S16, SLAB_C),
+      mma_split(COL_P, KV(OFF_QS, SLAB_T), SPLIT ? KV(oQSL, SLAB_T) : NONE, KST_T, KV(OFF_KS, SLAB_T),
+                SPLIT ? KV(oKSL, SLAB_T) : NONE, KST_T, D / 16, instr_desc(128, C, fmt, MAJOR_K, MAJOR_K), false);
+      mma_split(COL_A, KV(OFF_QS, SLAB_T), SPLIT ? KV(oQSL, SLAB_T) : NONE, KST_T, MV(OFF_S16, SLAB_C),
                 SPLIT ? MV(OFF_S16L, SLAB_C) : NONE, MST, D / 16, instr_desc(128, NV, fmt, MAJOR_K, MAJOR_MN), false);
       mma_commit(bar);
     }
@@ -513,7 +525,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
         tmem_wait_ld();
 #pragma unroll
         for (int i = 0; i < 8; ++i) w[i] = (c0 + i <= row) ? s[i] : 0.f;
-        put8(OFF_PM, OFF_PML, SLAB_T, row, c0, w, f16, SPLIT);
+        put8(OFF_PM, oPML, SLAB_T, row, c0, w, f16, SPLIT);
       }
     }
     __syncthreads();
@@ -521,11 +533,11 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
     publish();
     GTL(5);
     if (tid == 0) {
-      mma_split(COL_A, KV(OFF_PM, SLAB_T), SPLIT ? KV(OFF_PML, SLAB_T) : NONE, KST_T, MV(OFF_VP, SLAB_T), NONE, MST, C / 16,
+      mma_split(COL_A, KV(OFF_PM, SLAB_T), SPLIT ? KV(oPML, SLAB_T) : NONE, KST_T, MV(OFF_VP, SLAB_T), NONE, MST, C / 16,
                 instr_desc(128, NV, fmt, MAJOR_K, MAJOR_MN), true);
       // (two-term kh in the backward: the state must hold each key's contribution exactly as the reverse sweep's own
       // products see that key, or the pairs that cancel in the gate gradient leave their rounding behind)
-      mma_split(COL_ST, MV(OFF_KQ, SLAB_T), SPLIT ? MV(OFF_KQL, SLAB_T) : NONE, MST, MV(OFF_VP, SLAB_T), NONE, MST, C / 16,
+      mma_split(COL_ST, MV(OFF_KQ, SLAB_T), SPLIT ? MV(oKQL, SLAB_T) : NONE, MST, MV(OFF_VP, SLAB_T), NONE, MST, C / 16,
                 instr_desc(128, NV, fmt, MAJOR_MN, MAJOR_MN), true);
       mma_commit(bar);
     }
@@ -595,21 +607,22 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
     }
   }
 
+  if (MODE == 1) {  // the largest |do'| of the head, for the reverse sweep's scale
+    domax = warp_max(domax);
+    if (lane == 0) atomicMax(const_cast<int*>(&s_flags[4]), __float_as_int(domax < 3.0e38f ? domax : 3.0e38f));
+    __syncthreads();
+    if (tid == 0) a.ws_scale[bh] = __int_as_float(s_flags[4]);
+  }
   // ====================================================================================================== reverse sweep
-  if (BWD) {
+  if (MODE == 2) {
     // one power-of-two scale for do' over the whole head (every gradient is linear in do'): the largest |do'| lands just
     // below 2^8. The first tokens of a sequence have small denominators and a do' a hundred times the typical size; the
     // typical entries, and the adjoint state built from them, must stay clear of the fp16 subnormals. The masked score
     // gradients, sums of up to 65 such products, are saturated at the fp16 maximum.
-    domax = warp_max(domax);
-    if (lane == 0) atomicMax(const_cast<int*>(&s_flags[4]), __float_as_int(domax < 3.0e38f ? domax : 3.0e38f));
-    __syncthreads();
-    const float dm_all = fmaxf(__int_as_float(s_flags[4]), 1e-30f);
+    const float dm_all = fmaxf(a.ws_scale[bh], 1e-30f);
     const int ex = ((__float_as_int(dm_all) >> 23) & 0xff) - 127 + 1 - 8;           // 2^(ex + 8) > max |do'|
     const float sc = __int_as_float((127 - min(max(ex, -100), 100)) << 23);        // 2^-ex
     const float isc = __int_as_float((127 + min(max(ex, -100), 100)) << 23);       // 2^ex
-    __syncthreads();
-    load_state(false);  // R = 0
     bool prev_f16 = true;
     tc_fence_before_sync();
     __syncthreads();
@@ -675,7 +688,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
       publish();
       GTL(12);
       if (tid == 0) {
-        mma_split(COL_P, KV(OFF_QS, SLAB_T), KV(OFF_QSL, SLAB_T), KST_T, KV(OFF_KS, SLAB_T), KV(OFF_KSL, SLAB_T), KST_T,
+        mma_split(COL_P, KV(OFF_QS, SLAB_T), KV(oQSL, SLAB_T), KST_T, KV(OFF_KS, SLAB_T), KV(oKSL, SLAB_T), KST_T,
                   D / 16, instr_desc(128, C, fmt, MAJOR_K, MAJOR_K), false);
         // dO v^T with both operands exact: the row terms are applied in fp32 by the mask pass
         mma_chain(COL_DP, KV(OFF_DOX, SLAB_T), KST_T, KV(OFF_VP, SLAB_T), KST_T, D / 16,
@@ -697,7 +710,7 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
             s[i] = (c0 + i <= row) ? s[i] : 0.f;
             w[i] = (c0 + i <= row) ? fminf(fmaxf((w[i] - dl) * inv, -65000.f), 65000.f) : 0.f;
           }
-          put8(OFF_PM, OFF_PML, SLAB_T, row, c0, s, f16, true);
+          put8(OFF_PM, oPML, SLAB_T, row, c0, s, f16, true);
           put8(OFF_DPM, OFF_DPL, SLAB_T, row, c0, w, f16, true);
         }
       }
@@ -708,22 +721,22 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
                        ID_KK = instr_desc(128, D, fmt, MAJOR_K, MAJOR_K);
         const uint32_t IV_MM = instr_desc(128, NV, fmt, MAJOR_MN, MAJOR_MN), IV_KM = instr_desc(128, NV, fmt, MAJOR_K, MAJOR_MN);
         // dQ = dP ks + do' (2^bm S')^T
-        mma_split(COL_A, KV(OFF_DPM, SLAB_T), KV(OFF_DPL, SLAB_T), KST_T, MV(OFF_KS, SLAB_T), MV(OFF_KSL, SLAB_T), MST,
+        mma_split(COL_A, KV(OFF_DPM, SLAB_T), KV(OFF_DPL, SLAB_T), KST_T, MV(OFF_KS, SLAB_T), MV(oKSL, SLAB_T), MST,
                   C / 16, ID_KM, false);
         mma_split(COL_A, KV(OFF_DO, SLAB_T), KV(OFF_DOL, SLAB_T), KST_T, KV(OFF_S16, SLAB_C), KV(OFF_S16L, SLAB_C), KST_C,
                   NV / 16, ID_KK, true);
         // dK = dP^T qs + v' (2^ft R)^T
-        mma_split(COL_B, MV(OFF_DPM, SLAB_T), MV(OFF_DPL, SLAB_T), MST, MV(OFF_QS, SLAB_T), MV(OFF_QSL, SLAB_T), MST,
+        mma_split(COL_B, MV(OFF_DPM, SLAB_T), MV(OFF_DPL, SLAB_T), MST, MV(OFF_QS, SLAB_T), MV(oQSL, SLAB_T), MST,
                   C / 16, ID_MM, false);
         mma_split(COL_B, KV(OFF_VP, SLAB_T), NONE, KST_T, KV(OFF_R16, SLAB_C), KV(OFF_R16L, SLAB_C), KST_C, NV / 16, ID_KK,
                   true);
         // dV' = P^T do' + ks (2^ft R)
-        mma_split(COL_V, MV(OFF_PM, SLAB_T), MV(OFF_PML, SLAB_T), MST, MV(OFF_DO, SLAB_T), MV(OFF_DOL, SLAB_T), MST, C / 16,
+        mma_split(COL_V, MV(OFF_PM, SLAB_T), MV(oPML, SLAB_T), MST, MV(OFF_DO, SLAB_T), MV(OFF_DOL, SLAB_T), MST, C / 16,
                   IV_MM, false);
-        mma_split(COL_V, KV(OFF_KS, SLAB_T), KV(OFF_KSL, SLAB_T), KST_T, MV(OFF_R16, SLAB_C), MV(OFF_R16L, SLAB_C), MST,
+        mma_split(COL_V, KV(OFF_KS, SLAB_T), KV(oKSL, SLAB_T), KST_T, MV(OFF_R16, SLAB_C), MV(OFF_R16L, SLAB_C), MST,
                   D / 16, IV_KM, true);
         // R += (qs 2^bm)^T do'
-        mma_split(COL_ST, MV(OFF_KQ, SLAB_T), MV(OFF_KQL, SLAB_T), MST, MV(OFF_DO, SLAB_T), MV(OFF_DOL, SLAB_T), MST, C / 16,
+        mma_split(COL_ST, MV(OFF_KQ, SLAB_T), MV(oKQL, SLAB_T), MST, MV(OFF_DO, SLAB_T), MV(OFF_DOL, SLAB_T), MST, C / 16,
                   IV_MM, true);
         mma_commit(bar);
       }
@@ -746,11 +759,11 @@ __global__ void __launch_bounds__(THREADS, BWD ? 1 : 2) gla_tc_kernel(const GArg
           {
             float lo[8];
             unpack8h(*reinterpret_cast<const uint4*>(sg + OFF_QS + toff(SLAB_T, row, c0)), f16, rq);
-            unpack8h(*reinterpret_cast<const uint4*>(sg + OFF_QSL + toff(SLAB_T, row, c0)), f16, lo);
+            unpack8h(*reinterpret_cast<const uint4*>(sg + oQSL + toff(SLAB_T, row, c0)), f16, lo);
 #pragma unroll
             for (int i = 0; i < 8; ++i) rq[i] += lo[i];
             unpack8h(*reinterpret_cast<const uint4*>(sg + OFF_KS + toff(SLAB_T, row, c0)), f16, rk);
-            unpack8h(*reinterpret_cast<const uint4*>(sg + OFF_KSL + toff(SLAB_T, row, c0)), f16, lo);
+            unpack8h(*reinterpret_cast<const uint4*>(sg + oKSL + toff(SLAB_T, row, c0)), f16, lo);
 #pragma unroll
             for (int i = 0; i < 8; ++i) rk[i] += lo[i];
           }
@@ -871,9 +884,13 @@ static int set_smem_once() {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LAWCAT_ERR_CUDA;
   std::lock_guard<std::mutex> lk(mu);
   if (!done[dev]) {
-    if (cudaFuncSetAttribute(gla_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_FWD) != cudaSuccess ||
-        cudaFuncSetAttribute(gla_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BWD) != cudaSuccess)
+    cudaError_t e = cudaFuncSetAttribute(gla_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_FWD);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gla_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_SWEEP);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gla_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BWD);
+    if (e != cudaSuccess) {
+      note_cuda_error(e, __FILE__, __LINE__);
       return LAWCAT_ERR_CUDA;
+    }
     done[dev] = true;
   }
   return LAWCAT_OK;
@@ -898,6 +915,7 @@ bool gla_tc_supported(const lawcat_params& p) {
 size_t gla_tc_bwd_workspace_bytes(const lawcat_params& p) {
   const size_t bth = (size_t)p.B * p.T * p.H, chunks = (p.T + gtc::C - 1) / gtc::C;
   return align_up(sizeof(float) * bth * gtc::D, 256) + 2 * align_up(sizeof(float) * bth, 256) +
+         align_up(sizeof(float) * (size_t)p.B * p.H, 256) +
          align_up((size_t)p.B * p.H * chunks * (2 * gtc::TILE_CV + 16), 256);
 }
 
@@ -920,7 +938,7 @@ int launch_gla_fwd_tc(const Ctx& c, const void* qdot, const void* kdot, const vo
   a.qdot = qdot; a.kdot = kdot; a.v = (const bf16*)v; a.gate = (const bf16*)gate;
   a.S0 = S0; a.z0 = z0; a.o = (bf16*)o; a.den = den; a.S_T = S_T; a.z_T = z_T; a.feat_f32 = feat_f32 ? 1 : 0;
   LaunchScope _ls("gla_tc_fwd", c.stream);
-  gla_tc_kernel<false><<<p.B * p.H, THREADS, SMEM_FWD, c.stream>>>(a);
+  gla_tc_kernel<0><<<p.B * p.H, THREADS, SMEM_FWD, c.stream>>>(a);
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }
@@ -941,10 +959,16 @@ int launch_gla_bwd_tc(const Ctx& c, const void* qdot, const void* kdot, const vo
   a.dvh = (float*)w; w += align_up(sizeof(float) * bth * D, 256);
   a.ws_den = (float*)w; w += align_up(sizeof(float) * bth, 256);
   a.ws_delta = (float*)w; w += align_up(sizeof(float) * bth, 256);
+  a.ws_scale = (float*)w; w += align_up(sizeof(float) * (size_t)p.B * p.H, 256);
   a.ws_s16 = (uint8_t*)w;
   {
+    LaunchScope _ls("gla_tc_bwd_sweep", c.stream);
+    gla_tc_kernel<1><<<p.B * p.H, THREADS, SMEM_SWEEP, c.stream>>>(a);
+    LAWCAT_CHECK_LAUNCH();
+  }
+  {
     LaunchScope _ls("gla_tc_bwd", c.stream);
-    gla_tc_kernel<true><<<p.B * p.H, THREADS, SMEM_BWD, c.stream>>>(a);
+    gla_tc_kernel<2><<<p.B * p.H, THREADS, SMEM_BWD, c.stream>>>(a);
     LAWCAT_CHECK_LAUNCH();
   }
   const size_t total = (size_t)p.B * p.T * p.H_kv * (D / 8);

@@ -37,6 +37,14 @@ LaunchScope::~LaunchScope() {
   std::lock_guard<std::mutex> lk(g_mu);
   cudaEventRecord(g_recs[idx].b, stream);
 }
+
+static thread_local char t_cuda_error[256] = "";
+
+void note_cuda_error(cudaError_t e, const char* file, int line) {
+  const char* base = strrchr(file, '/');
+  snprintf(t_cuda_error, sizeof(t_cuda_error), "%s (%s) at %s:%d", cudaGetErrorString(e), cudaGetErrorName(e),
+           base ? base + 1 : file, line);
+}
 }  // namespace lawcat
 
 using namespace lawcat;
@@ -44,6 +52,8 @@ using namespace lawcat;
 extern "C" {
 
 unsigned long long lawcat_launch_count(void) { return g_launches.load(); }
+
+const char* lawcat_last_cuda_error(void) { return t_cuda_error; }
 
 int lawcat_trace_begin(void) {
   std::lock_guard<std::mutex> lk(g_mu);
