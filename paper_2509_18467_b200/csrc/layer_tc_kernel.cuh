@@ -40,11 +40,20 @@ namespace tc {
 // Optional time line (profiling builds only, -DLAWCAT_TIMELINE): one lane per role of thread block 0 stamps the clock at
 // fixed points of four consecutive chunks into a device array that lawcat_timeline_read copies out.
 #ifdef LAWCAT_TIMELINE
-constexpr int TL_ROLES = 6, TL_IDS = 16, TL_N0 = 40, TL_NCH = 4;
+#ifndef LAWCAT_TIMELINE_MODE
+#define LAWCAT_TIMELINE_MODE 0   // which kernel mode stamps: 0 the layer, 1 the state-only pass
+#endif
+#ifndef LAWCAT_TIMELINE_N0
+#define LAWCAT_TIMELINE_N0 40    // first of the four chunks that stamp
+#endif
+#ifndef LAWCAT_TL_BLOCK
+#define LAWCAT_TL_BLOCK 0        // the thread block whose pending waits are recorded when a wait runs out
+#endif
+constexpr int TL_ROLES = 6, TL_IDS = 16, TL_N0 = LAWCAT_TIMELINE_N0, TL_NCH = 4;
 __device__ long long g_timeline[TL_ROLES * TL_IDS * TL_NCH];
 #define TL(role, id, n, who)                                                                        \
   do {                                                                                              \
-    if (MODE == 0 && blockIdx.x == 0 && (who) && (n) >= TL_N0 && (n) < TL_N0 + TL_NCH)              \
+    if (MODE == LAWCAT_TIMELINE_MODE && blockIdx.x == 0 && (who) && (n) >= TL_N0 && (n) < TL_N0 + TL_NCH) \
       g_timeline[((role) * TL_IDS + (id)) * TL_NCH + ((n) - TL_N0)] = clock64();                    \
   } while (0)
 #else
@@ -217,6 +226,14 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
 #pragma unroll 1
     for (int i = 0; i < batch; ++i)
       if (mbar_try_wait(bar, parity)) return true;
+#ifdef LAWCAT_TIMELINE
+    // (profiling builds) when a wait runs out, every warp of one block notes the barrier it is waiting for: entry 0 of the
+    // time line counts the notes, each note = barrier index | parity << 8 | thread << 16 | kind << 40
+    if ((*abort_flag || clock64() - t0 > limit) && blockIdx.x == LAWCAT_TL_BLOCK && (threadIdx.x & 31) == 0) {
+      const unsigned long long i = atomicAdd(reinterpret_cast<unsigned long long*>(&g_timeline[0]), 1ull);
+      if (i < 40) g_timeline[1 + i] = (long long)(((bar & 1023u) - (OFF_BAR & 1023u)) / 8u) | ((long long)parity << 8) | ((long long)threadIdx.x << 16) | (1ll << 40);
+    }
+#endif
     if (*abort_flag) return false;
     if (clock64() - t0 > limit) {
       *abort_flag = 1;
@@ -250,6 +267,12 @@ __device__ __forceinline__ bool wait_set_or_abort(uint32_t bar0, uint32_t mask, 
       }
     }
     bool stop = *abort_flag != 0;
+#ifdef LAWCAT_TIMELINE
+    if ((stop || clock64() - t0 > limit) && !ok && blockIdx.x == LAWCAT_TL_BLOCK) {
+      const unsigned long long i = atomicAdd(reinterpret_cast<unsigned long long*>(&g_timeline[0]), 1ull);
+      if (i < 40) g_timeline[1 + i] = (long long)(((b & 1023u) - (OFF_BAR & 1023u)) / 8u) | ((long long)par << 8) | ((long long)threadIdx.x << 16) | (2ll << 40);
+    }
+#endif
     if (!stop && clock64() - t0 > limit) {
       *abort_flag = 1;
       stop = true;
