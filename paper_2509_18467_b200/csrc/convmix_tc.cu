@@ -32,6 +32,10 @@ struct CArgs {
   int B, T, H, Hkv, K, phi;
 };
 
+// hint: fetch the 128-byte line at p towards L2 (these kernels walk their tiles in lock-step; the hint lets the next
+// tile's rows travel while the current one is computed)
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 // raw rows [t0 - HALO, t0 + TT) of one head into shared memory (rows before the sequence come from the conv cache or are
 // zero, rows past its end are zero), and the head's taps as fp32 [D][4] (zero beyond the conv width)
 template <int D>
@@ -112,6 +116,11 @@ __global__ void __launch_bounds__(128) convmix_tc_fwd_kernel(const CArgs a) {
     const int NH = stream ? a.Hkv : a.H, head = stream ? j : h;
     load_raw_and_taps<D>(sg + OFF_RAW, reinterpret_cast<float*>(sg + OFF_TAPS), x, stream ? a.w_k : a.w_q,
                          stream ? a.cache_k : a.cache_q, b, t0, a.T, NH, head, a.K, tid, 128);
+    if (stream == 0 && t0 + tid < a.T) {  // the key stream's raw row of this thread, towards L2 meanwhile
+      const bf16* kr = a.k + (((size_t)b * a.T + t0 + tid) * a.Hkv + j) * D;
+      prefetch_l2(kr);
+      if (D * 2 > 128) prefetch_l2(kr + 64);
+    }
     __syncthreads();
     conv_tile<D>(sg + OFF_RAW, reinterpret_cast<const float*>(sg + OFF_TAPS), sg + OFF_U, tid, 128);
     fence_proxy_async();
@@ -228,6 +237,20 @@ __global__ void __launch_bounds__(128, 2) convmix_tc_bwd_kernel(const CArgs a) {
       const int NH = stream ? a.Hkv : a.H, head = stream ? j : h;
       load_raw_and_taps<D>(sg + OFF_RAW, reinterpret_cast<float*>(sg + OFF_TAPS), x, stream ? a.w_k : a.w_q,
                            stream ? a.cache_k : a.cache_q, b, t0, a.T, NH, head, a.K, tid, 128);
+      if (valid) {
+        // towards L2 while conv and mix run: this thread's row of the incoming gradient (read in the epilogue below),
+        // and its raw row of the next (head, stream) step
+        const char* dpr = reinterpret_cast<const char*>(stream ? a.d_kdot : a.d_qdot) +
+                          ((((size_t)b * a.T + t) * a.H + h) * D) * sizeof(TG);
+        prefetch_l2(dpr);
+        if (sizeof(TG) * D > 128) prefetch_l2(dpr + 128);
+        const int ns = stream ^ 1, ng = g + stream;  // the step that follows
+        if (ng < G) {
+          const bf16* nx = ns ? a.k : a.q;
+          const int nNH = ns ? a.Hkv : a.H, nhead = ns ? j : j * G + ng;
+          prefetch_l2(nx + (((size_t)b * a.T + t) * nNH + nhead) * D);
+        }
+      }
       __syncthreads();
       conv_tile<D>(sg + OFF_RAW, reinterpret_cast<const float*>(sg + OFF_TAPS), sg + OFF_U, tid, 128);
       fence_proxy_async();
