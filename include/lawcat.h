@@ -79,6 +79,9 @@ typedef struct {
   float gate_tau;    /* divisor of logsigmoid in LOGITS mode; 1 = the plain sigmoid gate */
   float eps;         /* added to the denominator of Eq. 8 */
   int32_t normalize; /* 1 = Eq. 8; 0 = numerator only (the "NN" ablation, Table 2) */
+  int32_t mix_unshared; /* 0 = one linear layer W[h] for the query and the key stream (Section 4.1, the paper's choice);
+                           1 = a separate one per stream (the "unshared linear" rows of the appendix table on sharing):
+                           W is then [2,H,d_k,d_k], query matrices first, and dW likewise */
 } lawcat_params;
 
 /* Scratch bytes entry point `op` (LAWCAT_OP_*) needs for these parameters; 0 on invalid parameters. */
@@ -122,6 +125,7 @@ void lawcat_test_set_wait_limit(long long cycles);
  * Causal depthwise conv on q and k (Section 4.1: qtilde_t = sum_delta w_delta q_{t-delta}), then, when W is not
  * NULL, the shared per-head linear layer and phi (Section 4.1; Section 4.2 defines qdot, kdot).
  *   q [B,T,H,d_k]  k [B,T,H_kv,d_k]  w_q [H*d_k,conv_k]  w_k [H_kv*d_k,conv_k]  W [H,d_k,d_k] or NULL
+ *   (p->mix_unshared = 1: W [2,H,d_k,d_k], the key stream mixes with W[1][h]; the same holds wherever W appears below)
  *   cache_q [B,conv_k-1,H*d_k], cache_k [B,conv_k-1,H_kv*d_k]  (nullable)
  *   out, W != NULL: qdot [B,T,H,d_k], kdot [B,T,H,d_k]   (kdot per query head: phi uses W[h])
  *   out, W == NULL: qdot = conv(q) [B,T,H,d_k], kdot = conv(k) [B,T,H_kv,d_k]

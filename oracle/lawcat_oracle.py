@@ -132,23 +132,32 @@ def gla_bwd(p: OracleParams, qdot, kdot, v, gate, dO, S0=None, z0=None):
 
 
 def conv_bwd(p: OracleParams, q, k, w_q, w_k, W, d_qdot, d_kdot, cache_q=None, cache_k=None):
-    """Backward of conv (-> mix -> phi when W is given) on both streams. Returns dict(dq, dk, dw_q, dw_k, dW)."""
+    """Backward of conv (-> mix -> phi when W is given) on both streams. Returns dict(dq, dk, dw_q, dw_k, dW).
+    W [H,d,d]: one linear layer for both streams (dW sums both); W [2,H,d,d]: one per stream (dW likewise)."""
     q, k, w_q, w_k, W, d_qdot, d_kdot, cache_q, cache_k = map(
         _f64, (q, k, w_q, w_k, W, d_qdot, d_kdot, cache_q, cache_k))
     B, T, H, Hkv, d, K = p.B, p.T, p.H, p.H_kv, p.d_k, p.conv_k
     dq, dk = np.empty_like(q), np.empty_like(k)
     dw_q, dw_k = np.empty_like(w_q), np.empty_like(w_k)
     dW = None if W is None else np.zeros_like(W)
+    unshared = W is not None and W.ndim == 4
+    Wq, Wk = (np.ascontiguousarray(W[0]), np.ascontiguousarray(W[1])) if unshared else (W, W)
+    dWq, dWk = (np.zeros_like(Wq), np.zeros_like(Wk)) if unshared else (dW, dW)
     L = _L()
-    L.oracle_conv_mix_bwd(_p(q), _p(w_q), _p(cache_q), _p(W), _p(d_qdot), B, T, H, H, d, K, p.phi, _p(dq),
-                          _p(dw_q), _p(dW))
-    L.oracle_conv_mix_bwd(_p(k), _p(w_k), _p(cache_k), _p(W), _p(d_kdot), B, T, Hkv, H if W is not None else Hkv,
-                          d, K, p.phi, _p(dk), _p(dw_k), _p(dW))
+    L.oracle_conv_mix_bwd(_p(q), _p(w_q), _p(cache_q), _p(Wq), _p(d_qdot), B, T, H, H, d, K, p.phi, _p(dq),
+                          _p(dw_q), _p(dWq))
+    L.oracle_conv_mix_bwd(_p(k), _p(w_k), _p(cache_k), _p(Wk), _p(d_kdot), B, T, Hkv, H if W is not None else Hkv,
+                          d, K, p.phi, _p(dk), _p(dw_k), _p(dWk))
+    if unshared:
+        dW = np.stack([dWq, dWk])
     return dict(dq=dq, dk=dk, dw_q=dw_q, dw_k=dw_k, dW=dW)
 
 
 def layer_fwd(p: OracleParams, q, k, v, gate, w_q, w_k, W, cache_q=None, cache_k=None, S0=None, z0=None):
-    """The whole layer (Fig. 1). Returns dict(o, den, qdot, kdot, cache_q, cache_k, S_T, z_T)."""
+    """The whole layer (Fig. 1). Returns dict(o, den, qdot, kdot, cache_q, cache_k, S_T, z_T).
+    W [2,H,d,d] = a separate linear layer per stream (appendix table on sharing): the same steps, composed here."""
+    if W is not None and np.ndim(W) == 4:
+        return _layer_fwd_unshared(p, q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0)
     q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0 = map(
         _f64, (q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0))
     cp = p.c()
@@ -165,6 +174,22 @@ def layer_fwd(p: OracleParams, q, k, v, gate, w_q, w_k, W, cache_q=None, cache_k
                           _p(cache_k), _p(S0), _p(z0), _p(o), _p(den), _p(qd), _p(kd), _p(cq), _p(ck), _p(S_T),
                           _p(z_T))
     return dict(o=o, den=den, qdot=qd, kdot=kd, cache_q=cq, cache_k=ck, S_T=S_T, z_T=z_T)
+
+
+def _layer_fwd_unshared(p, q, k, v, gate, w_q, w_k, W, cache_q, cache_k, S0, z0):
+    """conv (Section 4.1) -> linear layer of the stream + phi -> Eq. 4 / Eq. 8, from the same primitives as the shared form;
+    the conv caches are the last K - 1 raw rows of [cache, x]."""
+    W = _f64(W)
+    K = p.conv_k
+    qd = mix_phi(conv(q, w_q, cache_q, K), W[0], p.H, p.phi)
+    kd = mix_phi(conv(k, w_k, cache_k, K), W[1], p.H, p.phi)
+    r = gla_fwd(p, qd, kd, v, gate, S0, z0)
+    def tail(x, cache):
+        x = _f64(x).reshape(p.B, p.T, -1)
+        c = np.zeros((p.B, K - 1, x.shape[2])) if cache is None else _f64(cache).reshape(p.B, K - 1, -1)
+        return np.concatenate([c, x], 1)[:, p.T:]
+    return dict(o=r["o"], den=r["den"], qdot=qd, kdot=kd, cache_q=tail(q, cache_q), cache_k=tail(k, cache_k),
+                S_T=r["S_T"], z_T=r["z_T"])
 
 
 def decode_step(p: OracleParams, q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cache_q, cache_k):

@@ -44,15 +44,15 @@ class Params(ctypes.Structure):
                 ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("conv_k", ctypes.c_int32),
                 ("gate_dim", ctypes.c_int32), ("chunk", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("phi", ctypes.c_int32), ("gate_mode", ctypes.c_int32), ("gate_tau", ctypes.c_float),
-                ("eps", ctypes.c_float), ("normalize", ctypes.c_int32)]
+                ("eps", ctypes.c_float), ("normalize", ctypes.c_int32), ("mix_unshared", ctypes.c_int32)]
 
 
 def params(B, T, H, H_kv, d_k, d_v, conv_k=4, gate_dim=0, chunk=0, dtype=BF16, phi=PHI_SOFTMAX,
-           gate_mode=GATE_LOGITS, gate_tau=16.0, eps=0.0, normalize=1) -> Params:
+           gate_mode=GATE_LOGITS, gate_tau=16.0, eps=0.0, normalize=1, mix_unshared=0) -> Params:
     if isinstance(dtype, str):
         dtype = {"f32": F32, "bf16": BF16}[dtype]
     return Params(B, T, H, H_kv, d_k, d_v, conv_k, gate_dim or d_k, chunk, dtype, phi, gate_mode, gate_tau, eps,
-                  normalize)
+                  normalize, mix_unshared)
 
 
 _lib = None

@@ -20,6 +20,7 @@ int check_params(const lawcat_params* p, bool need_T) {
   if (p->gate_mode != LAWCAT_GATE_LOGITS && p->gate_mode != LAWCAT_GATE_LOGDECAY) return LAWCAT_ERR_INVALID_ARG;
   if (!(p->gate_tau > 0.f) || !(p->eps >= 0.f)) return LAWCAT_ERR_INVALID_ARG;
   if (p->normalize != 0 && p->normalize != 1) return LAWCAT_ERR_INVALID_ARG;
+  if (p->mix_unshared != 0 && p->mix_unshared != 1) return LAWCAT_ERR_INVALID_ARG;
   if (p->chunk < 0) return LAWCAT_ERR_INVALID_ARG;
   if (!pow2_dim(p->d_k) || !pow2_dim(p->d_v)) return LAWCAT_ERR_UNSUPPORTED;
   if (p->conv_k < 1 || p->conv_k > 8) return LAWCAT_ERR_UNSUPPORTED;
@@ -80,7 +81,8 @@ ExactBwdLayout exact_bwd_layout(const lawcat_params* p) {
   p32.dtype = LAWCAT_F32;
   const size_t n_in[10] = {elems(p, p->H, p->d_k), elems(p, p->H_kv, p->d_k), elems(p, p->H_kv, p->d_v),
                            elems(p, p->H, p->gate_dim), (size_t)p->H * p->d_k * p->conv_k,
-                           (size_t)p->H_kv * p->d_k * p->conv_k, (size_t)p->H * p->d_k * p->d_k, elems(p, p->H, p->d_v),
+                           (size_t)p->H_kv * p->d_k * p->conv_k, (size_t)(1 + p->mix_unshared) * p->H * p->d_k * p->d_k,
+                           elems(p, p->H, p->d_v),
                            (size_t)p->B * (p->conv_k - 1) * p->H * p->d_k, (size_t)p->B * (p->conv_k - 1) * p->H_kv * p->d_k};
   size_t off = 0;
   auto take = [&](size_t bytes) { const size_t o = off; off += align_up(bytes, 256); return o; };
@@ -233,8 +235,8 @@ int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const
   float* kdot = (float*)((char*)ws + align_up(sizeof(float) * elems(p, p->H, p->d_k), 256));
   // The feature maps of Section 2 other than the softmax (1 + ELU, identity) on head width 64: tensor-core conv + mix +
   // phi into fp32 scratch, then the chunkwise tensor-core attention on those features.
-  if ((size_t)p->B * p->T != 0 && p->phi != LAWCAT_PHI_SOFTMAX && p->chunk != 1 && convmix_tc_fwd_supported(*p) &&
-      gla_tc_supported(*p)) {
+  if ((size_t)p->B * p->T != 0 && (p->phi != LAWCAT_PHI_SOFTMAX || p->mix_unshared) && p->chunk != 1 &&
+      convmix_tc_fwd_supported(*p) && gla_tc_supported(*p)) {
     if ((r = launch_convmix_tc_fwd(c, q, k, w_q, w_k, W, cache_q_in, cache_k_in, qdot, kdot, true))) return r;
     if ((r = launch_gla_fwd_tc(c, qdot, kdot, v, gate, S0, z0, o, nullptr, S_T, z_T, true))) return r;
     return launch_cache_out(c, q, k, cache_q_in, cache_k_in, cache_q_out, cache_k_out);
@@ -338,7 +340,8 @@ int lawcat_layer_bwd(const lawcat_params* p, const void* q, const void* k, const
   void* out[4] = {dq, dk, dv, dgate};
   const size_t n_in[10] = {elems(p, p->H, p->d_k), elems(p, p->H_kv, p->d_k), elems(p, p->H_kv, p->d_v),
                            elems(p, p->H, p->gate_dim), (size_t)p->H * p->d_k * p->conv_k,
-                           (size_t)p->H_kv * p->d_k * p->conv_k, (size_t)p->H * p->d_k * p->d_k, elems(p, p->H, p->d_v),
+                           (size_t)p->H_kv * p->d_k * p->conv_k, (size_t)(1 + p->mix_unshared) * p->H * p->d_k * p->d_k,
+                           elems(p, p->H, p->d_v),
                            (size_t)p->B * (p->conv_k - 1) * p->H * p->d_k, (size_t)p->B * (p->conv_k - 1) * p->H_kv * p->d_k};
   const bool widen = p->dtype == LAWCAT_BF16;
   if (widen) {
@@ -425,7 +428,7 @@ static size_t host_arena_layout(const lawcat_params* p, size_t off[11]) {
                         elems(p, p->H_kv, p->d_v) * es,   // v
                         elems(p, p->H, p->gate_dim) * es, // gate
                         (size_t)p->H * p->d_k * p->conv_k * es, (size_t)p->H_kv * p->d_k * p->conv_k * es,
-                        (size_t)p->H * p->d_k * p->d_k * es,  // w_q, w_k, W
+                        (size_t)(1 + p->mix_unshared) * p->H * p->d_k * p->d_k * es,  // w_q, w_k, W
                         elems(p, p->H, p->d_v) * es,      // o
                         ws, 2 * host_state_set(p).bytes};
   size_t o = 0;
@@ -495,7 +498,7 @@ int lawcat_layer_fwd_host(const lawcat_params* p, const void* h_q, const void* h
   LAWCAT_HOST_TRY(cudaStreamWaitEvent(hp->out, e0, 0));
   const void* wsrc[3] = {h_w_q, h_w_k, h_W};
   const size_t wnb[3] = {(size_t)p->H * p->d_k * p->conv_k * es, (size_t)p->H_kv * p->d_k * p->conv_k * es,
-                         (size_t)p->H * p->d_k * p->d_k * es};
+                         (size_t)(1 + p->mix_unshared) * p->H * p->d_k * p->d_k * es};
   for (int i = 0; i < 3; ++i)
     LAWCAT_HOST_TRY(cudaMemcpyAsync(a + off[4 + i], wsrc[i], wnb[i], cudaMemcpyHostToDevice, hp->in));
   const HostStateSet hs = host_state_set(p);

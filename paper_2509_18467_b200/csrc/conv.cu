@@ -104,6 +104,7 @@ struct ConvMixArgs {
   const void *q, *k, *w_q, *w_k, *W, *cache_q, *cache_k;
   void *qdot, *kdot;
   int B, T, H, Hkv, d, K, phi;
+  int unshared;  // 1: W is [2,H,d,d], the key stream uses the second set
 };
 
 template <typename TI, typename TO>
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_fwd_kernel(ConvMixArgs a) 
   const TI* w = (const TI*)(stream ? a.w_k : a.w_q);
   const TI* cache = (const TI*)(stream ? a.cache_k : a.cache_q);
   TO* out = (TO*)(stream ? a.kdot : a.qdot);
-  const TI* Wh = (const TI*)a.W + (size_t)h * d * d;
+  const TI* Wh = (const TI*)a.W + ((size_t)(stream && a.unshared ? a.H : 0) + h) * d * d;
   const int tid = threadIdx.x, C = NH * d;
   for (int i = tid; i < d * d; i += CM_THREADS) Ws[i] = ldf(Wh + i);
   for (int i = tid; i < CM_TT * d; i += CM_THREADS) {
@@ -168,7 +169,8 @@ int launch_convmix_fwd(const Ctx& c, const void* q, const void* k, const void* w
   if (p.B * p.T == 0) return LAWCAT_OK;
   if (convmix_tc_fwd_supported(p) && !exact)  // tensor-core kernel
     return launch_convmix_tc_fwd(c, q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot, out_f32);
-  ConvMixArgs a{q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot, p.B, p.T, p.H, p.H_kv, p.d_k, p.conv_k, p.phi};
+  ConvMixArgs a{q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot, p.B, p.T, p.H, p.H_kv, p.d_k, p.conv_k, p.phi,
+                p.mix_unshared};
   const size_t smem = sizeof(float) * ((size_t)p.d_k * p.d_k + (size_t)CM_TT * p.d_k);
   dim3 grid(p.B * ((p.T + CM_TT - 1) / CM_TT), p.H, 2);
 #define LAUNCH_CM(TI, TO)                                                                                      \
@@ -199,6 +201,7 @@ struct ConvMixBwdArgs {
   const void *q, *k, *w_q, *w_k, *W, *cache_q, *cache_k, *d_qdot, *d_kdot;
   float *du_q, *du_k, *dW;
   int B, T, H, Hkv, K, phi;
+  int unshared;  // 1: W and dW are [2,H,D,D], the key stream uses the second set
 };
 
 template <typename TI, int D>
@@ -219,10 +222,13 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_bwd_kernel(ConvMixBwdArgs 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   for (int gi = 0; gi < G; ++gi) {
     const int h = j * G + gi;
-    const TI* Wh = (const TI*)a.W + (size_t)h * D * D;
-    __syncthreads();
-    for (int i = tid; i < D * D; i += CM_THREADS) Ws[(i / D) * LDW + (i % D)] = ldf(Wh + i);
     for (int stream = 0; stream < 2; ++stream) {
+      const size_t wset = (size_t)(stream && a.unshared ? a.H : 0) + h;  // which matrix of W / dW
+      if (stream == 0 || a.unshared) {
+        const TI* Wh = (const TI*)a.W + wset * D * D;
+        __syncthreads();
+        for (int i = tid; i < D * D; i += CM_THREADS) Ws[(i / D) * LDW + (i % D)] = ldf(Wh + i);
+      }
       const int NH = stream ? a.Hkv : a.H, n = stream ? j : h, C = NH * D;
       const TI* x = (const TI*)(stream ? a.k : a.q);
       const TI* w = (const TI*)(stream ? a.w_k : a.w_q);
@@ -352,7 +358,7 @@ __global__ void __launch_bounds__(CM_THREADS) convmix_bwd_kernel(ConvMixBwdArgs 
             for (int i = 0; i < 4; ++i)
 #pragma unroll
               for (int jj = 0; jj < 4; ++jj)
-                atomicAdd(a.dW + (size_t)h * D * D + (size_t)(4 * cb + i) * D + 4 * eb + jj, dWacc[m][4 * i + jj]);
+                atomicAdd(a.dW + wset * D * D + (size_t)(4 * cb + i) * D + 4 * eb + jj, dWacc[m][4 * i + jj]);
           }
         }
       }
@@ -450,7 +456,7 @@ static int conv_bwd_typed(const Ctx& c, const void* q, const void* k, const void
   if (p.B * p.T == 0) {
     if (dw_q && cudaMemsetAsync(dw_q, 0, sizeof(float) * (size_t)p.H * p.d_k * p.conv_k, c.stream)) return LAWCAT_ERR_CUDA;
     if (dw_k && cudaMemsetAsync(dw_k, 0, sizeof(float) * (size_t)p.H_kv * p.d_k * p.conv_k, c.stream)) return LAWCAT_ERR_CUDA;
-    if (dW && cudaMemsetAsync(dW, 0, sizeof(float) * (size_t)p.H * p.d_k * p.d_k, c.stream)) return LAWCAT_ERR_CUDA;
+    if (dW && cudaMemsetAsync(dW, 0, sizeof(float) * (size_t)(1 + p.mix_unshared) * p.H * p.d_k * p.d_k, c.stream)) return LAWCAT_ERR_CUDA;
     return LAWCAT_OK;
   }
   if (!W) {
@@ -462,10 +468,10 @@ static int conv_bwd_typed(const Ctx& c, const void* q, const void* k, const void
   }
   float* du_q = (float*)ws;
   float* du_k = (float*)((char*)ws + align_up(sizeof(float) * (size_t)p.B * p.T * p.H * p.d_k, 256));
-  if (dW && cudaMemsetAsync(dW, 0, sizeof(float) * (size_t)p.H * p.d_k * p.d_k, c.stream) != cudaSuccess)
+  if (dW && cudaMemsetAsync(dW, 0, sizeof(float) * (size_t)(1 + p.mix_unshared) * p.H * p.d_k * p.d_k, c.stream) != cudaSuccess)
     return LAWCAT_ERR_CUDA;
   ConvMixBwdArgs a{q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, du_q, du_k, dW,
-                   p.B, p.T, p.H, p.H_kv, p.conv_k, p.phi};
+                   p.B, p.T, p.H, p.H_kv, p.conv_k, p.phi, p.mix_unshared};
   if (std::is_same<TI, bf16>::value && convmix_tc_bwd_supported(p) && p.chunk != 1) {
     // tensor-core kernel for the mix and the softmax Jacobian; the conv's own backward follows on du as below
     int r0 = launch_convmix_tc_bwd(c, q, k, w_q, w_k, W, cache_q, cache_k, d_qdot, d_kdot, grads_f32, du_q, du_k, dW);

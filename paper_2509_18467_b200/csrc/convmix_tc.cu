@@ -30,6 +30,7 @@ struct CArgs {
   float *du_q, *du_k, *dW;           // backward outputs: d(conv out) per stream (fp32), dW (fp32, atomic adds)
   int* dev_status;
   int B, T, H, Hkv, K, phi;
+  int unshared;  // 1: W is [2,H,D,D], the key stream mixes with the second set (forward kernel only)
 };
 
 // hint: fetch the 128-byte line at p towards L2 (these kernels walk their tiles in lock-step; the hint lets the next
@@ -114,6 +115,9 @@ __global__ void __launch_bounds__(128) convmix_tc_fwd_kernel(const CArgs a) {
   for (int stream = 0; stream < 2; ++stream) {
     const bf16* x = stream ? a.k : a.q;
     const int NH = stream ? a.Hkv : a.H, head = stream ? j : h;
+    // (a separate linear layer per stream: the key stream's W_h replaces the tile; the product that read the query
+    // stream's has completed, and the barriers below publish the new tile together with the conv output)
+    if (stream == 1 && a.unshared) load_w_tile<D>(sg + OFF_WT, a.W + ((size_t)a.H + h) * D * D, tid, 128);
     load_raw_and_taps<D>(sg + OFF_RAW, reinterpret_cast<float*>(sg + OFF_TAPS), x, stream ? a.w_k : a.w_q,
                          stream ? a.cache_k : a.cache_q, b, t0, a.T, NH, head, a.K, tid, 128);
     if (stream == 0 && t0 + tid < a.T) {  // the key stream's raw row of this thread, towards L2 meanwhile
@@ -400,7 +404,7 @@ bool convmix_tc_fwd_supported(const lawcat_params& p) {
 }
 bool convmix_tc_bwd_supported(const lawcat_params& p) {
   return p.dtype == LAWCAT_BF16 && p.d_k == 64 && p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= ctc::HALO + 1 && p.B > 0 &&
-         p.T > 0;
+         p.T > 0 && !p.mix_unshared;
 }
 
 static ctc::CArgs convmix_tc_args(const Ctx& c, const void* q, const void* k, const void* w_q, const void* w_k, const void* W,
@@ -410,7 +414,7 @@ static ctc::CArgs convmix_tc_args(const Ctx& c, const void* q, const void* k, co
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.w_q = (const bf16*)w_q; a.w_k = (const bf16*)w_k; a.W = (const bf16*)W;
   a.cache_q = (const bf16*)cache_q; a.cache_k = (const bf16*)cache_k;
   a.dev_status = c.dev_status;
-  a.B = p.B; a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k; a.phi = p.phi;
+  a.B = p.B; a.T = p.T; a.H = p.H; a.Hkv = p.H_kv; a.K = p.conv_k; a.phi = p.phi; a.unshared = p.mix_unshared;
   return a;
 }
 

@@ -26,6 +26,7 @@ struct DecodeArgs {
   float* den;   // workspace [B*H]
   int B, H, Hkv, dk, dv, K, gd, phi, gate_mode, normalize;
   int w_smem;  // 1: W of the head is staged in shared memory
+  int unshared;  // 1: W is [2,H,dk,dk], the key stream's vectors mix with the second set
   float inv_tau, eps;
   int* dev_status;
 };
@@ -145,14 +146,16 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_features_kernel(DecodeArgs
   // serves the four vectors
   {
     const T* Wh = (const T*)a.W + (size_t)h * dk * dk;
+    const T* Wk = Wh + (a.unshared ? (size_t)H * dk * dk : 0);  // (vectors 4 vg + 1, 4 vg + 3 are key-stream vectors)
     for (int it = tid; it < dk * (DEC_NV / 4); it += DEC_THREADS) {
       const int e = it % dk, vg = it / dk;
       float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 8
       for (int c = 0; c < dk; ++c) {
         const float w = a.w_smem ? ldf(s_W + c * dk + e) : ldf(Wh + (size_t)c * dk + e);
+        const float wk = a.unshared ? ldf(Wk + (size_t)c * dk + e) : w;
         const float4 u = *reinterpret_cast<const float4*>(s_u + c * DEC_NV + 4 * vg);
-        y.x = fmaf(u.x, w, y.x); y.y = fmaf(u.y, w, y.y); y.z = fmaf(u.z, w, y.z); y.w = fmaf(u.w, w, y.w);
+        y.x = fmaf(u.x, w, y.x); y.y = fmaf(u.y, wk, y.y); y.z = fmaf(u.z, w, y.z); y.w = fmaf(u.w, wk, y.w);
       }
       s_y[(4 * vg + 0) * dk + e] = y.x; s_y[(4 * vg + 1) * dk + e] = y.y;
       s_y[(4 * vg + 2) * dk + e] = y.z; s_y[(4 * vg + 3) * dk + e] = y.w;
@@ -458,7 +461,7 @@ __global__ void __launch_bounds__(DFT_THREADS) decode_features_tc_kernel(DecodeA
 }
 
 bool decode_tc_supported(const lawcat_params& p) {
-  return p.dtype == LAWCAT_BF16 && (p.d_k == 64 || p.d_k == 128) && p.conv_k <= 4 && p.chunk != 1;
+  return p.dtype == LAWCAT_BF16 && (p.d_k == 64 || p.d_k == 128) && p.conv_k <= 4 && p.chunk != 1 && !p.mix_unshared;
 }
 
 template <int D>
@@ -585,7 +588,7 @@ static int decode_typed(const Ctx& c, DecodeArgs& a) {
     size_t smem1 = sizeof(float) * (size_t)p.d_k * (2 * DEC_NV + DEC_SEQ) + sizeof(T) * (size_t)p.d_k * p.conv_k * (DEC_NV + 2);
     if (p.d_k > 32 * DEC_ZR) return LAWCAT_ERR_UNSUPPORTED;  // (one warp holds a sequence's normalizer state)
     const size_t wbytes = sizeof(T) * (size_t)p.d_k * p.d_k;
-    a.w_smem = smem1 + wbytes <= 100 * 1024 ? 1 : 0;
+    a.w_smem = (!p.mix_unshared && smem1 + wbytes <= 100 * 1024) ? 1 : 0;  // (two sets of W are read from L2 in place)
     if (a.w_smem) smem1 += wbytes;
     if (smem1 > 48 * 1024 &&
         cudaFuncSetAttribute(decode_features_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess)
@@ -625,7 +628,7 @@ int launch_decode(const Ctx& c, const void* q_t, const void* k_t, const void* v_
   a.den = a.vecs + (size_t)p.B * p.H * 3 * p.d_k;
   a.B = p.B; a.H = p.H; a.Hkv = p.H_kv; a.dk = p.d_k; a.dv = p.d_v; a.K = p.conv_k; a.gd = p.gate_dim;
   a.phi = p.phi; a.gate_mode = p.gate_mode; a.normalize = p.normalize;
-  a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps; a.dev_status = c.dev_status;
+  a.inv_tau = 1.f / p.gate_tau; a.eps = p.eps; a.dev_status = c.dev_status; a.unshared = p.mix_unshared;
   if (p.dtype == LAWCAT_F32) return decode_typed<float>(c, a);
   return decode_typed<bf16>(c, a);
 }

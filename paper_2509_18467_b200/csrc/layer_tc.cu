@@ -162,7 +162,8 @@ bool layer_tc_supported(const lawcat_params& p) {
   return p.dtype == LAWCAT_BF16 && (p.d_k == tc::D || p.d_k == 64) && p.d_v == p.d_k &&
          (p.gate_dim == p.d_k || p.gate_dim == 1) && !sharp_unsupported &&
          p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
-         (p.chunk == 0 || p.chunk == tc::C);
+         (p.chunk == 0 || p.chunk == tc::C) &&
+         !p.mix_unshared;  // (one W_h is what lets both streams share the M = 128 mix)
 }
 
 int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, const void* gate, const void* w_q,

@@ -416,3 +416,47 @@ def test_whole_layer_gradient_chain():
     for name, got in (("q", g2["dq"]), ("k", g2["dk"]), ("v", g1["dv"]), ("gate", g1["dgate"]),
                       ("w_q", g2["dw_q"]), ("w_k", g2["dw_k"]), ("W", g2["dW"])):
         np.testing.assert_allclose(got, _fd(f, x[name], dO), rtol=5e-6, atol=1e-8, err_msg=name)
+
+
+# --------------------------------------------------------------------------- a separate linear layer per stream
+def test_unshared_linear_with_equal_matrices_is_the_shared_layer():
+    """Appendix table on sharing: the unshared form with W_q = W_k is the shared layer, and its two weight gradients add
+    up to the shared one."""
+    B, T, H, Hkv, d = 2, 7, 4, 2, 3
+    p = O.OracleParams(B, T, H, Hkv, d, d)
+    x = _layer_inputs(B, T, H, Hkv, d, d)
+    a = O.layer_fwd(p, **x)
+    y = dict(x)
+    y["W"] = np.stack([x["W"], x["W"]])
+    b = O.layer_fwd(p, **y)
+    for n in ("o", "qdot", "kdot", "S_T", "z_T", "cache_q", "cache_k"):
+        np.testing.assert_allclose(b[n], a[n], rtol=1e-13, atol=1e-15, err_msg=n)
+    dqd, dkd = rnd(B, T, H, d), rnd(B, T, H, d)
+    g = O.conv_bwd(p, x["q"], x["k"], x["w_q"], x["w_k"], x["W"], dqd, dkd)
+    gu = O.conv_bwd(p, x["q"], x["k"], x["w_q"], x["w_k"], y["W"], dqd, dkd)
+    np.testing.assert_allclose(gu["dW"][0] + gu["dW"][1], g["dW"], rtol=1e-12, atol=1e-14)
+    for n in ("dq", "dk", "dw_q", "dw_k"):
+        np.testing.assert_allclose(gu[n], g[n], rtol=1e-13, atol=1e-15, err_msg=n)
+
+
+def test_unshared_linear_streams_are_independent_and_gradients_match_finite_differences():
+    B, T, H, Hkv, d, K = 1, 5, 2, 1, 3, 3
+    p = O.OracleParams(B, T, H, Hkv, d, d, conv_k=K, gate_tau=1.0)
+    q, k, v, gate = rnd(B, T, H, d), rnd(B, T, Hkv, d), rnd(B, T, Hkv, d), rnd(B, T, H, d)
+    wq, wk, W = rnd(H * d, K), rnd(Hkv * d, K), rnd(2, H, d, d)
+    base = O.layer_fwd(p, q, k, v, gate, wq, wk, W)
+    # the key stream's matrices do not touch qdot, and the other way round
+    W2 = W.copy()
+    W2[1] += 0.5
+    np.testing.assert_array_equal(O.layer_fwd(p, q, k, v, gate, wq, wk, W2)["qdot"], base["qdot"])
+    W3 = W.copy()
+    W3[0] += 0.5
+    np.testing.assert_array_equal(O.layer_fwd(p, q, k, v, gate, wq, wk, W3)["kdot"], base["kdot"])
+    # whole-layer gradient chain against finite differences
+    dO = rnd(B, T, H, d)
+    g1 = O.gla_bwd(p, base["qdot"], base["kdot"], v, gate, dO)
+    g2 = O.conv_bwd(p, q, k, wq, wk, W, g1["d_qdot"], g1["d_kdot"])
+    f = lambda: O.layer_fwd(p, q, k, v, gate, wq, wk, W)["o"]
+    for name, arr, got in (("q", q, g2["dq"]), ("k", k, g2["dk"]), ("w_q", wq, g2["dw_q"]), ("w_k", wk, g2["dw_k"]),
+                           ("W", W, g2["dW"])):
+        np.testing.assert_allclose(got, _fd(f, arr, dO), rtol=5e-6, atol=1e-8, err_msg=name)
