@@ -156,8 +156,9 @@ int lawcat_conv_bwd(const lawcat_params* p, const void* q, const void* k, const 
  *   S0 [B,H,d_k,d_v] fp32, z0 [B,H,d_k] fp32: state before token 0 (nullable = zero, Eq. 5)
  *   out: o [B,T,H,d_v]; den [B,T,H] fp32 = qdot_t . z_t + eps (nullable; gla_bwd needs it);
  *        S_T, z_T = state after the last token (nullable)
- * Kernels: bf16 storage with d_k = d_v = 64 runs chunkwise (64 tokens) on the tensor cores; every other case, and
- * chunk = 1, runs the exact recurrence. ws: lawcat_workspace_bytes(p, LAWCAT_OP_GLA_FWD).
+ * Kernels: bf16 storage with d_k = d_v = 64 runs chunkwise (64 tokens) on the tensor cores, with the same two exceptions
+ * and the same LAWCAT_ERR_NUMERIC report as lawcat_layer_fwd (sharp sigmoid gates, calls of fewer than 16 tokens); every
+ * other case, and chunk = 1, runs the exact recurrence. ws: lawcat_workspace_bytes(p, LAWCAT_OP_GLA_FWD).
  */
 int lawcat_gla_fwd(const lawcat_params* p, const void* qdot, const void* kdot, const void* v, const void* gate,
                    const float* S0, const float* z0, void* o, float* den, float* S_T, float* z_T, void* ws,
@@ -170,9 +171,9 @@ int lawcat_gla_fwd(const lawcat_params* p, const void* qdot, const void* kdot, c
  *   out: d_qdot, d_kdot [B,T,H,d_k]; dv [B,T,H_kv,d_v] (summed over the G query heads of a group);
  *        dgate [B,T,H,gate_dim] -- the gradient with respect to the `gate` input (logits or log-decays).
  * No gradient flows into S0, z0 and none is taken from S_T, z_T.
- * Kernels: bf16 storage with d_k = d_v = 64, and log-decay gates or sigmoid gates with gate_tau >= 8, runs the
- * chunkwise tensor-core backward (two-term fp16 operands: gradients within 1e-2 of their RMS); sharper gates, other
- * shapes and chunk = 1 run the exact three-sweep backward. ws: lawcat_workspace_bytes(p, LAWCAT_OP_GLA_BWD).
+ * Kernels: bf16 storage with d_k = d_v = 64, log-decay gates or sigmoid gates with gate_tau >= 8, and at least 16
+ * tokens runs the chunkwise tensor-core backward (two-term fp16 operands: gradients within 1e-2 of their RMS); sharper
+ * gates, shorter calls, other shapes and chunk = 1 run the exact three-sweep backward. ws: lawcat_workspace_bytes(p, LAWCAT_OP_GLA_BWD).
  */
 int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, const void* v, const void* gate,
                    const float* S0, const float* z0, const void* o, const float* den, const void* dO,
@@ -188,15 +189,17 @@ int lawcat_gla_bwd(const lawcat_params* p, const void* qdot, const void* kdot, c
  * The *_out buffers must not alias the *_in buffers.
  * bf16 storage with d_k = d_v in {64, 128}, the softmax feature map, conv_k <= 4 and chunk in {0, 64} run on the
  * chunkwise tensor-core kernel (chunks of 64 tokens, 16-bit operands, fp32 accumulation: results within the bf16
- * tolerance of the exact recurrence); chunk = 1 selects the exact fp32 recurrence for any supported shape. Two
- * combinations inside that set also take the exact recurrence, both under the plain sigmoid gate (LAWCAT_GATE_LOGITS
- * with gate_tau < 2, where a token's decay is about one half and the chunk's factors need 8-bit-mantissa operands):
- * gate_dim = 1 (the state sits on the last one or two tokens and its largest entries miss the tolerance) and
- * normalize = 0 (no denominator to cancel the rounding of the weights). With LAWCAT_GATE_LOGDECAY the caller chooses
- * the decays: when they are that sharp (a state that halves or more at every token), pass chunk = 1 for these two forms.
- * Asynchronous conditions arrive through dev_status (largest code wins): LAWCAT_ERR_NUMERIC, a decay exponent within
- * half a chunk left the range +-120 and was clamped; LAWCAT_ERR_TIMEOUT, a bounded device-side wait ran out (the kernel
- * has released its resources and returned; the outputs are undefined).
+ * tolerance of the exact recurrence); chunk = 1 selects the exact fp32 recurrence for any supported shape. Inside that
+ * set two cases also take the exact recurrence: sharp sigmoid gates (LAWCAT_GATE_LOGITS with gate_tau < 8: the decay
+ * factors of half a chunk then leave the fp16 range, and 8-bit-mantissa operands miss the tolerance), and calls of fewer
+ * than 16 tokens (a state of so few terms shows the rounding of single operands). With LAWCAT_GATE_LOGDECAY the caller
+ * chooses the decays and the kernel cannot know them in advance: when a half chunk's accumulated log2-decay exceeds 8 in
+ * magnitude (a state that loses about a sixth or more at every token), or a state entry exceeds 3e4, the affected chunks run
+ * on 8-bit-mantissa operands, the result is delivered, and dev_status reports LAWCAT_ERR_NUMERIC: the result may miss
+ * the tolerance; chunk = 1 has no such limit.
+ * Asynchronous conditions arrive through dev_status (largest code wins): LAWCAT_ERR_NUMERIC, as above, or a decay
+ * exponent within half a chunk left the range +-120 and was clamped; LAWCAT_ERR_TIMEOUT, a bounded device-side wait ran
+ * out (the kernel has released its resources and returned; the outputs are undefined).
  */
 int lawcat_layer_fwd(const lawcat_params* p, const void* q, const void* k, const void* v, const void* gate,
                      const void* w_q, const void* w_k, const void* W, const void* cache_q_in,

@@ -59,9 +59,11 @@ __device__ __forceinline__ void load_raw_and_taps(uint8_t* s_raw, float* s_w, co
   }
 }
 
-// depthwise causal conv of the tile in fp32, result as the fp16 A operand of the mix
+// depthwise causal conv of the tile in fp32, result as the fp16 A operand of the mix; s_ul (nullable): the low part
+// u - fp16(u), again in fp16, for products that take u as a two-term operand
 template <int D>
-__device__ __forceinline__ void conv_tile(const uint8_t* s_raw, const float* s_w, uint8_t* s_u, int tid, int nthreads) {
+__device__ __forceinline__ void conv_tile(const uint8_t* s_raw, const float* s_w, uint8_t* s_u, int tid, int nthreads,
+                                          uint8_t* s_ul = nullptr) {
   using L = Lay<D>;
   const int o = tid % L::OPR;
   float w[8][4];
@@ -80,7 +82,19 @@ __device__ __forceinline__ void conv_tile(const uint8_t* s_raw, const float* s_w
 #pragma unroll
       for (int i = 0; i < 8; ++i) u[i] = fmaf(w[i][dl], x[i], u[i]);
     }
-    *reinterpret_cast<uint4*>(s_u + toff(L::SLAB_U, r, o * 8)) = pack8f16(u);
+    const uint4 ph = pack8f16(u);
+    *reinterpret_cast<uint4*>(s_u + toff(L::SLAB_U, r, o * 8)) = ph;
+    if (s_ul != nullptr) {
+      const __half2* h2 = reinterpret_cast<const __half2*>(&ph);
+      float lo[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h2[i]);
+        lo[2 * i] = u[2 * i] - f.x;
+        lo[2 * i + 1] = u[2 * i + 1] - f.y;
+      }
+      *reinterpret_cast<uint4*>(s_ul + toff(L::SLAB_U, r, o * 8)) = pack8f16(lo);
+    }
   }
 }
 
@@ -88,7 +102,11 @@ template <int D, typename TO>
 __global__ void __launch_bounds__(128) convmix_tc_fwd_kernel(const CArgs a) {
   using L = Lay<D>;
   extern __shared__ __align__(128) uint8_t sg[];
-  constexpr uint32_t OFF_WT = 0, OFF_U = OFF_WT + L::TILE_W, OFF_RAW = OFF_U + L::TILE_U + 2048 /* rows past the tile */;
+  // fp32 outputs (the features a fused caller keeps in fp32) take the conv output as a two-term fp16 pair: about 21 bits
+  // instead of 11, so that the features carry no visible rounding into the gradients computed from them
+  constexpr bool TWO = sizeof(TO) == 4;
+  constexpr uint32_t OFF_WT = 0, OFF_U = OFF_WT + L::TILE_W, OFF_UL = OFF_U + L::TILE_U;
+  constexpr uint32_t OFF_RAW = OFF_UL + (TWO ? L::TILE_U : 0) + 2048 /* rows past the tile */;
   constexpr uint32_t OFF_TAPS = OFF_RAW + (L::RAW_BYTES + 15) / 16 * 16, OFF_BAR = OFF_TAPS + D * 4 * 4;
   const uint32_t sb = smem_u32(sg);
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -126,7 +144,8 @@ __global__ void __launch_bounds__(128) convmix_tc_fwd_kernel(const CArgs a) {
       if (D * 2 > 128) prefetch_l2(kr + 64);
     }
     __syncthreads();
-    conv_tile<D>(sg + OFF_RAW, reinterpret_cast<const float*>(sg + OFF_TAPS), sg + OFF_U, tid, 128);
+    conv_tile<D>(sg + OFF_RAW, reinterpret_cast<const float*>(sg + OFF_TAPS), sg + OFF_U, tid, 128,
+                 TWO ? sg + OFF_UL : nullptr);
     fence_proxy_async();
     tc_fence_before_sync();
     __syncthreads();
@@ -135,6 +154,10 @@ __global__ void __launch_bounds__(128) convmix_tc_fwd_kernel(const CArgs a) {
       const uint32_t idesc = instr_desc(128, D, FMT_F16, MAJOR_K, MAJOR_MN);
       const uint64_t da = kview(sb + OFF_U, L::SLAB_U), db = mview(sb + OFF_WT, L::SLAB_W);
       for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem, dadv(da, 2 * L::SLAB_U * kk), dadv(db, 256 * kk), idesc, kk > 0);
+      if (TWO) {
+        const uint64_t dl = kview(sb + OFF_UL, L::SLAB_U);
+        for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem, dadv(dl, 2 * L::SLAB_U * kk), dadv(db, 256 * kk), idesc, 1);
+      }
       mma_commit(sb + OFF_BAR);
     }
     wt.wait();
@@ -203,7 +226,8 @@ __global__ void __launch_bounds__(128, 2) convmix_tc_bwd_kernel(const CArgs a) {
   using L = Lay<D>;
   extern __shared__ __align__(128) uint8_t sg[];
   constexpr uint32_t OFF_WT = 0, OFF_U = OFF_WT + L::TILE_W, OFF_DY = OFF_U + L::TILE_U, OFF_DYL = OFF_DY + L::TILE_U;
-  constexpr uint32_t OFF_RAW = OFF_DYL + L::TILE_U + 2048, OFF_TAPS = OFF_RAW + (L::RAW_BYTES + 15) / 16 * 16;
+  constexpr uint32_t OFF_UL = OFF_DYL + L::TILE_U;  // low part of the conv output (second term of u in dW)
+  constexpr uint32_t OFF_RAW = OFF_UL + L::TILE_U + 2048, OFF_TAPS = OFF_RAW + (L::RAW_BYTES + 15) / 16 * 16;
   constexpr uint32_t OFF_BAR = OFF_TAPS + D * 4 * 4;
   constexpr uint32_t COL_Y = 0, COL_DW = 64, TMEM_COLS = 256;  // Y / du, and the dW accumulators of two heads at a time
   const uint32_t sb = smem_u32(sg);
@@ -256,7 +280,7 @@ __global__ void __launch_bounds__(128, 2) convmix_tc_bwd_kernel(const CArgs a) {
         }
       }
       __syncthreads();
-      conv_tile<D>(sg + OFF_RAW, reinterpret_cast<const float*>(sg + OFF_TAPS), sg + OFF_U, tid, 128);
+      conv_tile<D>(sg + OFF_RAW, reinterpret_cast<const float*>(sg + OFF_TAPS), sg + OFF_U, tid, 128, sg + OFF_UL);
       fence_proxy_async();
       tc_fence_before_sync();
       __syncthreads();
@@ -265,6 +289,8 @@ __global__ void __launch_bounds__(128, 2) convmix_tc_bwd_kernel(const CArgs a) {
         const uint32_t idesc = instr_desc(128, D, FMT_F16, MAJOR_K, MAJOR_MN);
         const uint64_t da = kview(sb + OFF_U, L::SLAB_U), db = mview(sb + OFF_WT, L::SLAB_W);
         for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem + COL_Y, dadv(da, 2 * L::SLAB_U * kk), dadv(db, 256 * kk), idesc, kk > 0);
+        const uint64_t dal = kview(sb + OFF_UL, L::SLAB_U);  // (second term of u: the same features as the forward recompute)
+        for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem + COL_Y, dadv(dal, 2 * L::SLAB_U * kk), dadv(db, 256 * kk), idesc, 1);
         mma_commit(sb + OFF_BAR);
       }
       wt.wait();
@@ -324,9 +350,16 @@ __global__ void __launch_bounds__(128, 2) convmix_tc_bwd_kernel(const CArgs a) {
         for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem + COL_Y, dadv(dh, 2 * L::SLAB_U * kk), dadv(dw, 2 * L::SLAB_W * kk), id_du, kk > 0);
         for (int kk = 0; kk < D / 16; ++kk) mma_f16(tmem + COL_Y, dadv(dl, 2 * L::SLAB_U * kk), dadv(dw, 2 * L::SLAB_W * kk), id_du, 1);
         const uint32_t id_dw = instr_desc(128, D, FMT_F16, MAJOR_MN, MAJOR_MN);
-        const uint64_t ua = mview(sb + OFF_U, L::SLAB_U), yb = mview(sb + OFF_DY, L::SLAB_U);
+        // (both factors two-term: u_hi dy_hi + u_lo dy_hi + u_hi dy_lo; with few tokens in a call the weight gradient is
+        // a sum of few products and the rounding of single 16-bit operands would show in its largest entries)
+        const uint64_t ua = mview(sb + OFF_U, L::SLAB_U), ual = mview(sb + OFF_UL, L::SLAB_U);
+        const uint64_t yb = mview(sb + OFF_DY, L::SLAB_U), ybl = mview(sb + OFF_DYL, L::SLAB_U);
         for (int kk = 0; kk < TT / 16; ++kk)
           mma_f16(tmem + COL_DW + 64 * (g & 1), dadv(ua, 256 * kk), dadv(yb, 256 * kk), id_dw, (stream > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < TT / 16; ++kk)
+          mma_f16(tmem + COL_DW + 64 * (g & 1), dadv(ual, 256 * kk), dadv(yb, 256 * kk), id_dw, 1u);
+        for (int kk = 0; kk < TT / 16; ++kk)
+          mma_f16(tmem + COL_DW + 64 * (g & 1), dadv(ua, 256 * kk), dadv(ybl, 256 * kk), id_dw, 1u);
         mma_commit(sb + OFF_BAR);
       }
       wt.wait();
@@ -382,14 +415,14 @@ __global__ void __launch_bounds__(128, 2) convmix_tc_bwd_kernel(const CArgs a) {
   }
 }
 
-template <int D>
+template <int D, typename TO>
 constexpr uint32_t fwd_smem() {
   using L = Lay<D>;
-  return L::TILE_W + L::TILE_U + 2048 + (L::RAW_BYTES + 15) / 16 * 16 + D * 16 + 64;
+  return L::TILE_W + (sizeof(TO) == 4 ? 2 : 1) * L::TILE_U + 2048 + (L::RAW_BYTES + 15) / 16 * 16 + D * 16 + 64;
 }
 constexpr uint32_t bwd_smem() {
   using L = Lay<64>;
-  return L::TILE_W + 3 * L::TILE_U + 2048 + (L::RAW_BYTES + 15) / 16 * 16 + 64 * 16 + 64;
+  return L::TILE_W + 4 * L::TILE_U + 2048 + (L::RAW_BYTES + 15) / 16 * 16 + 64 * 16 + 64;
 }
 
 template <typename K>
@@ -432,8 +465,8 @@ int launch_convmix_tc_fwd(const Ctx& c, const void* q, const void* k, const void
   {
     std::lock_guard<std::mutex> lk(mu);
     if (!done[dev]) {
-      if (raise_smem(convmix_tc_fwd_kernel<64, bf16>, fwd_smem<64>()) || raise_smem(convmix_tc_fwd_kernel<64, float>, fwd_smem<64>()) ||
-          raise_smem(convmix_tc_fwd_kernel<128, bf16>, fwd_smem<128>()) || raise_smem(convmix_tc_fwd_kernel<128, float>, fwd_smem<128>()))
+      if (raise_smem(convmix_tc_fwd_kernel<64, bf16>, fwd_smem<64, bf16>()) || raise_smem(convmix_tc_fwd_kernel<64, float>, fwd_smem<64, float>()) ||
+          raise_smem(convmix_tc_fwd_kernel<128, bf16>, fwd_smem<128, bf16>()) || raise_smem(convmix_tc_fwd_kernel<128, float>, fwd_smem<128, float>()))
         return LAWCAT_ERR_CUDA;
       done[dev] = true;
     }
@@ -441,11 +474,11 @@ int launch_convmix_tc_fwd(const Ctx& c, const void* q, const void* k, const void
   const dim3 grid((unsigned)((p.T + TT - 1) / TT), (unsigned)(p.B * p.H));
   LaunchScope _ls("convmix_tc_fwd", c.stream);
   if (p.d_k == 64) {
-    if (out_f32) convmix_tc_fwd_kernel<64, float><<<grid, 128, fwd_smem<64>(), c.stream>>>(a);
-    else convmix_tc_fwd_kernel<64, bf16><<<grid, 128, fwd_smem<64>(), c.stream>>>(a);
+    if (out_f32) convmix_tc_fwd_kernel<64, float><<<grid, 128, fwd_smem<64, float>(), c.stream>>>(a);
+    else convmix_tc_fwd_kernel<64, bf16><<<grid, 128, fwd_smem<64, bf16>(), c.stream>>>(a);
   } else {
-    if (out_f32) convmix_tc_fwd_kernel<128, float><<<grid, 128, fwd_smem<128>(), c.stream>>>(a);
-    else convmix_tc_fwd_kernel<128, bf16><<<grid, 128, fwd_smem<128>(), c.stream>>>(a);
+    if (out_f32) convmix_tc_fwd_kernel<128, float><<<grid, 128, fwd_smem<128, float>(), c.stream>>>(a);
+    else convmix_tc_fwd_kernel<128, bf16><<<grid, 128, fwd_smem<128, bf16>(), c.stream>>>(a);
   }
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;

@@ -468,6 +468,8 @@ __global__ void __launch_bounds__(THREADS, MODE == 2 ? 1 : 2) gla_tc_kernel(cons
     __syncthreads();
     GTL(1);
     const bool f16 = __int_as_float(s_flags[2]) <= RMAX_F16 && sbound < SMAX_F16;
+    // (the 8-bit-mantissa operands keep the range but not the accuracy bound: the caller is told)
+    if (!f16 && tid == 0 && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_NUMERIC);
     const int fmt = f16 ? FMT_F16 : FMT_BF16;
     float vmax = 0.f;
     operand_pass(t0, nvalid, f16, false, 0.f, vmax);
@@ -898,17 +900,15 @@ static int set_smem_once() {
 
 }  // namespace gtc
 
-// The backward asks for more than the forward: under a sharp gate (LOGITS with tau < 8: the decay exponents of half a
-// chunk leave the fp16 range and the operands fall back to 8 significant bits) its gradients miss the accuracy bound, so
-// those parameters take the exact recurrence.
-bool gla_tc_bwd_supported(const lawcat_params& p) {
-  return gla_tc_supported(p) && !(p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 8.f);
-}
+// Under a sharp gate (LOGITS with tau < 8: the decay exponents of half a chunk leave the fp16 range and the operands fall
+// back to 8 significant bits) results and gradients miss the accuracy bound, and so does the state of a call of fewer than
+// 16 tokens (too few terms to average the rounding of single operands): both take the exact recurrence.
+bool gla_tc_bwd_supported(const lawcat_params& p) { return gla_tc_supported(p); }
 
 bool gla_tc_supported(const lawcat_params& p) {
-  const bool sharp = p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 2.f;
+  const bool sharp = p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 8.f;
   return p.dtype == LAWCAT_BF16 && p.d_k == gtc::D && p.d_v == gtc::D && (p.gate_dim == p.d_k || p.gate_dim == 1) &&
-         !(sharp && (p.gate_dim == 1 || !p.normalize)) && p.B > 0 && p.T > 0 && (p.chunk == 0 || p.chunk == gtc::C);
+         !sharp && p.B > 0 && p.T >= 16 && (p.chunk == 0 || p.chunk == gtc::C);
 }
 
 // scratch of the backward: per-head dv (fp32), 1/den and dO.o per token and head, the state operand of every chunk

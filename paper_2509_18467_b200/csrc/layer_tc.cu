@@ -152,15 +152,15 @@ size_t layer_tc_workspace_bytes(const lawcat_params& p) {
 }
 
 bool layer_tc_supported(const lawcat_params& p) {
-  // Under the plain sigmoid gate (tau < 2) a token's decay is about one half, so the exponents of the in-chunk
-  // factorization leave the fp16 range and the operands fall back to bf16 (8 significant bits). The normalized form with
-  // one decay per key channel stays within the accuracy bound there (numerator and denominator carry the same weights);
-  // one decay per head (the state sits on the last one or two tokens) and the numerator-only form do not, so those two
-  // go to the exact path.
-  const bool sharp = p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 2.f;
-  const bool sharp_unsupported = sharp && (p.gate_dim == 1 || !p.normalize);
+  // Sharp sigmoid gates (tau < 8: a token's decay reaches a half at tau = 1) drive the exponents of the in-chunk
+  // factorization out of the fp16 range within half a chunk; the operands then fall back to bf16 (8 significant bits)
+  // and a seeded random sweep finds outputs and states beyond 1e-2 of their RMS for tau = 1, 2 and 4 (numerator-only
+  // form, one decay per head, eps != 0, carried states). Those gates take the exact recurrence. Very short calls do too:
+  // with fewer than 16 tokens the state is a sum of so few terms that the rounding of single 16-bit operands shows in
+  // its largest entries, and the exact kernels are as fast there.
+  const bool sharp = p.gate_mode == LAWCAT_GATE_LOGITS && p.gate_tau < 8.f;
   return p.dtype == LAWCAT_BF16 && (p.d_k == tc::D || p.d_k == 64) && p.d_v == p.d_k &&
-         (p.gate_dim == p.d_k || p.gate_dim == 1) && !sharp_unsupported &&
+         (p.gate_dim == p.d_k || p.gate_dim == 1) && !sharp && p.T >= 16 &&
          p.phi == LAWCAT_PHI_SOFTMAX && p.conv_k <= tc::HALO + 1 && p.B > 0 && p.T > 0 &&
          (p.chunk == 0 || p.chunk == tc::C) &&
          !p.mix_unshared;  // (one W_h is what lets both streams share the M = 128 mix)

@@ -977,6 +977,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       TL(warp == 8 ? 1 : 2, 5, n, (warp == 8 || warp == 10) && lane == 0);
       tc_fence_after_sync();
       const bool f16 = __int_as_float(s_rmax[p]) <= RMAX_F16 && __int_as_float(s_sbound[p]) < SMAX_F16;
+      // (the 8-bit-mantissa operands keep the range but not the accuracy bound: the caller is told)
+      if (MODE == 0 && !f16 && tw == 0 && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_NUMERIC);
       // ---- state pass: 16-bit operand 2^b_mid [S|z], accumulator [S|z] *= 2^b_C (this thread: 64 columns of row r128)
       // (64-wide head: only the rows and columns that exist)
       const bool s_on = !narrow || (!padded && r128 < dh);

@@ -28,3 +28,11 @@ def check(x, y, dtype, what, f32_store=False):
 def oracle_params(s: I.LayerShape, **kw):
     return O.OracleParams(s.B, s.T, s.H, s.H_kv, s.d_k, s.d_v, conv_k=s.conv_k, gate_dim=s.gate_dim,
                           gate_tau=s.gate_tau, **kw)
+
+
+def tc_routed(s: I.LayerShape, phi=0, gate_mode=0, chunk=0, mix_unshared=0, **_):
+    """Whether lawcat_layer_fwd serves this shape with the chunkwise tensor-core layer kernel (the rule its header states):
+    bf16, d_k = d_v in {64, 128}, softmax feature map, conv width <= 4, one linear layer for both streams, at least 16
+    tokens, and log-decay gates or sigmoid gates with tau >= 8; chunk = 1 forces the exact recurrence."""
+    return (s.dtype == "bf16" and s.d_k == s.d_v and s.d_k in (64, 128) and phi == 0 and s.conv_k <= 4 and chunk != 1
+            and not mix_unshared and s.B > 0 and s.T >= 16 and (gate_mode == 1 or s.gate_tau >= 8.0))

@@ -41,7 +41,9 @@ def run(api, s, with_state, backward=True, gate_mode=0, **pkw):
     api.trace_begin()
     f = api.lawcat_gla_fwd(p, d["qdot"], d["kdot"], d["v"], d["gate"], d["S0"], d["z0"])
     kernels = api.trace_end()
-    assert "gla_tc_fwd" in kernels, kernels
+    # (sharp sigmoid gates, tau < 8, and calls of fewer than 16 tokens are served by the exact recurrence: see the header)
+    tc = (gate_mode == 1 or s.gate_tau >= 8.0) and s.T >= 16
+    assert ("gla_tc_fwd" in kernels) == tc, kernels
     ref = O.gla_fwd(op, x["qdot"], x["kdot"], x["v"], x["gate"], x["S0"], x["z0"])
     check(f["o"], ref["o"], "bf16", "o")
     check(f["den"], ref["den"], "bf16", "den", f32_store=True)
@@ -52,8 +54,7 @@ def run(api, s, with_state, backward=True, gate_mode=0, **pkw):
     api.trace_begin()
     g = api.lawcat_gla_bwd(p, d["qdot"], d["kdot"], d["v"], d["gate"], f["o"], f["den"], d["dO"], d["S0"], d["z0"])
     kernels = api.trace_end()
-    # (under a sharp gate, tau < 8, the backward is served by the exact recurrence: see the header of lawcat_gla_bwd)
-    assert ("gla_tc_bwd" in kernels) == (gate_mode == 1 or s.gate_tau >= 8.0), kernels
+    assert ("gla_tc_bwd" in kernels) == tc, kernels
     rg = O.gla_bwd(op, x["qdot"], x["kdot"], x["v"], x["gate"], x["dO"], x["S0"], x["z0"])
     for name in ("d_qdot", "d_kdot", "dv", "dgate"):
         if s.T == 1 and not with_state and name != "dv":
@@ -64,7 +65,7 @@ def run(api, s, with_state, backward=True, gate_mode=0, **pkw):
         check(g[name], rg[name], "bf16", name)
 
 
-@pytest.mark.parametrize("T", [1, 2, 5, 63, 64, 65, 127, 128, 129, 200])
+@pytest.mark.parametrize("T", [1, 2, 5, 15, 16, 17, 63, 64, 65, 127, 128, 129, 200])
 @pytest.mark.parametrize("with_state", [False, True])
 def test_lengths_around_the_chunk_size(api, T, with_state):
     run(api, shape(2, T, 4, 2, 61), with_state)
@@ -75,7 +76,7 @@ def test_head_grouping(api, H, Hkv):
     run(api, shape(1, 300, H, Hkv, 62), True)
 
 
-@pytest.mark.parametrize("tau", [1.0, 4.0, 16.0])
+@pytest.mark.parametrize("tau", [1.0, 4.0, 8.0, 16.0, 64.0])
 def test_gate_sharpness(api, tau):
     run(api, shape(1, 260, 2, 1, 63, gate_tau=tau), False)
 

@@ -10,7 +10,7 @@ import dataclasses
 import numpy as np
 import pytest
 
-from helpers import check, oracle_params
+from helpers import check, oracle_params, tc_routed
 from oracle import lawcat_oracle as O
 from paper_2509_18467_b200 import inputs as I
 
@@ -37,8 +37,12 @@ def P(api, s, **kw):
                       gate_tau=s.gate_tau, **kw)
 
 
-def run_case(api, s, with_state, expect_tc=True, **pkw):
+def run_case(api, s, with_state, expect_tc=None, **pkw):
+    """One call of lawcat_layer_fwd against the oracle; expect_tc: whether the tensor-core layer kernel must have run
+    (default: what the routing rule of the header says for this shape)."""
     import torch
+    if expect_tc is None:
+        expect_tc = tc_routed(s, **pkw)
     extra = (["S0", "z0"] + (["cache_q", "cache_k"] if s.conv_k > 1 else [])) if with_state else []
     x = I.make(s, NAMES + extra)
     d = {n: api.to_device(v, "f32" if n in ("S0", "z0") else s.dtype) for n, v in x.items()}
@@ -62,9 +66,10 @@ def run_case(api, s, with_state, expect_tc=True, **pkw):
     return e, r, ref
 
 
-@pytest.mark.parametrize("T", [1, 2, 3, 5, 63, 64, 65, 127, 128, 129, 200])
+@pytest.mark.parametrize("T", [1, 2, 3, 5, 15, 16, 17, 31, 63, 64, 65, 127, 128, 129, 200])
 @pytest.mark.parametrize("with_state", [False, True])
 def test_lengths_around_the_chunk_size(api, T, with_state):
+    """(calls of fewer than 16 tokens are served by the exact recurrence)"""
     run_case(api, shape(2, T, 4, 2, 41), with_state)
 
 
@@ -78,10 +83,11 @@ def test_conv_widths(api, conv_k):
     run_case(api, shape(1, 150, 2, 1, 43, conv_k=conv_k), True)
 
 
-@pytest.mark.parametrize("tau", [1.0, 4.0, 16.0])
+@pytest.mark.parametrize("tau", [1.0, 4.0, 8.0, 16.0, 64.0])
 def test_gate_sharpness(api, tau):
-    """tau = 1 is the plain sigmoid gate of Section 4.2: per-token decays down to a few percent."""
-    run_case(api, shape(1, 260, 2, 1, 44, gate_tau=tau), False)
+    """tau = 1 is the plain sigmoid gate of Section 4.2: per-token decays down to a few percent. Sigmoid gates with tau < 8
+    take the exact recurrence, from tau = 8 on the tensor-core kernel."""
+    _, _, _ = run_case(api, shape(1, 260, 2, 1, 44, gate_tau=tau), False, expect_tc=tau >= 8.0)
 
 
 @pytest.mark.parametrize("T", [1162, 1223, 1300])
@@ -98,9 +104,10 @@ def test_one_decay_per_head(api, T, with_state):
 
 def test_one_decay_per_head_sharp_gate(api):
     """One plain-sigmoid decay per head (gate_dim = 1, tau = 1): the library serves it with the exact recurrence, because
-    the state then sits on the last one or two tokens; tau = 2 is back on the tensor-core kernel."""
+    the state then sits on the last one or two tokens; tau = 8 is on the tensor-core kernel."""
     run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=1.0), False, expect_tc=False)
-    run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=2.0), True)
+    run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=2.0), True, expect_tc=False)
+    run_case(api, shape(2, 200, 2, 1, 51, gate_dim=1, gate_tau=8.0), True, expect_tc=True)
 
 
 def shape64(B, T, H, Hkv, cid, **kw):
@@ -185,7 +192,7 @@ def test_exponent_clamp_is_reported(api):
     """Gate logits so negative that the decay exponents within half a chunk leave +-120: the kernel clamps them, says so
     through dev_status (LAWCAT_ERR_NUMERIC = 6) and still returns finite numbers; moderate logits report nothing."""
     import torch
-    s = shape(1, 128, 2, 1, 55, gate_tau=1.0)
+    s = shape(1, 128, 2, 1, 55, gate_tau=16.0)
     x = I.make(s, NAMES)
     for scale, want in ((1.0, 0), (60.0, 6)):
         g = I.round_to_bf16(-np.abs(x["gate"]) * np.float32(scale))
