@@ -442,6 +442,7 @@ static size_t host_arena_layout(const lawcat_params* p, size_t off[11]) {
 
 // copy streams and events of the host path, one set per device, created on first use and kept
 struct HostPipe {
+  std::mutex mu;  // held while a call enqueues: the events are shared by every caller on the device
   cudaStream_t in = nullptr, out = nullptr;
   std::vector<cudaEvent_t> ev;
   cudaEvent_t event(size_t i) {
@@ -485,6 +486,7 @@ int lawcat_layer_fwd_host(const lawcat_params* p, const void* h_q, const void* h
   if (p->B * p->T == 0) return LAWCAT_OK;
   HostPipe* hp = host_pipe();
   if (!hp) return LAWCAT_ERR_CUDA;
+  std::lock_guard<std::mutex> hold(hp->mu);
   char* a = (char*)arena;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t es = p->dtype == LAWCAT_F32 ? 4 : 2;
