@@ -117,11 +117,18 @@ struct TcPlan {
 // segment (a thread block spends about three chunk times on its set-up and on filling its pipeline). Pieces per segment
 // in the state-only pre-pass: its thread blocks are independent, so cutting the segments finer lets them fill the SMs in
 // whole waves; the split with the fewest chunks per SM wins (a small charge per extra piece).
+// Two 64-wide heads share a thread block when they can: an even number of query heads per key/value head (the two heads
+// of a block read the same k and v) and one decay per key channel.
+static bool layer_tc_paired(const lawcat_params& p) {
+  return p.d_k == 64 && p.gate_dim == p.d_k && (p.H / p.H_kv) % 2 == 0;
+}
+
 static TcPlan layer_tc_plan(const lawcat_params& p) {
   constexpr int MIN_SEG_CHUNKS = 4;
   const int sms = sm_count();
   const int chunks = (p.T + tc::C - 1) / tc::C;
-  int n = sms / (p.B * p.H);
+  const int seqs = p.B * (layer_tc_paired(p) ? p.H / 2 : p.H);  // sequences of thread blocks
+  int n = sms / seqs;
   if (n > chunks / MIN_SEG_CHUNKS) n = chunks / MIN_SEG_CHUNKS;
   if (n < 1) n = 1;
   TcPlan pl;
@@ -131,7 +138,7 @@ static TcPlan layer_tc_plan(const lawcat_params& p) {
   const int cps = pl.seg_len / tc::C;
   int best = 1, best_cost = 1 << 30;
   for (int ns = 1; ns <= 8 && ns * 4 <= cps; ++ns) {
-    const int ctas = p.B * p.H * (pl.nseg - 1) * ns;
+    const int ctas = seqs * (pl.nseg - 1) * ns;
     const int cost = ((ctas + sms - 1) / sms) * ((cps + ns - 1) / ns + 2);
     if (cost < best_cost) { best_cost = cost; best = ns; }
   }
@@ -173,11 +180,14 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   const lawcat_params& p = *c.p;
   CUtensorMap tq, tk, tv, tg;
   const int dh = p.d_k;
-  if (!make_map(&tq, q, p.H, p.T, p.B, C, dh) || !make_map(&tk, k, p.H_kv, p.T, p.B, C, dh) ||
+  const bool paired = layer_tc_paired(p);
+  // (pair: q, gate and o of two neighbouring heads are 128 contiguous channels and are mapped as one head of 128)
+  const int Hmap = paired ? p.H / 2 : p.H, dmap = paired ? 128 : dh;
+  if (!make_map(&tq, q, Hmap, p.T, p.B, C, dmap) || !make_map(&tk, k, p.H_kv, p.T, p.B, C, dh) ||
       !make_map(&tv, v, p.H_kv, p.T, p.B, C, dh))
     return LAWCAT_ERR_CUDA;
   if (p.gate_dim == 1) tg = tq;  // (never used: one logit per token and head is read without a tensor map)
-  else if (!make_map(&tg, gate, p.H, p.T, p.B, C, dh)) return LAWCAT_ERR_CUDA;
+  else if (!make_map(&tg, gate, Hmap, p.T, p.B, C, dmap)) return LAWCAT_ERR_CUDA;
   TcArgs a{};
   a.q = (const bf16*)q; a.k = (const bf16*)k; a.o = (bf16*)o;
   a.gate = (const bf16*)gate; a.gate_dim = p.gate_dim; a.dh = dh;
@@ -192,9 +202,8 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   const int nseg = pl.nseg;
   a.nseg = nseg;
   a.seg_len = pl.seg_len;
-  const bool narrow = dh == 64;
-  auto* const k_layer = narrow ? layer_tc_kernel<0, true> : layer_tc_kernel<0, false>;
-  auto* const k_state = narrow ? layer_tc_kernel<1, true> : layer_tc_kernel<1, false>;
+  auto* const k_layer = paired ? layer_tc_kernel<0, 2> : dh == 64 ? layer_tc_kernel<0, 1> : layer_tc_kernel<0, 0>;
+  auto* const k_state = paired ? layer_tc_kernel<1, 2> : dh == 64 ? layer_tc_kernel<1, 1> : layer_tc_kernel<1, 0>;
   {
     // the kernels' shared-memory limit is raised once per device
     static std::mutex mu;
@@ -203,20 +212,23 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LAWCAT_ERR_CUDA;
     std::lock_guard<std::mutex> lk(mu);
     if (!done[dev]) {
-      if (cudaFuncSetAttribute(layer_tc_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
-          cudaFuncSetAttribute(layer_tc_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
-          cudaFuncSetAttribute(layer_tc_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
-          cudaFuncSetAttribute(layer_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess)
+      if (cudaFuncSetAttribute(layer_tc_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess ||
+          cudaFuncSetAttribute(layer_tc_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_ALLOC) != cudaSuccess)
         return LAWCAT_ERR_CUDA;
       done[dev] = true;
     }
   }
-  const int BH = p.B * p.H;
+  const int BH = p.B * p.H;                       // real heads: the states in the workspace are per real head
+  const int NB = paired ? BH / 2 : BH;            // sequences of thread blocks
   if (nseg == 1) {
     a.S0 = S0; a.z0 = z0; a.S_T = S_T; a.z_T = z_T; a.dtot = nullptr;
     a.grid_nseg = 1; a.nsub = 1; a.seg_in = 0; a.seg_out = 0;
     LaunchScope _ls("layer_tc", c.stream);
-    k_layer<<<BH, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
+    k_layer<<<NB, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, a);
     LAWCAT_CHECK_LAUNCH();
     return LAWCAT_OK;
   }
@@ -235,7 +247,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
     b1.S0 = nullptr; b1.z0 = nullptr; b1.S_T = loc_S; b1.z_T = loc_z; b1.dtot = dtot;
     b1.grid_nseg = nseg - 1; b1.nsub = nsub; b1.seg_in = 1; b1.seg_out = 1;
     LaunchScope _ls("layer_tc_state", c.stream);
-    k_state<<<BH * (nseg - 1) * nsub, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, b1);
+    k_state<<<NB * (nseg - 1) * nsub, THREADS, SMEM_ALLOC, c.stream>>>(tq, tk, tv, tg, b1);
     LAWCAT_CHECK_LAUNCH();
   }
   {
@@ -259,7 +271,7 @@ int launch_layer_tc(const Ctx& c, const void* q, const void* k, const void* v, c
   LaunchScope _ls("layer_tc", c.stream);
   {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(BH * nseg));
+    cfg.gridDim = dim3((unsigned)(NB * nseg));
     cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = SMEM_ALLOC;
     cfg.stream = c.stream;

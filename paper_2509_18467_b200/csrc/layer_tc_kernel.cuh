@@ -76,6 +76,9 @@ constexpr uint32_t OFF_SBF = OFF_W + 32768;       // 2^b_mid * [S | z], 16 bit, 
                                                   // unswizzled 8x8 core matrices: block of 8 columns nb at nb * 2048,
                                                   // key channel c at (c / 8) * 128 + (c % 8) * 16 inside a block; the
                                                   // blocks of S are followed by two blocks whose first column is z
+constexpr uint32_t OFF_PH2 = OFF_SBF + 20480;     // (two 64-wide heads per block: the state operand has 80 columns = 20 KB;
+                                                  // the second head's masked scores [64 x 128 B] use the rest, and the 8 KB an
+                                                  // M = 128 product reads behind them stay inside this tile)
 constexpr uint32_t OFF_AU = OFF_SBF + 36864;      // raw q|k tile, then conv output in place: A of MMA 1, 2 slabs
 constexpr uint32_t OFF_QK = OFF_AU + 32768;       // qs (rows 0-63) | ks (rows 64-127), 16 bit, K-major, 2 slabs
 constexpr uint32_t OFF_X = OFF_QK + 32768;        // exponents x fp32 [64 x 128], XOR-swizzled 16-byte chunks
@@ -283,9 +286,9 @@ __device__ __forceinline__ bool wait_set_or_abort(uint32_t bar0, uint32_t mask, 
 
 // MODE 0: the layer forward. MODE 1: state only (no query stream, no output): the end state of a segment that starts
 // from the given state, used to hand the state across segments of one sequence.
-// NARROW: heads of width 64 (a.dh == 64) instead of 128; a compile-time switch, so that the 128-wide kernel carries none
-// of its tests.
-template <int MODE, bool NARROW>
+// WIDTH: 0 = heads of 128 channels; 1 = one head of 64 channels per block (padded to 128); 2 = two 64-wide heads of one
+// key/value group per block. A compile-time switch, so that the 128-wide kernel carries none of the others' tests.
+template <int MODE, int WIDTH>
 __global__ void __launch_bounds__(THREADS, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g, const TcArgs a) {
@@ -306,19 +309,33 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  constexpr int dh = NARROW ? 64 : 128, nslab = dh >> 6;  // tensor width and its 64-channel slabs (1 or 2)
-  constexpr bool narrow = NARROW;  // 64-wide head: everything that belongs to the upper 64 channels is left out
+  // WIDTH 0: heads of 128 channels. WIDTH 1 (narrow): one head of 64 channels, run as a 128-wide one whose upper 64
+  // channels are zero. WIDTH 2 (pair): two 64-wide heads of one key/value group side by side -- channels 0-63 belong to head
+  // 2 h, channels 64-127 to head 2 h + 1; q, gate and o of the two are contiguous in memory and are addressed as one head
+  // of 128 channels, the shared k is loaded into both halves, W is block-diagonal, and everything that contracts over the
+  // channels (scores, read-out) is issued per half into accumulators of its own.
+  constexpr bool narrow = WIDTH == 1, pair = WIDTH == 2, wide = WIDTH == 0;
+  constexpr int dh = narrow ? 64 : 128, nslab = dh >> 6;  // width of the q / gate / o tiles as addressed, and their slabs
+  constexpr int hd = wide ? 128 : 64, vslab = hd >> 6;    // width of a real head: of k and v as stored, of the state's value side
+  // tensor memory columns (the pair keeps two read-out and two score accumulators where the state needs half the columns)
+  constexpr uint32_t cS = COL_S, cSZ = pair ? 192u : COL_SZ, cO = pair ? 208u : COL_O, cO2 = 288u;
+  constexpr uint32_t cP = pair ? 368u : COL_P, cP2 = 432u, cMAIL = pair ? 496u : COL_MAIL;
   const int sub = blockIdx.x % a.nsub;
   const int seg = (blockIdx.x / a.nsub) % a.grid_nseg;
   const int bh = blockIdx.x / (a.nsub * a.grid_nseg);
-  const int h = bh % a.H, b = bh / a.H;
-  const int G = a.H / a.Hkv, j = h / G;
+  const int Hn = pair ? a.H / 2 : a.H;   // heads as addressed (units of dh channels)
+  const int h = bh % Hn, b = bh / Hn;
+  const int h0 = pair ? 2 * h : h;       // first real head of this block
+  const int G = a.H / a.Hkv, j = h0 / G;
   const int cps = a.seg_len / C;  // chunks per segment; piece `sub` covers chunks [sub cps / nsub, (sub + 1) cps / nsub)
   const int t_begin = min(a.T, seg * a.seg_len + (sub * cps / a.nsub) * C);
   const int t_end = min(a.T, seg * a.seg_len + ((sub + 1) * cps / a.nsub) * C);
   const int nchunks = max(0, (t_end - t_begin + C - 1) / C);
-  const size_t seg_idx = ((size_t)bh * a.nseg + seg) * a.nsub + sub;
-  const size_t in_idx = a.seg_in ? seg_idx : (size_t)bh, out_idx = a.seg_out ? seg_idx : (size_t)bh;
+  // index of the state of the real head that owns state row c (rows 64-127 of a pair: the second head)
+  auto state_idx = [&](int c, int per_segment) -> size_t {
+    const size_t hr = (size_t)b * a.H + h0 + (pair ? (c >> 6) : 0);
+    return per_segment ? (hr * a.nseg + seg) * a.nsub + sub : hr;
+  };
 
   if ((sb & 1023u) != 0) {  // the swizzled tiles need a 1024-byte aligned base
     if (tid == 0 && a.dev_status) atomicMax(a.dev_status, (int)LAWCAT_ERR_CUDA);
@@ -356,13 +373,22 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tmem_relinquish();
   }
   // W_h^T into its K-major slabs as fp16: row e holds W[h][c][e] over c
+  // (pair: block-diagonal, W of head 2 h in the upper left 64 x 64 block, W of head 2 h + 1 in the lower right)
   {
-    const bf16* Wh = a.W + (size_t)h * dh * dh;
+    const bf16* Wh = a.W + (size_t)h0 * hd * hd;
 #pragma unroll 1
     for (int idx = tid; idx < 16 * D; idx += THREADS) {
       const int e = idx & (D - 1), oc = idx >> 7;
       uint32_t w[4] = {0u, 0u, 0u, 0u};
-      if (e < dh && oc * 8 < dh) {
+      if (pair) {
+        if ((e >> 6) == (oc >> 3)) {
+          const bf16* Wp = Wh + (size_t)(oc >> 3) * hd * hd;
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            w[i] = pack_f16(__bfloat162float(Wp[(size_t)((oc & 7) * 8 + 2 * i) * hd + (e & 63)]),
+                            __bfloat162float(Wp[(size_t)((oc & 7) * 8 + 2 * i + 1) * hd + (e & 63)]));
+        }
+      } else if (e < dh && oc * 8 < dh) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
           w[i] = pack_f16(__bfloat162float(Wh[(size_t)(oc * 8 + 2 * i) * dh + e]),
@@ -378,21 +404,24 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     for (int i = tid; i < 8192 / 16; i += THREADS) reinterpret_cast<uint4*>(sg + OFF_KH + 8192)[i] = make_uint4(0u, 0u, 0u, 0u);
   // constant "ones" operand and the zeroed column blocks of the state operand that carry z (unswizzled 8x8 core matrices)
   for (int i = tid; i < 2048 / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_ONES)[i] = 0u;
-  for (int i = tid; i < 4096 / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_SBF + (dh >> 3) * 2048)[i] = 0u;
+  for (int i = tid; i < 4096 / 4; i += THREADS) reinterpret_cast<uint32_t*>(sg + OFF_SBF + (hd >> 3) * 2048)[i] = 0u;
   // raw rows in front of the segment: earlier tokens, or the conv cache, or zeros (Section 4.1)
   if (tid < 96) {
     const int st = tid / 48, r = (tid % 48) / 16, oc = tid % 16;
-    const int NH = st ? a.Hkv : a.H, head = st ? j : h;
+    // row stride and offset of this block's channels in the stream as stored (pair: the key stream's 64 channels serve
+    // both halves of the tile)
+    const size_t rstride = st ? (size_t)a.Hkv * hd : (size_t)Hn * dh;
+    const size_t coff = (st ? (size_t)j * hd : (size_t)h * dh) + (size_t)((st && pair) ? (oc & 7) : oc) * 8;
     const int t = t_begin - HALO + r;  // token of halo row r
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (oc * 8 >= dh) {
       // padded channels: zero
     } else if (t >= 0) {
-      v = *reinterpret_cast<const uint4*>((st ? a.k : a.q) + ((size_t)b * a.T + t) * NH * dh + head * dh + oc * 8);
+      v = *reinterpret_cast<const uint4*>((st ? a.k : a.q) + ((size_t)b * a.T + t) * rstride + coff);
     } else {
       const bf16* cache = st ? a.cache_k : a.cache_q;
       const int ci = t + (a.K - 1);  // the cache holds tokens -(K-1) .. -1, oldest first
-      if (cache && ci >= 0) v = *reinterpret_cast<const uint4*>(cache + ((size_t)b * (a.K - 1) + ci) * NH * dh + head * dh + oc * 8);
+      if (cache && ci >= 0) v = *reinterpret_cast<const uint4*>(cache + ((size_t)b * (a.K - 1) + ci) * rstride + coff);
     }
     *reinterpret_cast<uint4*>(sg + OFF_HALO + ((st * 3 + r) * 16 + oc) * 16) = v;
   }
@@ -400,18 +429,20 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // conv caches after the last token (Section 4.1: the last K - 1 raw rows of [cache_in, x]): they depend on the raw
   // inputs alone, so the block of a head's last segment writes them here (the key stream by the first head of a group)
   if (MODE == 0 && seg == a.nseg - 1 && sub == 0 && a.K > 1 && tid < PREP_THREADS) {
-    const int per = (a.K - 1) * (dh / 8);  // 16-byte units per stream
+    const int per = (a.K - 1) * (dh / 8);  // 16-byte units per stream (the key stream of a pair uses the first hd / 8 per row)
     for (int idx = tid; idx < 2 * per; idx += PREP_THREADS) {
       const int st = idx / per, r = (idx % per) / (dh / 8), oc = idx % (dh / 8);
       bf16* dst = st ? a.cache_k_out : a.cache_q_out;
-      if (dst == nullptr || (st == 1 && h % G != 0)) continue;
-      const int NH = st ? a.Hkv : a.H, head = st ? j : h, tok = a.T - (a.K - 1) + r;
+      if (dst == nullptr || (st == 1 && (h0 % G != 0 || oc * 8 >= hd))) continue;
+      const size_t rstride = st ? (size_t)a.Hkv * hd : (size_t)Hn * dh;
+      const size_t coff = (st ? (size_t)j * hd : (size_t)h * dh) + (size_t)oc * 8;
+      const int tok = a.T - (a.K - 1) + r;
       const bf16* x = st ? a.k : a.q;
       const bf16* cin = st ? a.cache_k : a.cache_q;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (tok >= 0) v = *reinterpret_cast<const uint4*>(x + (((size_t)b * a.T + tok) * NH + head) * dh + oc * 8);
-      else if (cin != nullptr) v = *reinterpret_cast<const uint4*>(cin + (((size_t)b * (a.K - 1) + tok + a.K - 1) * NH + head) * dh + oc * 8);
-      *reinterpret_cast<uint4*>(dst + (((size_t)b * (a.K - 1) + r) * NH + head) * dh + oc * 8) = v;
+      if (tok >= 0) v = *reinterpret_cast<const uint4*>(x + ((size_t)b * a.T + tok) * rstride + coff);
+      else if (cin != nullptr) v = *reinterpret_cast<const uint4*>(cin + ((size_t)b * (a.K - 1) + tok + a.K - 1) * rstride + coff);
+      *reinterpret_cast<uint4*>(dst + ((size_t)b * (a.K - 1) + r) * rstride + coff) = v;
     }
   }
   if (tid < C) *reinterpret_cast<__half*>(sg + OFF_ONES + (tid >> 3) * 128 + (tid & 7) * 16) = __float2half(1.f);
@@ -427,23 +458,26 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // initial state into tensor memory: row thread (c, half) owns 64 columns of row c of [S | z]
   if (warp >= ROW_WARP0 && warp < ROW_WARP0 + 8) {
+    // (pair: the state is [128 key channels x 64 value columns], the thread owns 32 columns; rows 64-127 are the second head)
     const int tw = tid - ROW_WARP0 * 32, c = tw & 127, chh = tw >> 7;
     const bool have = a.S0 != nullptr && (a.seg_in || seg == 0);
+    const size_t in_idx = state_idx(c, a.seg_in);
+    const int cr = c & (hd - 1);  // row inside the real head's state
     float s[32], mx = 0.f;
 #pragma unroll 1
-    for (int b2 = 0; b2 < 2; ++b2) {
-      const int blk = chh * 2 + b2;
+    for (int b2 = 0; b2 < (pair ? 1 : 2); ++b2) {
+      const int blk = pair ? chh : chh * 2 + b2;
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        s[i] = (have && c < dh && blk * 32 < dh) ? a.S0[(in_idx * dh + c) * dh + blk * 32 + i] : 0.f;
+        s[i] = (have && c < dh && blk * 32 < hd) ? a.S0[(in_idx * hd + cr) * hd + blk * 32 + i] : 0.f;
         mx = fmaxf(mx, fabsf(s[i]));
       }
-      tmem_st32(lane_base + COL_S + blk * 32, s);
+      tmem_st32(lane_base + cS + blk * 32, s);
     }
     if (chh == 1) {
       const bool havez = a.z0 != nullptr && (a.seg_in || seg == 0);
-      const float z0v = (havez && c < dh) ? a.z0[in_idx * dh + c] : 0.f;
-      tmem_st1(lane_base + COL_SZ, z0v);
+      const float z0v = (havez && c < dh) ? a.z0[in_idx * hd + cr] : 0.f;
+      tmem_st1(lane_base + cSZ, z0v);
       mx = fmaxf(mx, fabsf(z0v));
     }
     tmem_wait_st();
@@ -479,7 +513,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll 1
         for (int s = 0; s < nslab; ++s) {
           if (MODE == 0) tma_load_4d(sb + OFF_AU + s * 16384, &tm_q, bar(B_RAW_FULL), s * 64, h, t0, b);
-          tma_load_4d(sb + OFF_AU + s * 16384 + 8192, &tm_k, bar(B_RAW_FULL), s * 64, j, t0, b);
+          // (pair: the same 64 key channels into both halves of the tile)
+          tma_load_4d(sb + OFF_AU + s * 16384 + 8192, &tm_k, bar(B_RAW_FULL), pair ? 0 : s * 64, j, t0, b);
         }
         ar_raw = n;
         if (a.gate_dim != 1) {
@@ -490,9 +525,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           ar_g = n;
         }
         if (n > 0) WAIT(MODE == 0 ? B_MMA3 : B_MMA2, pp);  // the last MMA that reads v
-        mbar_arrive_expect_tx(bar(B_V_FULL), 8192u * (uint32_t)nslab);
+        mbar_arrive_expect_tx(bar(B_V_FULL), 8192u * (uint32_t)vslab);
         tma_load_4d(sb + OFF_V, &tm_v, bar(B_V_FULL), 0, j, t0, b);
-        if (nslab == 2) tma_load_4d(sb + OFF_V + 8192, &tm_v, bar(B_V_FULL), 64, j, t0, b);
+        if (vslab == 2) tma_load_4d(sb + OFF_V + 8192, &tm_v, bar(B_V_FULL), 64, j, t0, b);
         ar_v = n;
       }
       if (*s_abort) {
@@ -518,13 +553,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const uint64_t dsc_v = smem_desc(sb + OFF_V, 8192, 1024, LAYOUT_SW128);
       const uint64_t dsc_one = smem_desc(sb + OFF_ONES, 128, 1024, LAYOUT_NONE);
       const uint64_t dsc_p = smem_desc(sb + OFF_PH, 16, 1024, LAYOUT_SW128);
+      // (pair: the masked scores of the second head; see OFF_PH2)
+      const uint64_t dsc_p2 = smem_desc(sb + OFF_PH2, 16, 1024, LAYOUT_SW128);
       // only the 14-bit start-address field (bits 0-13) moves, and it cannot carry: a 32-bit add on the low word
       auto adv = [](uint64_t d, uint32_t off16) -> uint64_t {
         return (d & 0xFFFFFFFF00000000ull) | (uint64_t)((uint32_t)d + off16);
       };
       auto kstep = [](int k) -> uint32_t { return (uint32_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2); };
       // (a 64-wide head: 4 instead of 8 K steps over the channels, 64 instead of 128 output columns)
-      const int ksteps = narrow ? 4 : 8, NW = narrow ? 64 : 128;
+      const int ksteps = narrow ? 4 : 8, NW = narrow ? 64 : 128;  // (the mix: channels contracted, output columns)
+      constexpr int NV = hd;  // value columns of the state and of the read-out
       auto issue_mma1 = [&]() {
         const uint32_t ID = instr_desc(128, NW, FMT_F16, MAJOR_K, MAJOR_K);
 #pragma unroll
@@ -548,10 +586,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (MODE == 0 && lane == 0) {
           // the scores first: their mask pass is the longest chain behind this hand-over
           tc_fence_after_sync();
+          // (pair: channels 0-63 give the first head's scores, channels 64-127 the second head's, in accumulators of their own)
           const uint32_t ID_P = instr_desc(128, 64, fmt, MAJOR_K, MAJOR_K);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            if (k < ksteps) mma_f16(tmem + COL_P, adv(dsc_qk, kstep(k)), adv(dsc_ks, kstep(k)), ID_P, k > 0);
+            if (k < ksteps)
+              mma_f16(tmem + ((pair && k >= 4) ? cP2 : cP), adv(dsc_qk, kstep(k)), adv(dsc_ks, kstep(k)), ID_P,
+                      pair ? (k & 3) > 0 : k > 0);
           mma_commit(bar(B_P));
         }
         TL(0, 1, n, lane == 0);
@@ -568,18 +609,21 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           tc_fence_after_sync();
           if (MODE == 0) {
             // read-out O' | denominator = qs [2^b_mid S | 2^b_mid z] in one product per K step
-            const uint32_t ID_O = instr_desc(128, NW + 16, fmt, MAJOR_K, MAJOR_MN);
+            // (pair: the first head's read-out contracts channels 0-63 with state rows 0-63, the second head's the rest)
+            const uint32_t ID_O = instr_desc(128, NV + 16, fmt, MAJOR_K, MAJOR_MN);
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-              if (k < ksteps) mma_f16(tmem + COL_O, adv(dsc_qk, kstep(k)), adv(dsc_s, k * (256 >> 4)), ID_O, k > 0);
+              if (k < ksteps)
+                mma_f16(tmem + ((pair && k >= 4) ? cO2 : cO), adv(dsc_qk, kstep(k)), adv(dsc_s, k * (256 >> 4)), ID_O,
+                        pair ? (k & 3) > 0 : k > 0);
           }
-          const uint32_t ID_S = instr_desc(128, NW, FMT_F16, MAJOR_MN, MAJOR_MN);
+          const uint32_t ID_S = instr_desc(128, NV, FMT_F16, MAJOR_MN, MAJOR_MN);
           constexpr uint32_t ID_SZ = instr_desc(128, 16, FMT_F16, MAJOR_MN, MAJOR_MN);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const uint64_t ad = adv(dsc_kh, k * (2048 >> 4));
-            mma_f16(tmem + COL_S, ad, adv(dsc_v, k * (2048 >> 4)), ID_S, 1);
-            mma_f16(tmem + COL_SZ, ad, adv(dsc_one, k * (256 >> 4)), ID_SZ, 1);
+            mma_f16(tmem + cS, ad, adv(dsc_v, k * (2048 >> 4)), ID_S, 1);
+            mma_f16(tmem + cSZ, ad, adv(dsc_one, k * (256 >> 4)), ID_SZ, 1);
           }
           mma_commit(bar(B_MMA2));
         }
@@ -590,10 +634,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (lane == 0) {
             // O' += P v  (the scores' part of the denominator is summed by the mask pass)
             tc_fence_after_sync();
-            const uint32_t ID_O = instr_desc(128, NW, FMT_F16, MAJOR_K, MAJOR_MN);
+            const uint32_t ID_O = instr_desc(128, NV, FMT_F16, MAJOR_K, MAJOR_MN);
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              mma_f16(tmem + COL_O, adv(dsc_p, k * 2), adv(dsc_v, k * (2048 >> 4)), ID_O, 1);
+              mma_f16(tmem + cO, adv(dsc_p, k * 2), adv(dsc_v, k * (2048 >> 4)), ID_O, 1);
+            if (pair) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                mma_f16(tmem + cO2, adv(dsc_p2, k * 2), adv(dsc_v, k * (2048 >> 4)), ID_O, 1);
+            }
             mma_commit(bar(B_MMA3));
           }
           TL(0, 5, n, lane == 0);
@@ -608,12 +657,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint64_t cw[4][4];  // [channel pair][tap], packed pairs of fp32
     {
       const bf16* w = cv_stream ? a.w_k : a.w_q;
-      const int head = cv_stream ? j : h;
+      // first channel of this thread's octet among the stream's taps (pair: both halves of the key tile are the same 64 channels)
+      const size_t ch0 = cv_stream ? (size_t)j * hd + (size_t)(pair ? (cv_oct & 7) : cv_oct) * 8 : (size_t)h * dh + cv_oct * 8;
 #pragma unroll
       for (int cp = 0; cp < 4; ++cp)
 #pragma unroll
         for (int dl = 0; dl < 4; ++dl) {
-          const size_t i0 = ((size_t)head * dh + cv_oct * 8 + 2 * cp) * a.K + dl;
+          const size_t i0 = (ch0 + 2 * cp) * a.K + dl;
           cw[cp][dl] = (dl < a.K && cv_oct * 8 < dh) ? f2_pack(__bfloat162float(w[i0]), __bfloat162float(w[i0 + a.K]))
                                                     : f2_pack(0.f, 0.f);
         }
@@ -637,24 +687,26 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int ot0 = t_begin + m * C;
       const int onvalid = min(C, t_end - ot0);
       tc_fence_after_sync();
-      float den = tmem_ld1(lane_base + COL_O + dh);
-      const float den_p0 = tmem_ld1(lane_base + COL_MAIL + 8 + 2 * (m & 1));
-      const float den_p1 = tmem_ld1(lane_base + COL_MAIL + 8 + 2 * (m & 1) + 1);
+      // (pair: column half = head; each head has its own read-out accumulator, denominator parts and dropped normalizer)
+      const uint32_t ocol = pair ? (och ? cO2 : cO) : cO + och * 64;
+      float den = tmem_ld1(lane_base + (pair ? ocol + hd : cO + dh));
+      const float den_p0 = tmem_ld1(lane_base + cMAIL + 8 + 2 * (m & 1) + (pair ? och : 0));
+      const float den_p1 = pair ? 0.f : tmem_ld1(lane_base + cMAIL + 8 + 2 * (m & 1) + 1);
       // The query features went in as exp(y - max), without their softmax normalizer: it cancels in Eq. 8 except next to
       // eps, which therefore gets scaled by it; without normalization the numerator is divided by it.
       float qs = 0.f;
       if (a.eps != 0.f || !a.normalize) {
-        qs = tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1));
-        if (!narrow) qs += tmem_ld1(lane_base + COL_MAIL + 4 * (m & 1) + 1);
+        qs = tmem_ld1(lane_base + cMAIL + 4 * (m & 1) + (pair ? och : 0));
+        if (wide) qs += tmem_ld1(lane_base + cMAIL + 4 * (m & 1) + 1);
       }
       tmem_wait_ld();
       den += den_p0 + den_p1;
       const float inv = 1.f / (a.normalize ? fmaf(a.eps, qs, den) : qs);
-      bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * a.H + h) * dh + och * 64;
+      bf16* orow = a.o + (((size_t)b * a.T + ot0 + orow_i) * Hn + h) * dh + och * 64;
       float y[32];
 #pragma unroll 1
       for (int b2 = 0; b2 < 2; ++b2) {
-        tmem_ld32(lane_base + COL_O + och * 64 + b2 * 32, y);
+        tmem_ld32(lane_base + ocol + b2 * 32, y);
         tmem_wait_ld();
         if (b2 == 1) {  // O' is in registers: the next chunk's products may overwrite it
           tc_fence_before_sync();
@@ -816,7 +868,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const int vt = MODE == 1 ? tid : (tid >> 7) * 64 + ((warp & 3) - 2) * 32 + lane;
         float vm = 0.f;
 #pragma unroll 4
-        for (int i = 0; i < nslab * 512 / vthreads; ++i) {
+        for (int i = 0; i < vslab * 512 / vthreads; ++i) {
           const uint32_t ad = sb + OFF_V + (uint32_t)(vt + vthreads * i) * 16;
           float x[8];
           unpack8(lds128(ad), x);
@@ -852,7 +904,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const float L2E = 1.4426950408889634f;
     // the dropped softmax normalizer of the query rows only matters next to eps, and without normalization
     const bool need_qsum = a.eps != 0.f || !a.normalize;
-    const uint32_t mail_mine = lane_base + COL_MAIL + 2 + ch, mail_other = lane_base + COL_MAIL + 2 + (ch ^ 1);
+    const uint32_t mail_mine = lane_base + cMAIL + 2 + ch, mail_other = lane_base + cMAIL + 2 + (ch ^ 1);
     const uint32_t ycol = lane_base + COL_Y + ch * 64;
     float dsum = 0.f;  // log2 of this state row's total decay over the segment
     bool fail = false;
@@ -863,26 +915,31 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       WAITSETF(BIT(B_P) | (m > 0 ? BIT(B_MMA3) : 0u), PAR(B_P, m & 1) | PAR(B_MMA3, (m - 1) & 1));
       if (fail) return;
       tc_fence_after_sync();
-      float s[32];
-      tmem_ld32(lane_base + COL_P + ch * 32, s);
-      tmem_wait_ld();
       // The chunk's own part of the denominator is the row sum of the masked scores AS ROUNDED to fp16: numerator and
       // denominator then carry the same weights (the first tokens of a sequence do not average a mismatch out).
+      // (pair: this thread masks all 64 columns of its own head's scores, two blocks of 32, into that head's tile)
       float rs = 0.f;
+#pragma unroll 1
+      for (int hb = 0; hb < (pair ? 2 : 1); ++hb) {
+        const int c32 = pair ? hb : ch;  // which block of 32 key tokens
+        float s[32];
+        tmem_ld32(lane_base + (pair ? (ch ? cP2 : cP) : cP) + c32 * 32, s);
+        tmem_wait_ld();
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        uint32_t w[4];
+        for (int q4 = 0; q4 < 4; ++q4) {
+          uint32_t w[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int col = ch * 32 + q4 * 8 + 2 * i;
-          const __half2 h2 = __floats2half2_rn(col <= row ? s[q4 * 8 + 2 * i] : 0.f, col + 1 <= row ? s[q4 * 8 + 2 * i + 1] : 0.f);
-          const float2 f2 = __half22float2(h2);
-          rs += f2.x + f2.y;
-          w[i] = *reinterpret_cast<const uint32_t*>(&h2);
+          for (int i = 0; i < 4; ++i) {
+            const int col = c32 * 32 + q4 * 8 + 2 * i;
+            const __half2 h2 = __floats2half2_rn(col <= row ? s[q4 * 8 + 2 * i] : 0.f, col + 1 <= row ? s[q4 * 8 + 2 * i + 1] : 0.f);
+            const float2 f2 = __half22float2(h2);
+            rs += f2.x + f2.y;
+            w[i] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          sts128(sb + ((pair && ch) ? OFF_PH2 : OFF_PH) + sw128(row, c32 * 4 + q4), make_uint4(w[0], w[1], w[2], w[3]));
         }
-        sts128(sb + OFF_PH + sw128(row, ch * 4 + q4), make_uint4(w[0], w[1], w[2], w[3]));
       }
-      tmem_st1(lane_base + COL_MAIL + 8 + 2 * (m & 1) + ch, rs);
+      tmem_st1(lane_base + cMAIL + 8 + 2 * (m & 1) + ch, rs);
       tmem_wait_st();
       fence_proxy_async();
       tc_fence_before_sync();
@@ -921,7 +978,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int i = 0; i < 16; ++i) m = fmaxf(m, yb[i]);
           }
         }
-        if (!narrow) {
+        if (wide) {  // (narrow, pair: a row's softmax lives in one thread's 64 columns)
           if (!fail) {
             tmem_st1(mail_mine, m);
             tmem_wait_st();
@@ -957,7 +1014,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
               tmem_st16(ycol + b2 * 32 + 16, yb);
             }
           }
-          if (!narrow) {
+          if (wide) {
             named_bar_sync(phi_bar, 128);  // the partner has read the row max out of the mailbox
             if (!fail) {
               tmem_st1(mail_mine, sum);
@@ -992,10 +1049,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const float dm = ex2f(bm), dC = ex2f(bm + ft);
         if (ch == 0) dsum += bm + ft;
         float mx = 0.f;
+        // (pair: 64 value columns, 32 per thread)
 #pragma unroll 1
-        for (int b2 = 0; b2 < 2; ++b2) {
-          const int blk = ch * 2 + b2;
-          tmem_ld32(lane_base + COL_S + blk * 32, y);
+        for (int b2 = 0; b2 < (pair ? 1 : 2); ++b2) {
+          const int blk = pair ? ch : ch * 2 + b2;
+          tmem_ld32(lane_base + cS + blk * 32, y);
           tmem_wait_ld();
           if (MODE == 0) {
             if (track) {
@@ -1009,7 +1067,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
               for (int i = 0; i < 4; ++i) w[i] = f2_mul(dm2, f2_pack(y[8 * q4 + 2 * i], y[8 * q4 + 2 * i + 1]));
               // columns [8 nb, 8 nb + 8) of row c: block nb of the unswizzled operand (a warp's 32 rows: 512 contiguous bytes)
-              sts128(sb + OFF_SBF + (uint32_t)(ch * 8 + b2 * 4 + q4) * 2048u + (uint32_t)c * 16u, pack8p(w, f16));
+              sts128(sb + OFF_SBF + (uint32_t)(blk * 4 + q4) * 2048u + (uint32_t)c * 16u, pack8p(w, f16));
             }
           }
           {
@@ -1017,16 +1075,16 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 32; i += 2) f2_unpack(f2_mul(dC2, f2_pack(y[i], y[i + 1])), y[i], y[i + 1]);
           }
-          tmem_st32(lane_base + COL_S + blk * 32, y);
+          tmem_st32(lane_base + cS + blk * 32, y);
         }
         if (ch == (narrow ? 0 : 1)) {  // (the thread of the row's last existing column half also carries z)
-          const float z = tmem_ld1(lane_base + COL_SZ);
+          const float z = tmem_ld1(lane_base + cSZ);
           tmem_wait_ld();
           if (MODE == 0) {
-            *reinterpret_cast<uint16_t*>(sg + OFF_SBF + (dh >> 3) * 2048 + c * 16) = to16(dm * z, f16);
+            *reinterpret_cast<uint16_t*>(sg + OFF_SBF + (hd >> 3) * 2048 + c * 16) = to16(dm * z, f16);
             if (track) mx = fmaxf(mx, fabsf(z));
           }
-          tmem_st1(lane_base + COL_SZ, dC * z);
+          tmem_st1(lane_base + cSZ, dC * z);
         }
         if (MODE == 0 && track) {
           mx = warp_max(mx);
@@ -1067,7 +1125,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           }
           if (need_qsum) {
             // the dropped normalizer travels to the output pass through tensor memory: each half adds its part
-            tmem_st1(lane_base + COL_MAIL + 4 * p + ch, qsum);
+            tmem_st1(lane_base + cMAIL + 4 * p + ch, qsum);
             tmem_wait_st();
           }
         } else {
@@ -1129,27 +1187,28 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ---- final state -------------------------------------------------------------------------------------------------
     if (!fail && !*s_abort && (nchunks == 0 || wait_or_abort(bar(B_MMA2), (uint32_t)((nchunks - 1) & 1), s_abort, a.wait_limit))) {
       tc_fence_after_sync();
-      const int c = r128;
-      if (a.dtot != nullptr && ch == 0 && c < dh) a.dtot[seg_idx * dh + c] = dsum;
+      const int c = r128, cr = c & (hd - 1);  // state row, and the row inside its real head's state
+      const size_t out_idx = state_idx(c, a.seg_out);
+      if (a.dtot != nullptr && ch == 0 && c < dh) a.dtot[state_idx(c, 1) * hd + cr] = dsum;
       const bool last = a.seg_out || seg == a.nseg - 1;  // (each of the two outputs is optional on its own)
       if (a.S_T != nullptr && last) {
         float s[32];
 #pragma unroll 1
-        for (int b2 = 0; b2 < 2; ++b2) {
-          const int blk = ch * 2 + b2;
-          tmem_ld32(lane_base + COL_S + blk * 32, s);
+        for (int b2 = 0; b2 < (pair ? 1 : 2); ++b2) {
+          const int blk = pair ? ch : ch * 2 + b2;
+          tmem_ld32(lane_base + cS + blk * 32, s);
           tmem_wait_ld();
-          if (c < dh && blk * 32 < dh) {
+          if (c < dh && blk * 32 < hd) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
-              *reinterpret_cast<float4*>(a.S_T + (out_idx * dh + c) * dh + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
+              *reinterpret_cast<float4*>(a.S_T + (out_idx * hd + cr) * hd + blk * 32 + i) = make_float4(s[i], s[i + 1], s[i + 2], s[i + 3]);
           }
         }
       }
       if (a.z_T != nullptr && last && ch == 1) {
-        const float z = tmem_ld1(lane_base + COL_SZ);
+        const float z = tmem_ld1(lane_base + cSZ);
         tmem_wait_ld();
-        if (c < dh) a.z_T[out_idx * dh + c] = z;
+        if (c < dh) a.z_T[out_idx * hd + cr] = z;
       }
     }
   }
