@@ -200,3 +200,26 @@ def decode_step(p: OracleParams, q_t, k_t, v_t, gate_t, w_q, w_k, W, S, z, cache
                   np.reshape(v_t, (B, 1, Hkv, dv)), np.reshape(gate_t, (B, 1, H, p.gd)), w_q, w_k, W,
                   cache_q, cache_k, S, z)
     return dict(o=r["o"].reshape(B, H, dv), S=r["S_T"], z=r["z_T"], cache_q=r["cache_q"], cache_k=r["cache_k"])
+
+
+def gate_logits(x, A1, A2, bias=None):
+    """The gate function in front of the layer (Section 4.2: additional linear layers whose output goes through a sigmoid;
+    appendix, ablation on the rank of the gate function: two consecutive low-rank linear layers).
+    x [B,T,d_model], A1 [rank,d_model] (first layer), A2 [n_out,rank] (second layer), bias [n_out] or None ->
+    logits a [B,T,n_out] with a_t = A2 (A1 x_t) + bias. n_out = H * gate_dim: reshaped to [B,T,H,gate_dim] they are the
+    `gate` input of gla_fwd / layer_fwd, where the sigmoid and the power 1/tau are applied (GATE_LOGITS)."""
+    x, A1, A2, bias = map(_f64, (x, A1, A2, bias))
+    B, T, dm = x.shape
+    rank, n_out = A1.shape[0], A2.shape[0]
+    assert A1.shape == (rank, dm) and A2.shape == (n_out, rank)
+    h = np.empty((B, T, rank))
+    for b in range(B):
+        for t in range(T):
+            h[b, t] = A1 @ x[b, t]          # bottleneck activations of token t
+    a = np.empty((B, T, n_out))
+    for b in range(B):
+        for t in range(T):
+            a[b, t] = A2 @ h[b, t]
+            if bias is not None:
+                a[b, t] += bias
+    return a

@@ -6,6 +6,8 @@ that the CPU oracle and the GPU see identical bits), and names the benchmark con
 
 Recipe: q, k, v ~ N(0,1); gate logits ~ N(0,1); mix weights W_h ~ N(0, 1/d_k); conv taps ~ N(0, 1/conv_k);
 upstream gradients ~ N(0,1). Tensor i of configuration c uses seed BASE_SEED + 16*c + i.
+Gate function (two low-rank linear layers in front of the gate): hidden states x ~ N(0,1), first layer ~ N(0, 1/d_model),
+second layer ~ N(0, 1/rank), bias ~ N(0, 1/4), so that the logits are about N(0, 1.25); seeds BASE_SEED + 2^20 + 16*c + i.
 """
 from __future__ import annotations
 
@@ -101,4 +103,18 @@ def make(shape: LayerShape, names, seed_offset: int = 0) -> dict:
         elif s.dtype == "bf16":
             a = round_to_bf16(a)
         out[n] = a
+    return out
+
+
+def make_gate_fn(shape: LayerShape, d_model: int, rank: int, seed_offset: int = 0) -> dict:
+    """Inputs of the gate function for a workload: x [B,T,d_model], A1 [rank,d_model], A2 [H*gate_dim,rank],
+    bias [H*gate_dim], float32 arrays (bf16-representable values for dtype 'bf16')."""
+    s = shape
+    n_out = s.H * s.gd
+    shp = dict(x=(s.B, s.T, d_model), A1=(rank, d_model), A2=(n_out, rank), bias=(n_out,))
+    scale = dict(x=1.0, A1=1.0 / np.sqrt(d_model), A2=1.0 / np.sqrt(rank), bias=0.5)
+    out = {}
+    for i, n in enumerate(("x", "A1", "A2", "bias")):
+        a = _normal(BASE_SEED + (1 << 20) + 16 * s.config_id + i + 1024 * seed_offset, shp[n], scale[n])
+        out[n] = round_to_bf16(a) if s.dtype == "bf16" else a
     return out

@@ -460,3 +460,72 @@ def test_unshared_linear_streams_are_independent_and_gradients_match_finite_diff
     for name, arr, got in (("q", q, g2["dq"]), ("k", k, g2["dk"]), ("w_q", wq, g2["dw_q"]), ("w_k", wk, g2["dw_k"]),
                            ("W", W, g2["dW"])):
         np.testing.assert_allclose(got, _fd(f, arr, dO), rtol=5e-6, atol=1e-8, err_msg=name)
+
+
+# ---- gate function (Section 4.2; appendix on the rank of the gate function) -------------------------------------------
+def _gate_fn_inputs(B=2, T=5, dm=12, rank=3, n_out=8, seed=77):
+    g = np.random.default_rng(seed)
+    return (g.standard_normal((B, T, dm)), g.standard_normal((rank, dm)), g.standard_normal((n_out, rank)),
+            g.standard_normal(n_out))
+
+
+def test_gate_function_brute_force_sums():
+    """Every logit written out as the double sum over the bottleneck units and the hidden channels."""
+    x, A1, A2, b = _gate_fn_inputs()
+    got = O.gate_logits(x, A1, A2, b)
+    for bb in range(x.shape[0]):
+        for t in range(x.shape[1]):
+            for j in range(A2.shape[0]):
+                want = b[j]
+                for r in range(A1.shape[0]):
+                    hr = 0.0
+                    for c in range(A1.shape[1]):
+                        hr += A1[r, c] * x[bb, t, c]
+                    want += A2[j, r] * hr
+                assert abs(got[bb, t, j] - want) <= 1e-12 * (1 + abs(want))
+
+
+def test_gate_function_is_one_matrix_of_bounded_rank():
+    """Two consecutive linear layers are the single linear layer A2 A1 (library product), whose rank is at most the
+    bottleneck width; without a bias the map is linear in x."""
+    x, A1, A2, b = _gate_fn_inputs(rank=3)
+    M = A2 @ A1
+    assert np.linalg.matrix_rank(M) <= 3
+    np.testing.assert_allclose(O.gate_logits(x, A1, A2, None), np.einsum("jc,btc->btj", M, x), rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(O.gate_logits(x, A1, A2, b) - O.gate_logits(x, A1, A2, None),
+                               np.broadcast_to(b, (2, 5, 8)), rtol=0, atol=1e-12)
+    y = np.random.default_rng(5).standard_normal(x.shape)
+    np.testing.assert_allclose(O.gate_logits(2.0 * x - 3.0 * y, A1, A2, None),
+                               2.0 * O.gate_logits(x, A1, A2, None) - 3.0 * O.gate_logits(y, A1, A2, None),
+                               rtol=1e-11, atol=1e-11)
+
+
+def test_gate_function_special_cases():
+    """Rank 1: logit j of token t is (u . x_t) w_j. Full rank with an identity first layer: a plain linear layer.
+    A transposed operand or swapped layers would change the shape or the value in each of these."""
+    g = np.random.default_rng(3)
+    x = g.standard_normal((1, 4, 6)); u = g.standard_normal((1, 6)); w = g.standard_normal((5, 1))
+    got = O.gate_logits(x, u, w)
+    for t in range(4):
+        np.testing.assert_allclose(got[0, t], float(u[0] @ x[0, t]) * w[:, 0], rtol=1e-12)
+    A2 = g.standard_normal((5, 6)); b = g.standard_normal(5)
+    np.testing.assert_allclose(O.gate_logits(x, np.eye(6), A2, b), x @ A2.T + b, rtol=1e-12, atol=1e-12)
+    # a first layer that picks hidden channel 2 and a second layer that routes it to logit 4 only
+    A1 = np.zeros((1, 6)); A1[0, 2] = 1.0
+    A2 = np.zeros((5, 1)); A2[4, 0] = 2.0
+    want = np.zeros((1, 4, 5)); want[0, :, 4] = 2.0 * x[0, :, 2]
+    np.testing.assert_array_equal(O.gate_logits(x, A1, A2), want)
+
+
+def test_gate_function_feeds_the_decay_of_eq4():
+    """The logits are the layer's `gate` input: through gla_fwd the decay of channel c at token t is
+    sigmoid(a_tc)^(1/tau) (Section 4.2). One token after a known state isolates it."""
+    x, A1, A2, b = _gate_fn_inputs(B=1, T=1, dm=7, rank=2, n_out=2 * 4)
+    a = O.gate_logits(x, A1, A2, b).reshape(1, 1, 2, 4)
+    p = O.OracleParams(1, 1, 2, 2, 4, 4, gate_tau=3.0)
+    S0 = np.ones((1, 2, 4, 4)); z0 = np.ones((1, 2, 4))
+    zero = np.zeros((1, 1, 2, 4))
+    r = O.gla_fwd(p, zero + 1.0, zero, zero, a, S0, z0)     # k = 0: the state only decays
+    alpha = (1.0 / (1.0 + np.exp(-a[0, 0]))) ** (1.0 / 3.0)  # [H, d_k]
+    np.testing.assert_allclose(r["S_T"][0], alpha[:, :, None] * S0[0], rtol=1e-12)
+    np.testing.assert_allclose(r["z_T"][0], alpha * z0[0], rtol=1e-12)
