@@ -138,6 +138,27 @@ int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const 
                     size_t ws_bytes, void* stream, int* dev_status);
 
 /*
+ * The gate function in front of the layer (Section 4.2: additional linear layers whose output goes through a sigmoid;
+ * appendix, ablation on the rank of the gate function: two consecutive low-rank linear layers, rank 16 ... 128 or full):
+ *   a_t = A2 (A1 x_t) + bias
+ *   x [B,T,d_model] hidden states, A1 [rank,d_model] first layer, A2 [H*gate_dim,rank] second layer,
+ *   bias [H*gate_dim] (nullable), all in p->dtype
+ *   out: gate [B,T,H,gate_dim] in p->dtype: the logits, i.e. the `gate` input of the entry points below with
+ *        gate_mode = LAWCAT_GATE_LOGITS, which apply the sigmoid and the power 1/gate_tau where they read them.
+ * Only B, T, H, gate_dim, dtype and chunk of *p are used. d_model <= 16384, rank <= 1024.
+ * Kernels: bf16 storage with rank 16, 32, 64 or 128, d_model and H*gate_dim multiples of 8 runs both layers in one
+ * tensor-core kernel (bf16 operands, the bottleneck activations as a two-term bf16 pair, fp32 accumulation; one rounding
+ * to bf16 at the end); every other case, and chunk = 1, runs exact fp32 kernels with the bottleneck activations [B*T,rank]
+ * in fp32 scratch (lawcat_gate_fn_workspace_bytes; 0 for the tensor-core kernel).
+ * Errors: as for every entry point (see the top of this header); the tensor-core kernel's waits are bounded
+ * (LAWCAT_ERR_TIMEOUT through dev_status).
+ */
+size_t lawcat_gate_fn_workspace_bytes(const lawcat_params* p, int32_t d_model, int32_t rank);
+int lawcat_gate_fn_fwd(const lawcat_params* p, int32_t d_model, int32_t rank, const void* x, const void* A1,
+                       const void* A2, const void* bias, void* gate, void* ws, size_t ws_bytes, void* stream,
+                       int* dev_status);
+
+/*
  * Backward of lawcat_conv_fwd (needed by the layer-wise distillation of Section 5.1; the paper prints no formulas,
  * this is the chain rule on conv -> mix -> phi). d_qdot, d_kdot have the shapes of the forward outputs.
  *   out: dq [B,T,H,d_k], dk [B,T,H_kv,d_k] in p->dtype; dw_q, dw_k, dW in fp32, shaped like w_q, w_k, W.

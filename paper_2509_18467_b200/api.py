@@ -24,7 +24,8 @@ EXPORTS = ["lawcat_workspace_bytes", "lawcat_status_string", "lawcat_version", "
            "lawcat_trace_begin", "lawcat_trace_end", "lawcat_test_set_wait_limit", "lawcat_conv_fwd", "lawcat_conv_bwd", "lawcat_gla_fwd",
            "lawcat_gla_bwd", "lawcat_layer_fwd", "lawcat_layer_fwd_varlen_workspace_bytes",
            "lawcat_layer_fwd_varlen", "lawcat_layer_bwd", "lawcat_decode_step", "lawcat_layer_fwd_host_arena_bytes",
-           "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc", "lawcat_last_cuda_error"]
+           "lawcat_layer_fwd_host", "lawcat_noalloc_scratch_bytes", "lawcat_layer_fwd_noalloc", "lawcat_last_cuda_error", "lawcat_gate_fn_workspace_bytes",
+           "lawcat_gate_fn_fwd"]
 
 
 class LawcatError(RuntimeError):
@@ -168,6 +169,27 @@ def lawcat_conv_fwd(p: Params, q, k, w_q, w_k, W=None, cache_q=None, cache_k=Non
     ws, nb = _ws(p, OP_CONV_FWD, ws, dev)
     _call("lawcat_conv_fwd", p, [q, k, w_q, w_k, W, cache_q, cache_k, qdot, kdot], ws, nb, stream, dev_status)
     return qdot, kdot
+
+
+def lawcat_gate_fn_fwd(p: Params, d_model: int, rank: int, x, A1, A2, bias=None, gate=None, ws=None, stream=None,
+                       dev_status=None):
+    """x [B,T,d_model], A1 [rank,d_model], A2 [H*gate_dim,rank], bias [H*gate_dim] -> gate logits [B,T,H,gate_dim]."""
+    dt, dev = torch_dtype(p), x.device
+    if gate is None:
+        gate = torch.empty(p.B, p.T, p.H, p.gate_dim, dtype=dt, device=dev)
+    f = lib().lawcat_gate_fn_workspace_bytes
+    f.restype = ctypes.c_size_t
+    f.argtypes = [ctypes.POINTER(Params), ctypes.c_int32, ctypes.c_int32]
+    need = f(ctypes.byref(p), d_model, rank)
+    if ws is None and need:
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    nb = 0 if ws is None else ws.numel() * ws.element_size()
+    st = lib().lawcat_gate_fn_fwd(ctypes.byref(p), ctypes.c_int32(d_model), ctypes.c_int32(rank), _ptr(x), _ptr(A1),
+                                  _ptr(A2), _ptr(bias), _ptr(gate), _ptr(ws), ctypes.c_size_t(nb), _stream(stream),
+                                  _ptr(dev_status))
+    if st != 0:
+        raise LawcatError(st, "lawcat_gate_fn_fwd")
+    return gate
 
 
 def lawcat_conv_bwd(p: Params, q, k, w_q, w_k, W, d_qdot, d_kdot, cache_q=None, cache_k=None, ws=None, stream=None,

@@ -161,6 +161,30 @@ int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const 
   return launch_conv_plain(c, k, w_k, cache_k, kdot, p->H_kv);
 }
 
+size_t lawcat_gate_fn_workspace_bytes(const lawcat_params* p, int32_t d_model, int32_t rank) {
+  if (check_params(p, true) != LAWCAT_OK || d_model <= 0 || rank <= 0) return 0;
+  return align_up(gate_fn_workspace_bytes(*p, d_model, rank), 256);
+}
+
+int lawcat_gate_fn_fwd(const lawcat_params* p, int32_t d_model, int32_t rank, const void* x, const void* A1,
+                       const void* A2, const void* bias, void* gate, void* ws, size_t ws_bytes, void* stream,
+                       int* dev_status) {
+  int r = check_params(p, true);
+  if (r) return r;
+  if (d_model <= 0 || rank <= 0) return LAWCAT_ERR_INVALID_ARG;
+  if (d_model > 16384 || rank > 1024) return LAWCAT_ERR_UNSUPPORTED;
+  if ((long long)p->B * p->T > 0x7fffffffLL) return LAWCAT_ERR_UNSUPPORTED;
+  const bool empty = (size_t)p->B * p->T == 0;
+  const void* const req[] = {x, gate};
+  const void* const opt[] = {bias, ws};
+  if ((r = check_ptrs(req, opt, empty))) return r;
+  if (!A1 || !A2 || !aligned16(A1) || !aligned16(A2)) return LAWCAT_ERR_INVALID_ARG;
+  const size_t need = lawcat_gate_fn_workspace_bytes(p, d_model, rank);
+  if (need && !empty && (!ws || ws_bytes < need)) return LAWCAT_ERR_WORKSPACE_TOO_SMALL;
+  Ctx c{p, (cudaStream_t)stream, dev_status};
+  return launch_gate_fn(c, d_model, rank, x, A1, A2, bias, gate, ws);
+}
+
 int lawcat_conv_bwd(const lawcat_params* p, const void* q, const void* k, const void* w_q, const void* w_k,
                     const void* W, const void* cache_q, const void* cache_k, const void* d_qdot,
                     const void* d_kdot, void* dq, void* dk, float* dw_q, float* dw_k, float* dW, void* ws,

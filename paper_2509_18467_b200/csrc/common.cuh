@@ -100,6 +100,12 @@ int launch_convmix_tc_bwd(const Ctx& c, const void* q, const void* k, const void
                           const void* cache_q, const void* cache_k, const void* d_qdot, const void* d_kdot, bool grads_f32,
                           float* du_q, float* du_k, float* dW);
 
+// The gate function in front of the layer: two consecutive low-rank linear layers producing the gate logits (gate_fn.cu).
+bool gate_fn_tc_supported(const lawcat_params& p, int d_model, int rank);
+size_t gate_fn_workspace_bytes(const lawcat_params& p, int d_model, int rank);
+int launch_gate_fn(const Ctx& c, int d_model, int rank, const void* x, const void* A1, const void* A2, const void* bias,
+                   void* gate, void* ws);
+
 // Counts one kernel launch; while tracing is on it also brackets the launch with CUDA events on its stream.
 struct LaunchScope {
   LaunchScope(const char* name, cudaStream_t s);

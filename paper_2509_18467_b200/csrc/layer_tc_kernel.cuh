@@ -202,24 +202,6 @@ __device__ __forceinline__ float log2_sigmoid(float a) {
   return -fmaxf(x, lg2f(1.f + ex2f(fminf(x, 126.f))));
 }
 
-__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
-// Named barrier that also returns the OR of `flag` over its threads: roles that synchronize among themselves leave
-// their loop only through such a barrier, all together.
-__device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool flag) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 q, %3, 0;\n\t"
-      "bar.red.or.pred p, %1, %2, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r)
-      : "r"(id), "r"(nthreads), "r"((uint32_t)flag)
-      : "memory");
-  return r != 0;
-}
-
 // Bounded wait that also gives up as soon as another role has raised the abort flag.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
