@@ -10,6 +10,8 @@ Workloads (seeded synthetic inputs of `paper_2509_18467_b200.inputs`, through th
   c4                    distillation step: `lawcat_layer_fwd` (the output the loss needs) + `lawcat_layer_bwd` (every gradient of
                         the layer for a seeded upstream gradient) at B = 8, T = 1024
   c5-decode             one recurrent `lawcat_decode_step` for B = 64 sequences
+  c3-gate-fn            the gate function in front of the c3 layer: one `lawcat_gate_fn_fwd` (hidden states of width 4096 ->
+                        rank 32 -> 4096 gate logits per token) over the 32768 tokens
 Prints ONE JSON line (rank 0). N > 1 runs N independent replicas (the layer has no inter-GPU exchange), one process per
 GPU; the time is the max over ranks. Started without a launcher, `--gpus N` starts the N ranks itself.
 
@@ -38,24 +40,29 @@ UNIT = "tokens/s"
 LAYER_NAMES = ["q", "k", "v", "gate", "w_q", "w_k", "W"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 SWEEP_T = (1024, 4096, 16384, 65536, 131072)
-WORKLOADS = ["c1", "c2", "c3", "c4", "c5-decode"] + [f"c5-T{t}" for t in SWEEP_T]
+WORKLOADS = ["c1", "c2", "c3", "c4", "c5-decode"] + [f"c5-T{t}" for t in SWEEP_T] + ["c3-gate-fn"]
+# the gate function in front of the headline layer: hidden width of the 7B model, the rank the paper settles on
+GATE_FN = {"d_model": 4096, "rank": 32}
 
 
 def workload_shape(name: str) -> I.LayerShape:
     if name.startswith("c5-T"):
         T = int(name[4:])
         return dataclasses.replace(I.CONFIGS["c3"], T=T, config_id=5, name=f"c5-mistral-7b-T{T}")
+    if name == "c3-gate-fn":
+        return dataclasses.replace(I.CONFIGS["c3"], name="c3-gate-fn-mistral-7b-T32768")
     return I.CONFIGS[name]
 
 
 def workload_kind(name: str) -> str:
-    return {"c4": "train", "c5-decode": "decode"}.get(name, "prefill")
+    return {"c4": "train", "c5-decode": "decode", "c3-gate-fn": "gatefn"}.get(name, "prefill")
 
 
 def metric_name(kind: str) -> str:
     return {"prefill": "prefill tokens/sec per LAWCAT layer",
             "train": "training tokens/sec per LAWCAT layer (forward + backward)",
-            "decode": "decode tokens/sec per LAWCAT layer (one token per sequence and step)"}[kind]
+            "decode": "decode tokens/sec per LAWCAT layer (one token per sequence and step)",
+            "gatefn": "gate-function tokens/sec per LAWCAT layer (hidden states -> gate logits)"}[kind]
 
 
 def peaks():
@@ -82,6 +89,9 @@ def io_bytes_per_token(s: I.LayerShape) -> dict:
 def alg_bytes_per_step(kind: str, s: I.LayerShape) -> float:
     b = io_bytes_per_token(s)
     fwd = b["q"] + b["k"] + b["v"] + b["gate"] + b["o"]
+    if kind == "gatefn":    # hidden states read once, logits written once, the two weight matrices and the bias once
+        dm, r, n_out = GATE_FN["d_model"], GATE_FN["rank"], s.H * s.gd
+        return (es(s) * dm + b["gate"]) * s.B * s.T + es(s) * (r * dm + n_out * r + n_out)
     if kind == "prefill":   # q, k, v, gate read once, o written once
         return fwd * s.B * s.T
     if kind == "train":     # forward; backward: the inputs and dO read once, dq, dk, dv, dgate written once
@@ -93,6 +103,8 @@ def alg_bytes_per_step(kind: str, s: I.LayerShape) -> float:
 
 def alg_flops_per_step(kind: str, s: I.LayerShape) -> float:
     """Recurrent minimum (chunk overhead not credited): mix on both streams, state update + read-out, conv."""
+    if kind == "gatefn":
+        return 2.0 * GATE_FN["rank"] * (GATE_FN["d_model"] + s.H * s.gd) * s.B * s.T
     G = s.H // s.H_kv
     per_tok = s.H * (4.0 * s.d_k * s.d_k + 4.0 * s.d_k * (s.d_v + 1) + 2.0 * s.conv_k * s.d_k * (1 + 1.0 / G))
     tokens = s.B * (1 if kind == "decode" else s.T)
@@ -180,6 +192,12 @@ def oracle_sample(kind: str, s: I.LayerShape, x: dict, tokens: int):
     that hold `tokens` tokens; decode: the step of every sequence."""
     from oracle import lawcat_oracle as O
     O.threads()  # build / load outside the timed region
+    if kind == "gatefn":
+        Ts = min(tokens, s.T)
+        t0 = time.perf_counter()
+        a = O.gate_logits(x["x"][:, :Ts], x["A1"], x["A2"], x["bias"])
+        dt = time.perf_counter() - t0
+        return dt, dict(gate=a.reshape(s.B, Ts, s.H, s.gd)), s.B * Ts, 1, f"first {Ts} of {s.T} tokens, one pass ({dt:.1f} s)"
     if kind == "prefill":
         Ts = min(tokens, s.T)
         p = oracle_params_of(dataclasses.replace(s, T=Ts))
@@ -214,6 +232,8 @@ def make_inputs(kind: str, s: I.LayerShape) -> dict:
     stand-in prefill: S0, z0 and caches drawn by the same generator (positive states, as positive features produce)."""
     if kind == "prefill":
         return I.make(s, LAYER_NAMES)
+    if kind == "gatefn":
+        return I.make_gate_fn(s, GATE_FN["d_model"], GATE_FN["rank"])
     if kind == "train":
         return I.make(s, LAYER_NAMES + ["dO"])
     x = I.make(dataclasses.replace(s, T=1), LAYER_NAMES + ["S0", "z0", "cache_q", "cache_k"])
@@ -228,7 +248,7 @@ def run_reference(args):
     kind = workload_kind(args.workload)
     s = workload_shape(args.workload)
     sample = args.ref_tokens
-    if kind == "prefill":
+    if kind in ("prefill", "gatefn"):
         s_small = dataclasses.replace(s, T=min(s.T, sample))
     elif kind == "train":
         s_small = dataclasses.replace(s, B=max(1, min(s.B, sample // s.T)))
@@ -323,6 +343,8 @@ class Runner:
         if kind == "prefill":
             self.o = torch.empty(s.B, s.T, s.H, s.d_v, dtype=self.tdt, device=dev)
             self.ws = torch.empty(max(api.workspace_bytes(p, api.OP_LAYER_FWD), 16), dtype=torch.uint8, device=dev)
+        elif kind == "gatefn":
+            self.o = torch.empty(s.B, s.T, s.H, s.gd, dtype=self.tdt, device=dev)
         elif kind == "train":
             self.o = torch.empty(s.B, s.T, s.H, s.d_v, dtype=self.tdt, device=dev)
             self.ws = torch.empty(max(api.workspace_bytes(p, api.OP_LAYER_FWD), 16), dtype=torch.uint8, device=dev)
@@ -337,6 +359,8 @@ class Runner:
         api, d, p = self.api, self.d, self.p
         if self.kind == "prefill":   # the state and the caches are part of what a prefill hands back
             self.res = api.lawcat_layer_fwd(p, *[d[n] for n in LAYER_NAMES], o=self.o, ws=self.ws)
+        elif self.kind == "gatefn":
+            api.lawcat_gate_fn_fwd(p, GATE_FN["d_model"], GATE_FN["rank"], d["x"], d["A1"], d["A2"], d["bias"], gate=self.o)
         elif self.kind == "train":
             api.lawcat_layer_fwd(p, *[d[n] for n in LAYER_NAMES], o=self.o, want_state=False, want_cache=False, ws=self.ws)
             g = api.lawcat_layer_bwd(p, *[d[n] for n in LAYER_NAMES], d["dO"], ws=self.ws_b)
@@ -355,7 +379,8 @@ class Runner:
         torch, api, s = self.torch, self.api, self.s
         # what arrives with every step: the whole batch for prefill and training; for decode the token's tensors (the
         # state and the conv caches live on the device and are advanced in place)
-        names = {"prefill": LAYER_NAMES, "train": LAYER_NAMES[:4] + ["dO"], "decode": LAYER_NAMES[:4]}[self.kind]
+        names = {"prefill": LAYER_NAMES, "train": LAYER_NAMES[:4] + ["dO"], "decode": LAYER_NAMES[:4],
+                 "gatefn": ["x"]}[self.kind]
         self.h = {n: (self.d[n].cpu().pin_memory()) for n in names}
         if self.kind == "prefill":
             self.h_o = torch.empty(s.B, s.T, s.H, s.d_v, dtype=self.tdt).pin_memory()
@@ -514,6 +539,8 @@ def run_ours(args):
             return strict if f32_store else comp
         if kind == "prefill":
             errs = {"o": err(R.o, ref["o"])}
+        elif kind == "gatefn":
+            errs = {"gate": err(R.o, ref["gate"])}
         elif kind == "train":
             # the oracle differentiates the whole layer from the raw inputs
             errs = {n: err(R.res[n], ref[n], n in ("dw_q", "dw_k", "dW")) for n in ("o", "dq", "dk", "dv", "dgate",

@@ -6,14 +6,17 @@
 //
 // Tensor-core kernel (bf16 storage, rank 16 / 32 / 64 / 128): one thread block per 128 tokens, three roles.
 //   copy warp      first layer: x tiles [128 tokens x 64 hidden channels] and A1 tiles [rank x 64] through a ring of
-//                  stages (TMA, 128-byte swizzle); second layer: A2 tiles [128 outputs x rank], double buffered
+//                  stages (TMA, 128-byte swizzle)
 //   product warp   H = X A1^T accumulated over d_model in tensor memory (M = 128, N = rank); then per 128 outputs
 //                  OUT = [H_hi | H_lo] [A2 | A2]^T (M = 128, N = 128) into one of two accumulators
-//   4 epilogue     H: tensor memory -> two-term bf16 (hi + lo, 16 significant bits) -> shared-memory operand;
-//     warps        OUT: tensor memory -> + bias -> bf16 -> swizzled staging tile -> TMA store (clipped at the tensor's edge)
+//   4 epilogue     A2 tiles [128 outputs x rank] from L2 into the operand layout, two tiles ahead of the products (rows
+//     warps        of 2 * rank bytes are too short for efficient TMA boxes; the loads of a tile are issued before the
+//                  epilogue of the tile two earlier and stored behind it);
+//                  H: tensor memory -> two-term bf16 (hi + lo, 16 significant bits) -> shared-memory operand;
+//                  OUT: tensor memory -> + bias -> bf16 -> swizzled staging tile -> TMA store (clipped at the tensor's edge)
 // x and the logits cross HBM once each (the roofline of the kernel); A1 and A2 are re-read from L2 by every block.
 // The buffers of the second layer alias the ring of the first (which is drained by then) except the A2 tiles, so that
-// the first of those is already in flight while the first layer finishes.
+// the first two of those are in place while the first layer runs.
 // Every wait is bounded: a wait that runs out raises the block's abort flag, every role leaves its loop, the block lets
 // its copies land, frees its tensor memory and reports LAWCAT_ERR_TIMEOUT through dev_status.
 //
@@ -52,7 +55,7 @@ struct Lay {
   static constexpr uint32_t OUT_BYTES = TT * NT * 2;                // staging: 2 slabs of [128 x 128 B], swizzled
   static constexpr uint32_t SLAB_H = TT * 16 + 16;                  // H operand: octet slabs of 128 rows (padded)
   static constexpr uint32_t H_BYTES = (2 * R / 8) * SLAB_H;         // columns [0, R) hi, [R, 2R) lo
-  static constexpr uint32_t SLAB_B = NT * 16;                       // A2 operand: octet slabs of 128 rows, written by TMA
+  static constexpr uint32_t SLAB_B = NT * 16 + 16;                  // A2 operand: octet slabs of 128 rows (padded)
   static constexpr uint32_t B_BYTES = (R / 8) * SLAB_B;
   static constexpr uint32_t OFF_RING = 0;
   static constexpr uint32_t OFF_OUT = 0;                            // (second layer: over the drained ring)
@@ -67,10 +70,11 @@ struct Lay {
 };
 
 // mbarriers
-enum { B_FULL0 = 0, B_EMPTY0 = 4, B_HFULL = 8, B_HREADY, B_BFULL0, B_BEMPTY0 = B_BFULL0 + 2, B_ACCFULL0 = B_BEMPTY0 + 2,
-       B_ACCFREE0 = B_ACCFULL0 + 2, NUM_BARS = B_ACCFREE0 + 2 };
+enum { B_FULL0 = 0, B_EMPTY0 = 4, B_HFULL = 8, B_HREADY, B_BFULL0, B_ACCFULL0 = B_BFULL0 + 2, B_ACCFREE0 = B_ACCFULL0 + 2,
+       NUM_BARS = B_ACCFREE0 + 2 };
 
 struct GArgs {
+  const bf16* A2;     // [n_out, rank]
   const bf16* bias;   // [n_out] or null
   int N, dm, n_out;
   int* dev_status;
@@ -94,7 +98,7 @@ __device__ __forceinline__ bool gwait(uint32_t bar, uint32_t parity, volatile in
 template <int R>
 __global__ void __launch_bounds__(THREADS)
 gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_a1,
-                  const __grid_constant__ CUtensorMap tm_a2, const __grid_constant__ CUtensorMap tm_out, const GArgs a) {
+                  const __grid_constant__ CUtensorMap tm_out, const GArgs a) {
   using L = Lay<R>;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sb = smem_u32(smem);
@@ -110,11 +114,11 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   if (tid == 0) {
     if (sb & 1023u) { s_flags[1] = 1; } else { s_flags[1] = 0; }
     for (int i = 0; i < NUM_BARS; ++i) {
-      const bool many = i == B_HREADY || i == B_ACCFREE0 || i == B_ACCFREE0 + 1;
+      const bool many = i == B_HREADY || i == B_ACCFREE0 || i == B_ACCFREE0 + 1 || i == B_BFULL0 || i == B_BFULL0 + 1;
       mbar_init(BAR(i), many ? EPI_THREADS : 1);
     }
     mbar_fence_init();
-    tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_a1); tma_prefetch_desc(&tm_a2); tma_prefetch_desc(&tm_out);
+    tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_a1); tma_prefetch_desc(&tm_out);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<int*>(s_flags)), TMEM_COLS);
@@ -128,11 +132,6 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   if (warp == 0) {
     // ------------------------------------------------------------------------------------------------ copies
     if (lane == 0) {
-      // the first A2 tiles do not touch the ring: they go out at once
-      for (int nt = 0; nt < 2 && nt < ntile; ++nt) {
-        mbar_arrive_expect_tx(BAR(B_BFULL0 + nt), L::B_BYTES);
-        tma_load_3d(sb + L::OFF_B + nt * L::B_BYTES, &tm_a2, BAR(B_BFULL0 + nt), 0, nt * NT, 0);
-      }
       bool ok = true;
       for (int i = 0; i < nk && ok; ++i) {
         const int s = i % L::ST;
@@ -141,13 +140,6 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         mbar_arrive_expect_tx(BAR(B_FULL0 + s), L::STAGE);
         tma_load_2d(sb + L::OFF_RING + s * L::STAGE, &tm_x, BAR(B_FULL0 + s), i * KS, n0);
         tma_load_2d(sb + L::OFF_RING + s * L::STAGE + L::X_BYTES, &tm_a1, BAR(B_FULL0 + s), i * KS, 0);
-      }
-      for (int nt = 2; nt < ntile && ok; ++nt) {
-        const int b = nt & 1;
-        ok = gwait(BAR(B_BEMPTY0 + b), ((nt >> 1) - 1) & 1, s_abort);
-        if (!ok) break;
-        mbar_arrive_expect_tx(BAR(B_BFULL0 + b), L::B_BYTES);
-        tma_load_3d(sb + L::OFF_B + b * L::B_BYTES, &tm_a2, BAR(B_BFULL0 + b), 0, nt * NT, 0);
       }
     }
   } else if (warp == 1) {
@@ -187,8 +179,7 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
           for (int kk = 0; kk < R / 16; ++kk)
             mma_f16(acc, dadv(dh, (uint32_t)(part * (R / 8) + 2 * kk) * L::SLAB_H), dadv(db, (uint32_t)(2 * kk) * L::SLAB_B),
                     idesc2, (part | kk) != 0);
-        mma_commit(BAR(B_BEMPTY0 + b));
-        mma_commit(BAR(B_ACCFULL0 + b));
+        mma_commit(BAR(B_ACCFULL0 + b));  // (also: the A2 tile in buffer b has been read)
       }
     }
   } else {
@@ -196,6 +187,29 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     const int et = tid - 64;                     // 0 ... 127
     const int row = (warp & 3) * 32 + lane;      // token row of the tile = TMEM lane
     const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    // A2 tile nt as registers of this thread: 16-byte piece idx = et + 128 k is octet idx % (R / 8) of output row idx / (R / 8)
+    constexpr int BPT = NT * (R / 8) / EPI_THREADS;  // pieces per thread
+    uint4 breg[BPT];
+    auto b_load = [&](int nt) {
+#pragma unroll
+      for (int k = 0; k < BPT; ++k) {
+        const int idx = et + k * EPI_THREADS, j = nt * NT + idx / (R / 8), o = idx % (R / 8);
+        breg[k] = j < a.n_out ? __ldg(reinterpret_cast<const uint4*>(a.A2 + (size_t)j * R + o * 8)) : make_uint4(0u, 0u, 0u, 0u);
+      }
+    };
+    auto b_store = [&](int b) {
+#pragma unroll
+      for (int k = 0; k < BPT; ++k) {
+        const int idx = et + k * EPI_THREADS;
+        *reinterpret_cast<uint4*>(smem + L::OFF_B + b * L::B_BYTES + (idx % (R / 8)) * L::SLAB_B + (idx / (R / 8)) * 16) = breg[k];
+      }
+      fence_proxy_async();
+      mbar_arrive(BAR(B_BFULL0 + b));
+    };
+    for (int nt = 0; nt < 2 && nt < ntile; ++nt) {   // (the first two tiles: while the first layer runs)
+      b_load(nt);
+      b_store(nt);
+    }
     bool fail = !gwait(BAR(B_HFULL), 0, s_abort);
     if (!fail) {
       tc_fence_after_sync();
@@ -230,6 +244,8 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       fail = named_bar_or(1, EPI_THREADS, fail);
       if (fail) break;
       tc_fence_after_sync();
+      const bool more = nt + 2 < ntile;
+      if (more) b_load(nt + 2);   // (in flight during this tile's epilogue)
       const uint32_t acc = tlane + (uint32_t)b * NT;
       uint8_t* const stg = smem + L::OFF_OUT + b * L::OUT_BYTES;
 #pragma unroll 1
@@ -247,6 +263,7 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       }
       tc_fence_before_sync();
       mbar_arrive(BAR(B_ACCFREE0 + b));
+      if (more) b_store(b);       // (the products of tile nt, which read buffer b, completed before this tile's accumulator did)
       fence_proxy_async();
       named_bar_sync(2, EPI_THREADS);
       if (et == 0) {
@@ -329,27 +346,12 @@ static bool map_2d(CUtensorMap* m, const void* ptr, size_t rows, size_t cols, in
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// A2 [n_out, rank] as (8 channels of an octet, output row, octet): a box of 8 x 128 x rank/8 lands as octet slabs of 128
-// rows, the unswizzled K-major operand layout
-static bool map_a2(CUtensorMap* m, const void* ptr, int n_out, int rank) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[3] = {8, (cuuint64_t)n_out, (cuuint64_t)(rank / 8)};
-  const cuuint64_t strides[2] = {(cuuint64_t)rank * 2, 16};
-  const cuuint32_t box[3] = {8, (cuuint32_t)NT, (cuuint32_t)(rank / 8)};
-  const cuuint32_t es[3] = {1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int R>
 static int launch_tc(const Ctx& c, int d_model, const void* x, const void* A1, const void* A2, const void* bias,
                      void* gate, size_t N, int n_out) {
   using L = Lay<R>;
-  CUtensorMap tx, ta1, ta2, to;
-  if (!map_2d(&tx, x, N, d_model, TT) || !map_2d(&ta1, A1, R, d_model, R) || !map_a2(&ta2, A2, n_out, R) ||
-      !map_2d(&to, gate, N, n_out, TT))
+  CUtensorMap tx, ta1, to;
+  if (!map_2d(&tx, x, N, d_model, TT) || !map_2d(&ta1, A1, R, d_model, R) || !map_2d(&to, gate, N, n_out, TT))
     return LAWCAT_ERR_CUDA;
   static std::atomic<bool> raised[64] = {};
   int dev = 0;
@@ -359,9 +361,9 @@ static int launch_tc(const Ctx& c, int d_model, const void* x, const void* A1, c
       return LAWCAT_ERR_CUDA;
     raised[dev].store(true);
   }
-  GArgs a{(const bf16*)bias, (int)N, d_model, n_out, c.dev_status};
+  GArgs a{(const bf16*)A2, (const bf16*)bias, (int)N, d_model, n_out, c.dev_status};
   LAWCAT_LAUNCH("gate_fn_tc", c.stream,
-                gate_fn_tc_kernel<R><<<(unsigned)((N + TT - 1) / TT), THREADS, L::BYTES, c.stream>>>(tx, ta1, ta2, to, a));
+                gate_fn_tc_kernel<R><<<(unsigned)((N + TT - 1) / TT), THREADS, L::BYTES, c.stream>>>(tx, ta1, to, a));
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }
