@@ -9,11 +9,14 @@
 //                  stages (TMA, 128-byte swizzle)
 //   product warp   H = X A1^T accumulated over d_model in tensor memory (M = 128, N = rank); then per 128 outputs
 //                  OUT = [H_hi | H_lo] [A2 | A2]^T (M = 128, N = 128) into one of two accumulators
-//   4 epilogue     A2 tiles [128 outputs x rank] from L2 into the operand layout, two tiles ahead of the products (rows
+//   2 x 4 epilogue A2 tiles [128 outputs x rank] from L2 into the operand layout, two tiles ahead of the products (rows
 //     warps        of 2 * rank bytes are too short for efficient TMA boxes; the loads of a tile are issued before the
 //                  epilogue of the tile two earlier and stored behind it);
 //                  H: tensor memory -> two-term bf16 (hi + lo, 16 significant bits) -> shared-memory operand;
-//                  OUT: tensor memory -> + bias -> bf16 -> swizzled staging tile -> TMA store (clipped at the tensor's edge)
+//                  OUT: tensor memory -> + bias -> bf16 -> swizzled staging tile -> TMA store (clipped at the tensor's edge).
+//                  Two groups of four warps take the output tiles in turn, each with an accumulator, an A2 buffer and a
+//                  staging tile of its own: a tile's chain of waits (product, tensor-memory load, store) is long compared
+//                  with its arithmetic, and two chains side by side hide most of it.
 // x and the logits cross HBM once each (the roofline of the kernel); A1 and A2 are re-read from L2 by every block.
 // The buffers of the second layer alias the ring of the first (which is drained by then) except the A2 tiles, so that
 // the first two of those are in place while the first layer runs.
@@ -41,8 +44,8 @@ using ctc::toff;
 constexpr int TT = 128;        // tokens per thread block
 constexpr int NT = 128;        // outputs per product of the second layer
 constexpr int KS = 64;         // hidden channels per stage of the first layer
-constexpr int THREADS = 192;   // warp 0 copies, warp 1 products, warps 2-5 epilogue (TMEM quadrant = warp & 3)
-constexpr int EPI_THREADS = 128;
+constexpr int THREADS = 320;   // warp 0 copies, warp 1 products, warps 2-5 and 6-9 epilogue groups (TMEM quadrant = warp & 3)
+constexpr int EPI_THREADS = 128;  // per group
 constexpr uint32_t TMEM_COLS = 256;  // accumulator 0 = columns 0-127 (H uses its first `rank` columns first), 1 = 128-255
 constexpr long long WAIT_LIMIT = 400000000LL;  // clock cycles (about a fifth of a second)
 
@@ -96,7 +99,7 @@ __device__ __forceinline__ bool gwait(uint32_t bar, uint32_t parity, volatile in
 }
 
 template <int R>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, R <= 32 ? 2 : 1)   // (rank <= 32: two blocks per SM, so at most 102 registers)
 gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_a1,
                   const __grid_constant__ CUtensorMap tm_out, const GArgs a) {
   using L = Lay<R>;
@@ -184,7 +187,8 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     }
   } else {
     // ------------------------------------------------------------------------------------------------ epilogue
-    const int et = tid - 64;                     // 0 ... 127
+    const int g = (warp - 2) >> 2;               // group: output tiles g, g + 2, ...
+    const int et = (tid - 64) & 127;             // thread of the group
     const int row = (warp & 3) * 32 + lane;      // token row of the tile = TMEM lane
     const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     // A2 tile nt as registers of this thread: 16-byte piece idx = et + 128 k is octet idx % (R / 8) of output row idx / (R / 8)
@@ -206,12 +210,18 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       fence_proxy_async();
       mbar_arrive(BAR(B_BFULL0 + b));
     };
-    for (int nt = 0; nt < 2 && nt < ntile; ++nt) {   // (the first two tiles: while the first layer runs)
-      b_load(nt);
-      b_store(nt);
+    if (g < ntile) {   // (each group's first tile: while the first layer runs)
+      b_load(g);
+      b_store(g);
     }
-    bool fail = !gwait(BAR(B_HFULL), 0, s_abort);
-    if (!fail) {
+    // this thread's entry of a tile's bias, fetched one tile ahead (its latency must not sit between two tiles)
+    auto bias_load = [&](int nt) -> float {
+      const int j = nt * NT + et;
+      return (a.bias && nt < ntile && j < a.n_out) ? __bfloat162float(a.bias[j]) : 0.f;
+    };
+    float bias_next = bias_load(g);
+    bool fail = g == 0 && !gwait(BAR(B_HFULL), 0, s_abort);
+    if (g == 0 && !fail) {
       tc_fence_after_sync();
 #pragma unroll 1
       for (int c0 = 0; c0 < R; c0 += 16) {
@@ -233,15 +243,13 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       tc_fence_before_sync();
       mbar_arrive(BAR(B_HREADY));
     }
-    for (int nt = 0; nt < ntile; ++nt) {
-      const int b = nt & 1;
+    for (int nt = g; nt < ntile; nt += 2) {
+      const int b = g;
       if (!fail) fail = !gwait(BAR(B_ACCFULL0 + b), (nt >> 1) & 1, s_abort);
-      {
-        const int j = nt * NT + et;
-        s_bias[b * NT + et] = (a.bias && j < a.n_out) ? __bfloat162float(a.bias[j]) : 0.f;
-      }
-      if (et == 0) tma_store_wait_read_1();  // the store that read staging tile b two tiles ago is through with it
-      fail = named_bar_or(1, EPI_THREADS, fail);
+      s_bias[b * NT + et] = bias_next;
+      bias_next = bias_load(nt + 2);
+      if (et == 0) tma_store_wait_read();  // the group's previous store is through with the staging tile
+      fail = named_bar_or(1 + 2 * g, EPI_THREADS, fail);
       if (fail) break;
       tc_fence_after_sync();
       const bool more = nt + 2 < ntile;
@@ -249,23 +257,26 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       const uint32_t acc = tlane + (uint32_t)b * NT;
       uint8_t* const stg = smem + L::OFF_OUT + b * L::OUT_BYTES;
 #pragma unroll 1
-      for (int cb = 0; cb < NT / 32; ++cb) {
-        float v[32];
-        tmem_ld32(acc + (uint32_t)cb * 32, v);
+      for (int sl = 0; sl < NT / 64; ++sl) {   // one 64-column slab of the staging tile per round: both loads, one wait
+        float v[64];
+        tmem_ld32(acc + (uint32_t)sl * 64, v);
+        tmem_ld32(acc + (uint32_t)sl * 64 + 32, v + 32);
         tmem_wait_ld();
-        const float* bs = s_bias + b * NT + cb * 32;
+        const float4* bs = reinterpret_cast<const float4*>(s_bias + b * NT + sl * 64);
+        uint8_t* const slab = stg + sl * (TT * 128);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] += bs[i];
-        uint8_t* const slab = stg + (cb >> 1) * (TT * 128);
-#pragma unroll
-        for (int o = 0; o < 4; ++o)
-          *reinterpret_cast<uint4*>(slab + sw128(row, (cb & 1) * 4 + o)) = ctc::pack8bf16(v + 8 * o);
+        for (int o = 0; o < 8; ++o) {
+          const float4 b0 = bs[2 * o], b1 = bs[2 * o + 1];
+          v[8 * o] += b0.x; v[8 * o + 1] += b0.y; v[8 * o + 2] += b0.z; v[8 * o + 3] += b0.w;
+          v[8 * o + 4] += b1.x; v[8 * o + 5] += b1.y; v[8 * o + 6] += b1.z; v[8 * o + 7] += b1.w;
+          *reinterpret_cast<uint4*>(slab + sw128(row, o)) = ctc::pack8bf16(v + 8 * o);
+        }
       }
       tc_fence_before_sync();
       mbar_arrive(BAR(B_ACCFREE0 + b));
       if (more) b_store(b);       // (the products of tile nt, which read buffer b, completed before this tile's accumulator did)
       fence_proxy_async();
-      named_bar_sync(2, EPI_THREADS);
+      named_bar_sync(2 + 2 * g, EPI_THREADS);
       if (et == 0) {
         tma_store_2d(&tm_out, smem_u32(stg), nt * NT, n0);
         if (nt * NT + 64 < a.n_out) tma_store_2d(&tm_out, smem_u32(stg) + TT * 128, nt * NT + 64, n0);

@@ -76,8 +76,6 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int
                ::"l"(tmap), "r"(src), "r"(c0), "r"(c1)
                : "memory");
 }
-// (at most one store group of this thread may still be reading its shared-memory source)
-__device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------------------------- proxies and fences
 // Orders this thread's generic-proxy shared-memory writes before later async-proxy (TMA, tcgen05.mma) accesses.
