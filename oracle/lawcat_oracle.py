@@ -223,3 +223,11 @@ def gate_logits(x, A1, A2, bias=None):
             if bias is not None:
                 a[b, t] += bias
     return a
+
+
+def gate_log_decay(a, tau):
+    """Section 4.2: the gate is the sigmoid of the logits; with the exponent 1/tau of the gate scaling the log of the decay
+    of one entry is log(sigmoid(a)) / tau (what GATE_LOGDECAY inputs hold). Written as -(max(-a, 0) + log1p(exp(-|a|))) / tau,
+    the form without overflow."""
+    a = _f64(a)
+    return -(np.maximum(-a, 0.0) + np.log1p(np.exp(-np.abs(a)))) / float(tau)

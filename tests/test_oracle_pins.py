@@ -529,3 +529,23 @@ def test_gate_function_feeds_the_decay_of_eq4():
     alpha = (1.0 / (1.0 + np.exp(-a[0, 0]))) ** (1.0 / 3.0)  # [H, d_k]
     np.testing.assert_allclose(r["S_T"][0], alpha[:, :, None] * S0[0], rtol=1e-12)
     np.testing.assert_allclose(r["z_T"][0], alpha * z0[0], rtol=1e-12)
+
+
+def test_gate_log_decay_is_the_log_of_the_gate():
+    """exp(log-decay) = sigmoid(a)^(1/tau) by the textbook sigmoid (moderate logits), the far tails behave like a / tau and
+    like -exp(-a) / tau, and the layer run on log-decays (GATE_LOGDECAY) equals the layer run on the logits themselves."""
+    a = np.linspace(-20.0, 20.0, 81)
+    for tau in (1.0, 3.0, 16.0):
+        g = O.gate_log_decay(a, tau)
+        np.testing.assert_allclose(np.exp(g), (1.0 / (1.0 + np.exp(-a))) ** (1.0 / tau), rtol=1e-12)
+        assert (g < 0).all() and (np.diff(g) > 0).all()
+    np.testing.assert_allclose(O.gate_log_decay(np.array([-800.0]), 4.0), [-200.0], rtol=1e-12)
+    np.testing.assert_allclose(O.gate_log_decay(np.array([40.0]), 2.0), [-np.exp(-40.0) / 2.0], rtol=1e-9)
+    g = np.random.default_rng(8)
+    B, T, H, d = 1, 9, 2, 4
+    q, k, v = (np.abs(g.standard_normal((B, T, H, d))) for _ in range(3))
+    logits = 2.0 * g.standard_normal((B, T, H, d))
+    r0 = O.gla_fwd(O.OracleParams(B, T, H, H, d, d, gate_tau=5.0), q, k, v, logits)
+    r1 = O.gla_fwd(O.OracleParams(B, T, H, H, d, d, gate_mode=O.GATE_LOGDECAY), q, k, v, O.gate_log_decay(logits, 5.0))
+    for n in ("o", "S_T", "z_T"):
+        np.testing.assert_allclose(r1[n], r0[n], rtol=1e-11, atol=1e-13)
