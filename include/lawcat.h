@@ -148,8 +148,11 @@ int lawcat_conv_fwd(const lawcat_params* p, const void* q, const void* k, const 
  * Only B, T, H, gate_dim, dtype and chunk of *p are used. d_model <= 16384, rank <= 1024.
  * Kernels: bf16 storage with rank 16, 32, 64 or 128, d_model and H*gate_dim multiples of 8 runs both layers in one
  * tensor-core kernel (bf16 operands, the bottleneck activations as a two-term bf16 pair, fp32 accumulation; one rounding
- * to bf16 at the end); every other case, and chunk = 1, runs exact fp32 kernels with the bottleneck activations [B*T,rank]
- * in fp32 scratch (lawcat_gate_fn_workspace_bytes; 0 for the tensor-core kernel).
+ * to bf16 at the end). Calls of up to 1024 tokens (a decode step, a short prompt; bf16, rank, d_model and H*gate_dim
+ * multiples of 8) run a latency-oriented fp32 CUDA-core kernel instead (about 18 us for a decode step of 64 sequences at
+ * the 7B widths, where one block of the tensor-core kernel takes 50). Every other case, and chunk = 1, runs exact fp32
+ * kernels with the bottleneck activations [B*T,rank] in fp32 scratch (lawcat_gate_fn_workspace_bytes; 0 for the other two
+ * kernels).
  * Errors: as for every entry point (see the top of this header); the tensor-core kernel's waits are bounded
  * (LAWCAT_ERR_TIMEOUT through dev_status).
  */

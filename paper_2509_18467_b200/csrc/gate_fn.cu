@@ -23,6 +23,11 @@
 // Every wait is bounded: a wait that runs out raises the block's abort flag, every role leaves its loop, the block lets
 // its copies land, frees its tensor memory and reports LAWCAT_ERR_TIMEOUT through dev_status.
 //
+// Few tokens (a decode step, a short call; bf16, widths multiples of 8): one block of the tensor-core kernel walks its
+// 64 stages and 32 output tiles one after the other, about 50 us whatever the number of tokens. Up to a few hundred tokens
+// gate_fn_small_kernel takes over: one thread block per token (or per four), both layers on the CUDA cores in fp32 with
+// the bottleneck activations in shared memory, every load a 16-byte one and many in flight; the weights come from L2.
+//
 // Exact kernels (any storage type and shape): fp32 accumulation on the CUDA cores, h in fp32 scratch.
 #include <cuda.h>
 
@@ -330,6 +335,89 @@ __global__ void __launch_bounds__(256) gate_fn_out_kernel(const float* __restric
   }
 }
 
+// ---------------------------------------------------------------------------------------------------- few tokens
+// One block per TOK tokens, 256 threads. First layer: warp w takes the bottleneck units w, w + 8, ...; its lanes stride
+// over the hidden channels in octets and meet in a shuffle sum. Second layer: a thread takes 8 consecutive outputs at a
+// time (their rows of A2 are contiguous) and keeps TOK x 8 sums.
+template <int TOK>
+__global__ void __launch_bounds__(256) gate_fn_small_kernel(const bf16* __restrict__ x, const bf16* __restrict__ A1,
+                                                            const bf16* __restrict__ A2, const bf16* __restrict__ bias,
+                                                            bf16* __restrict__ out, int N, int dm, int rank, int n_out) {
+  extern __shared__ __align__(16) uint8_t sm_small[];
+  uint4* const s_x = reinterpret_cast<uint4*>(sm_small);                           // [TOK][dm / 8] octets of bf16
+  float* const s_h = reinterpret_cast<float*>(sm_small + (size_t)TOK * dm * 2);    // [TOK][rank]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n0 = blockIdx.x * TOK, oct = dm >> 3;
+  for (int i = tid; i < TOK * oct; i += 256) {
+    const int t = i / oct, o = i - t * oct;
+    s_x[i] = n0 + t < N ? __ldg(reinterpret_cast<const uint4*>(x + (size_t)(n0 + t) * dm) + o) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  __syncthreads();
+  // (four units at a time, so that a lane has 16 loads of A1 in flight)
+  for (int r0 = warp; r0 < rank; r0 += 32) {
+    float acc[4][TOK];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int t = 0; t < TOK; ++t) acc[u][t] = 0.f;
+#pragma unroll 4
+    for (int c = lane; c < oct; c += 32) {
+      uint4 wa[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        wa[u] = r0 + 8 * u < rank ? __ldg(reinterpret_cast<const uint4*>(A1 + (size_t)(r0 + 8 * u) * dm) + c)
+                                  : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int t = 0; t < TOK; ++t) {
+        float fx[8];
+        ctc::unpack8b(s_x[t * oct + c], fx);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          float fa[8];
+          ctc::unpack8b(wa[u], fa);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc[u][t] = fmaf(fa[i], fx[i], acc[u][t]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int t = 0; t < TOK; ++t) {
+        const float v = warp_sum(acc[u][t]);
+        if (lane == 0 && r0 + 8 * u < rank) s_h[t * rank + r0 + 8 * u] = v;
+      }
+  }
+  __syncthreads();
+  for (int jo = tid; jo * 8 < n_out; jo += 256) {
+    const int j0 = jo * 8;
+    float acc[TOK][8];
+    {
+      float fb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (bias) ctc::unpack8b(__ldg(reinterpret_cast<const uint4*>(bias + j0)), fb);
+#pragma unroll
+      for (int t = 0; t < TOK; ++t)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[t][e] = fb[e];
+    }
+#pragma unroll 4
+    for (int rr = 0; rr < rank; rr += 8) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        float fa[8];
+        ctc::unpack8b(__ldg(reinterpret_cast<const uint4*>(A2 + (size_t)(j0 + e) * rank + rr)), fa);
+#pragma unroll
+        for (int t = 0; t < TOK; ++t)
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc[t][e] = fmaf(fa[i], s_h[t * rank + rr + i], acc[t][e]);
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < TOK; ++t)
+      if (n0 + t < N) *reinterpret_cast<uint4*>(out + (size_t)(n0 + t) * n_out + j0) = ctc::pack8bf16(acc[t]);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -379,6 +467,21 @@ static int launch_tc(const Ctx& c, int d_model, const void* x, const void* A1, c
   return LAWCAT_OK;
 }
 
+template <int TOK>
+static int launch_small(const Ctx& c, int d_model, int rank, const void* x, const void* A1, const void* A2,
+                        const void* bias, void* gate, size_t N, int n_out) {
+  const size_t smem = (size_t)TOK * d_model * 2 + sizeof(float) * (size_t)TOK * rank;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(gate_fn_small_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return LAWCAT_ERR_CUDA;
+  LAWCAT_LAUNCH("gate_fn_small", c.stream,
+                gate_fn_small_kernel<TOK><<<(unsigned)((N + TOK - 1) / TOK), 256, smem, c.stream>>>(
+                    (const bf16*)x, (const bf16*)A1, (const bf16*)A2, (const bf16*)bias, (bf16*)gate, (int)N, d_model, rank,
+                    n_out));
+  LAWCAT_CHECK_LAUNCH();
+  return LAWCAT_OK;
+}
+
 template <typename T>
 static int launch_exact(const Ctx& c, int d_model, int rank, const void* x, const void* A1, const void* A2,
                         const void* bias, void* gate, size_t N, int n_out, void* ws) {
@@ -405,8 +508,22 @@ bool gate_fn_tc_supported(const lawcat_params& p, int d_model, int rank) {
          n_out % 8 == 0 && p.chunk != 1;
 }
 
+// Few tokens: the latency-oriented CUDA-core kernel (see the head of this file). SMALL_1: tokens up to which one block per
+// token is used, SMALL_4: up to which one block per four tokens; beyond, the tensor-core kernel where it applies.
+constexpr size_t SMALL_1 = 128, SMALL_4 = 1024;
+// tokens per block of the few-token kernel for this call, 0 = not its case
+static int gate_fn_small_tok(const lawcat_params& p, int d_model, int rank) {
+  const long long n_out = (long long)p.H * p.gate_dim;
+  const size_t N = (size_t)p.B * p.T;
+  if (p.dtype != LAWCAT_BF16 || rank % 8 != 0 || d_model % 8 != 0 || n_out % 8 != 0 || p.chunk == 1) return 0;
+  if (N <= SMALL_1) return 1;
+  if (N <= SMALL_4 && d_model <= 8192) return 4;
+  return 0;
+}
+
 size_t gate_fn_workspace_bytes(const lawcat_params& p, int d_model, int rank) {
   if (gate_fn_tc_supported(p, d_model, rank)) return 0;
+  if (gate_fn_small_tok(p, d_model, rank)) return 0;
   return sizeof(float) * (size_t)p.B * p.T * rank;
 }
 
@@ -416,6 +533,11 @@ int launch_gate_fn(const Ctx& c, int d_model, int rank, const void* x, const voi
   const size_t N = (size_t)p.B * p.T;
   const int n_out = p.H * p.gate_dim;
   if (N == 0) return LAWCAT_OK;
+  switch (gate_fn_small_tok(p, d_model, rank)) {
+    case 1: return gfn::launch_small<1>(c, d_model, rank, x, A1, A2, bias, gate, N, n_out);
+    case 4: return gfn::launch_small<4>(c, d_model, rank, x, A1, A2, bias, gate, N, n_out);
+    default: break;
+  }
   if (gate_fn_tc_supported(p, d_model, rank)) {
     switch (rank) {
       case 16: return gfn::launch_tc<16>(c, d_model, x, A1, A2, bias, gate, N, n_out);

@@ -1,8 +1,9 @@
 """The gate function (two consecutive low-rank linear layers producing the gate logits; Section 4.2 and the appendix's
 ablation on its rank) through the C ABI against the fp64 oracle: the tensor-core kernel for bf16 and rank 16 / 32 / 64 /
-128 (ragged token tiles, hidden widths that are not a multiple of the stage width, output widths that are not a multiple
-of the product width, with and without a bias), the exact kernels for everything else, the logits feeding the layer, the
-benchmark's size on sampled tokens, and the edge cases.
+128 and more than 1024 tokens (ragged token tiles, hidden widths that are not a multiple of the stage width, output widths
+that are not a multiple of the product width, with and without a bias), the latency-oriented kernel for up to 1024 tokens,
+the exact kernels for everything else, the logits feeding the layer, the benchmark's size on sampled tokens, and the edge
+cases.
 
 Tolerance, bf16 storage: the logits are rounded to bf16 once, so beyond that rounding (half an ulp, allowed by
 metrics.err_bf16) the error must stay below 1e-3 of the RMS (bottleneck activations carry 16 significant bits, products
@@ -17,7 +18,7 @@ from paper_2509_18467_b200.metrics import err_bf16, err_f32
 pytestmark = pytest.mark.gpu
 
 
-def run(B, T, H, d, gd, dm, rank, dtype="bf16", bias=True, chunk=0, cfg=900, expect_tc=None):
+def run(B, T, H, d, gd, dm, rank, dtype="bf16", bias=True, chunk=0, cfg=900, expect_tc=None, expect_kernel=None):
     import torch
     from paper_2509_18467_b200 import api
     s = I.LayerShape(B, T, H, H, d, d, dtype=dtype, gate_dim=gd, config_id=cfg)
@@ -31,6 +32,8 @@ def run(B, T, H, d, gd, dm, rank, dtype="bf16", bias=True, chunk=0, cfg=900, exp
     assert int(status.item()) == 0
     if expect_tc is not None:
         assert ("gate_fn_tc" in kernels) == expect_tc, kernels
+    if expect_kernel is not None:
+        assert expect_kernel in kernels, kernels
     want = O.gate_logits(x["x"], x["A1"], x["A2"], x["bias"] if bias else None).reshape(B, T, H, s.gd)
     got = g.float().cpu().numpy()
     assert got.shape == want.shape and np.isfinite(got).all()
@@ -39,34 +42,56 @@ def run(B, T, H, d, gd, dm, rank, dtype="bf16", bias=True, chunk=0, cfg=900, exp
 
 @pytest.mark.parametrize("rank", [16, 32, 64, 128])
 @pytest.mark.parametrize("B,T,H,d,gd,dm", [
-    (2, 193, 3, 64, 0, 256),     # 386 tokens: three full tiles and a ragged one; 192 outputs = 1.5 products
-    (1, 128, 2, 128, 0, 320),    # exactly one tile; five stages (more than the ring holds)
-    (1, 70, 8, 64, 1, 72),       # one decay per head: 8 outputs; hidden width 72 = one stage and an eighth
-    (3, 50, 4, 128, 0, 1024),    # 16 stages, 512 outputs
+    (6, 193, 3, 64, 0, 256),     # 1158 tokens: nine full tiles and a ragged one; 192 outputs = 1.5 products
+    (9, 128, 2, 128, 0, 320),    # whole tiles only; five stages (more than the ring holds)
+    (15, 70, 8, 64, 1, 72),      # one decay per head: 8 outputs; hidden width 72 = one stage and an eighth
+    (21, 50, 4, 128, 0, 1024),   # 16 stages, 512 outputs
 ])
 def test_tensor_core_kernel(rank, B, T, H, d, gd, dm):
+    """More than 1024 tokens: the tensor-core kernel."""
     got, want = run(B, T, H, d, gd, dm, rank, expect_tc=True, cfg=900 + rank)
     _, e = err_bf16(got, want)
     assert e <= 1e-3, f"{e:.3e}"
 
 
-def test_without_bias_and_single_token():
-    got, want = run(1, 1, 2, 64, 0, 128, 32, bias=False, expect_tc=True)
+@pytest.mark.parametrize("rank", [8, 24, 32, 128])
+@pytest.mark.parametrize("B,T,H,d,gd,dm", [
+    (1, 1, 2, 64, 0, 128),       # one token (a decode step of one sequence)
+    (64, 1, 32, 128, 0, 4096),   # the decode step of the benchmark's batch at the 7B model's widths
+    (2, 193, 3, 64, 0, 256),     # 386 tokens: blocks of four tokens, the last one ragged
+    (1, 70, 8, 64, 1, 72),       # 8 outputs; hidden width 72 (fewer octets than lanes)
+    (1, 1024, 1, 64, 0, 64),     # the largest call of this kernel
+])
+def test_few_tokens_kernel(rank, B, T, H, d, gd, dm):
+    """Up to 1024 tokens (bf16, widths multiples of 8; any rank that is a multiple of 8): the latency-oriented kernel."""
+    import ctypes
+    from paper_2509_18467_b200 import api
+    got, want = run(B, T, H, d, gd, dm, rank, expect_tc=False, expect_kernel="gate_fn_small", cfg=930 + rank)
+    assert err_bf16(got, want)[1] <= 1e-4
+    p = api.params(B, T, H, H, d, d, gate_dim=gd)
+    f = api.lib().lawcat_gate_fn_workspace_bytes
+    f.restype = ctypes.c_size_t
+    f.argtypes = [ctypes.POINTER(api.Params), ctypes.c_int32, ctypes.c_int32]
+    assert f(ctypes.byref(p), dm, rank) == 0   # (no scratch: the bottleneck activations stay in shared memory)
+
+
+def test_without_bias():
+    got, want = run(1, 1, 2, 64, 0, 128, 32, bias=False, expect_tc=False)
     assert err_bf16(got, want)[1] <= 1e-3
-    got, want = run(2, 129, 2, 64, 0, 128, 16, bias=False, expect_tc=True)
+    got, want = run(9, 129, 2, 64, 0, 128, 16, bias=False, expect_tc=True)
     assert err_bf16(got, want)[1] <= 1e-3
 
 
 @pytest.mark.parametrize("dtype,rank,dm,H,d,gd,chunk", [
     ("f32", 5, 50, 3, 16, 0, 0),        # nothing about the shape suits the tensor-core kernel
     ("f32", 32, 256, 2, 64, 0, 0),      # fp32 storage
-    ("bf16", 24, 96, 2, 64, 0, 0),      # a rank the tensor-core kernel does not take
+    ("bf16", 20, 96, 2, 64, 0, 0),      # a rank neither bf16 kernel takes
     ("bf16", 32, 256, 2, 64, 0, 1),     # chunk = 1 asks for the exact kernels
     ("bf16", 16, 132, 2, 64, 0, 0),     # hidden width not a multiple of 8
     ("bf16", 16, 128, 3, 64, 1, 0),     # 3 outputs
 ])
 def test_exact_kernels(dtype, rank, dm, H, d, gd, chunk):
-    got, want = run(2, 37, H, d, gd, dm, rank, dtype=dtype, chunk=chunk, expect_tc=False, cfg=950)
+    got, want = run(2, 37, H, d, gd, dm, rank, dtype=dtype, chunk=chunk, expect_tc=False, expect_kernel="gate_fn_h", cfg=950)
     if dtype == "f32":
         assert err_f32(got, want) <= 1e-5
     else:
