@@ -31,6 +31,7 @@
 // Exact kernels (any storage type and shape): fp32 accumulation on the CUDA cores, h in fp32 scratch.
 #include <cuda.h>
 
+#include <algorithm>
 #include <atomic>
 
 #include "common.cuh"
@@ -117,7 +118,11 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
   float* const s_bias = reinterpret_cast<float*>(smem + L::OFF_BIAS);
   auto BAR = [&](int i) { return bars + 8u * (uint32_t)i; };
   const int n0 = blockIdx.x * TT;
-  const int nk = (a.dm + KS - 1) / KS, ntile = (a.n_out + NT - 1) / NT;
+  // With fewer token tiles than SMs the output tiles of a token tile are shared out over gridDim.y blocks (each repeats the
+  // first layer, whose x tile then comes from L2): this block's tiles are nt0 ... nt0 + ntile - 1, `nt` below counts from 0.
+  const int nk = (a.dm + KS - 1) / KS, ntile_all = (a.n_out + NT - 1) / NT;
+  const int per_y = (ntile_all + (int)gridDim.y - 1) / (int)gridDim.y, nt0 = (int)blockIdx.y * per_y;
+  const int ntile = min(per_y, ntile_all - nt0);
 
   if (tid == 0) {
     if (sb & 1023u) { s_flags[1] = 1; } else { s_flags[1] = 0; }
@@ -202,7 +207,7 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     auto b_load = [&](int nt) {
 #pragma unroll
       for (int k = 0; k < BPT; ++k) {
-        const int idx = et + k * EPI_THREADS, j = nt * NT + idx / (R / 8), o = idx % (R / 8);
+        const int idx = et + k * EPI_THREADS, j = (nt0 + nt) * NT + idx / (R / 8), o = idx % (R / 8);
         breg[k] = j < a.n_out ? __ldg(reinterpret_cast<const uint4*>(a.A2 + (size_t)j * R + o * 8)) : make_uint4(0u, 0u, 0u, 0u);
       }
     };
@@ -221,7 +226,7 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     }
     // this thread's entry of a tile's bias, fetched one tile ahead (its latency must not sit between two tiles)
     auto bias_load = [&](int nt) -> float {
-      const int j = nt * NT + et;
+      const int j = (nt0 + nt) * NT + et;
       return (a.bias && nt < ntile && j < a.n_out) ? __bfloat162float(a.bias[j]) : 0.f;
     };
     float bias_next = bias_load(g);
@@ -283,8 +288,8 @@ gate_fn_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
       fence_proxy_async();
       named_bar_sync(2 + 2 * g, EPI_THREADS);
       if (et == 0) {
-        tma_store_2d(&tm_out, smem_u32(stg), nt * NT, n0);
-        if (nt * NT + 64 < a.n_out) tma_store_2d(&tm_out, smem_u32(stg) + TT * 128, nt * NT + 64, n0);
+        tma_store_2d(&tm_out, smem_u32(stg), (nt0 + nt) * NT, n0);
+        if ((nt0 + nt) * NT + 64 < a.n_out) tma_store_2d(&tm_out, smem_u32(stg) + TT * 128, (nt0 + nt) * NT + 64, n0);
         tma_store_commit();
       }
     }
@@ -445,6 +450,17 @@ static bool map_2d(CUtensorMap* m, const void* ptr, size_t rows, size_t cols, in
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+// SMs of the current device (looked up once per device)
+static int sm_count_gfn() {
+  static std::atomic<int> cached[64] = {};
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if ((n = cached[dev].load()) > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  cached[dev].store(n);
+  return n;
+}
+
 template <int R>
 static int launch_tc(const Ctx& c, int d_model, const void* x, const void* A1, const void* A2, const void* bias,
                      void* gate, size_t N, int n_out) {
@@ -461,8 +477,15 @@ static int launch_tc(const Ctx& c, int d_model, const void* x, const void* A1, c
     raised[dev].store(true);
   }
   GArgs a{(const bf16*)A2, (const bf16*)bias, (int)N, d_model, n_out, c.dev_status};
+  // fewer token tiles than the SMs can hold (two blocks each for rank <= 32): share each tile's outputs out over up to 8
+  // blocks, every one of them with output tiles of its own
+  const size_t tiles = (N + TT - 1) / TT;
+  const int ntile_all = (n_out + NT - 1) / NT, room = (R <= 32 ? 2 : 1) * sm_count_gfn();
+  int ysplit = (int)std::min<size_t>(8, std::max<size_t>(1, room / tiles));
+  ysplit = std::min(ysplit, ntile_all);
+  ysplit = (ntile_all + ((ntile_all + ysplit - 1) / ysplit) - 1) / ((ntile_all + ysplit - 1) / ysplit);  // (no empty block)
   LAWCAT_LAUNCH("gate_fn_tc", c.stream,
-                gate_fn_tc_kernel<R><<<(unsigned)((N + TT - 1) / TT), THREADS, L::BYTES, c.stream>>>(tx, ta1, to, a));
+                gate_fn_tc_kernel<R><<<dim3((unsigned)tiles, (unsigned)ysplit), THREADS, L::BYTES, c.stream>>>(tx, ta1, to, a));
   LAWCAT_CHECK_LAUNCH();
   return LAWCAT_OK;
 }

@@ -46,6 +46,7 @@ def run(B, T, H, d, gd, dm, rank, dtype="bf16", bias=True, chunk=0, cfg=900, exp
     (9, 128, 2, 128, 0, 320),    # whole tiles only; five stages (more than the ring holds)
     (15, 70, 8, 64, 1, 72),      # one decay per head: 8 outputs; hidden width 72 = one stage and an eighth
     (21, 50, 4, 128, 0, 1024),   # 16 stages, 512 outputs
+    (8, 1024, 10, 128, 0, 64),   # 64 token tiles, 10 output tiles: a token tile's outputs are shared out 3 + 3 + 3 + 1
 ])
 def test_tensor_core_kernel(rank, B, T, H, d, gd, dm):
     """More than 1024 tokens: the tensor-core kernel."""
