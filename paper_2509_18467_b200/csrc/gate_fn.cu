@@ -4,7 +4,7 @@
 // written as the [B, T, H, gate_dim] gate tensor the layer consumes (n_out = H * gate_dim); the sigmoid and the power
 // 1 / tau are applied where the logits are read.
 //
-// Tensor-core kernel (bf16 storage, rank 16 / 32 / 64 / 128): one thread block per 128 tokens, three roles.
+// Tensor-core kernel (bf16 storage, rank 16 / 32 / 64 / 128): one thread block per 128 tokens, three roles (10 warps).
 //   copy warp      first layer: x tiles [128 tokens x 64 hidden channels] and A1 tiles [rank x 64] through a ring of
 //                  stages (TMA, 128-byte swizzle)
 //   product warp   H = X A1^T accumulated over d_model in tensor memory (M = 128, N = rank); then per 128 outputs
@@ -24,9 +24,11 @@
 // its copies land, frees its tensor memory and reports LAWCAT_ERR_TIMEOUT through dev_status.
 //
 // Few tokens (a decode step, a short call; bf16, widths multiples of 8): one block of the tensor-core kernel walks its
-// 64 stages and 32 output tiles one after the other, about 50 us whatever the number of tokens. Up to a few hundred tokens
+// 64 stages and 32 output tiles one after the other, about 50 us whatever the number of tokens. Up to 1024 tokens
 // gate_fn_small_kernel takes over: one thread block per token (or per four), both layers on the CUDA cores in fp32 with
 // the bottleneck activations in shared memory, every load a 16-byte one and many in flight; the weights come from L2.
+// Above that, while there are fewer token tiles than the SMs hold blocks, the output tiles of a token tile are shared out
+// over several blocks (gridDim.y), each of which repeats the first layer.
 //
 // Exact kernels (any storage type and shape): fp32 accumulation on the CUDA cores, h in fp32 scratch.
 #include <cuda.h>
