@@ -12,6 +12,7 @@ Workloads (seeded synthetic inputs of `paper_2509_18467_b200.inputs`, through th
   c5-decode             one recurrent `lawcat_decode_step` for B = 64 sequences
   c3-gate-fn            the gate function in front of the c3 layer: one `lawcat_gate_fn_fwd` (hidden states of width 4096 ->
                         rank 32 -> 4096 gate logits per token) over the 32768 tokens
+  c5-decode-gate-fn     the same gate function for the one new token of each of the B = 64 sequences of c5-decode
 Prints ONE JSON line (rank 0). N > 1 runs N independent replicas (the layer has no inter-GPU exchange), one process per
 GPU; the time is the max over ranks. Started without a launcher, `--gpus N` starts the N ranks itself.
 
@@ -40,7 +41,7 @@ UNIT = "tokens/s"
 LAYER_NAMES = ["q", "k", "v", "gate", "w_q", "w_k", "W"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 SWEEP_T = (1024, 4096, 16384, 65536, 131072)
-WORKLOADS = ["c1", "c2", "c3", "c4", "c5-decode"] + [f"c5-T{t}" for t in SWEEP_T] + ["c3-gate-fn"]
+WORKLOADS = ["c1", "c2", "c3", "c4", "c5-decode"] + [f"c5-T{t}" for t in SWEEP_T] + ["c3-gate-fn", "c5-decode-gate-fn"]
 # the gate function in front of the headline layer: hidden width of the 7B model, the rank the paper settles on
 GATE_FN = {"d_model": 4096, "rank": 32}
 
@@ -51,11 +52,13 @@ def workload_shape(name: str) -> I.LayerShape:
         return dataclasses.replace(I.CONFIGS["c3"], T=T, config_id=5, name=f"c5-mistral-7b-T{T}")
     if name == "c3-gate-fn":
         return dataclasses.replace(I.CONFIGS["c3"], name="c3-gate-fn-mistral-7b-T32768")
+    if name == "c5-decode-gate-fn":
+        return dataclasses.replace(I.CONFIGS["c5-decode"], name="c5-decode-gate-fn-mistral-7b-B64")
     return I.CONFIGS[name]
 
 
 def workload_kind(name: str) -> str:
-    return {"c4": "train", "c5-decode": "decode", "c3-gate-fn": "gatefn"}.get(name, "prefill")
+    return {"c4": "train", "c5-decode": "decode", "c3-gate-fn": "gatefn", "c5-decode-gate-fn": "gatefn"}.get(name, "prefill")
 
 
 def metric_name(kind: str) -> str:
